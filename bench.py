@@ -1,0 +1,366 @@
+#!/usr/bin/env python
+"""Throughput of the SFB minibatch step (samples/s) at the paper-scale MLR shape, with the update product's
+roofline fraction, an end-to-end (host buffers) figure and the CPU oracle timed beside it.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--precision bf16|fp32] [--workload mlr_large]
+    python bench.py --impl reference ...      # times the fp64 CPU oracle on a bounded sample instead
+
+A step is one pass of the whole hot path over one minibatch of K = P*B synthetic samples: pack, forward
+product, softmax-minus-onehot, gather, fused rank-K update of W.  Prints ONE JSON line on rank 0.
+With N > 1 (torchrun) every rank runs an independent replica on its own minibatches: the path has no
+cross-GPU exchange, so the aggregate is N replicas ("weak" scaling) and no collective is on the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import sfb_inputs as I  # noqa: E402
+
+METRIC = "sfb_step_samples_per_sec"
+UNIT = "samples/s"
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ----------------------------------------------------------------------------------------------------------
+# CPU oracle on a bounded sample of the workload
+# ----------------------------------------------------------------------------------------------------------
+def oracle_sample_setup(wl, budget_s):
+    """A slab of the workload the oracle can step in about ``budget_s`` seconds: all K samples and the full
+    feature dimension against the first J' rows of W (softmax over J' classes).  Cost is linear in rows, so
+    samples/s for the full matrix is the slab's figure times J'/J."""
+    from oracle import sfb_oracle as O  # the one place outside tests/ and smoke() that runs the oracle
+
+    def make(rows):
+        sub = I.scaled(wl, wl.name + f"_rows{rows}", rows=rows)
+        W = I.initial_W(sub)
+        inp = I.step_inputs(sub, 0)
+        if sub.model == I.MLR:
+            inp.labels = (inp.labels % rows).astype(np.int32)
+        L = O.lipschitz_power_iteration(W) if sub.model == I.SC else None
+
+        def step():
+            return O.sfb_step(sub.model, W, inp.X, inp.Y, inp.labels, workers=sub.workers, eta=sub.eta,
+                              margin=sub.dml_margin, lam=sub.sc_lambda, L=L, iters=sub.sc_iters,
+                              prox=(sub.model == I.SC))
+        return step
+
+    probe_rows = int(min(wl.rows, 2048))
+    probe = make(probe_rows)
+    probe()
+    t0 = time.perf_counter()
+    probe()
+    per_row = (time.perf_counter() - t0) / probe_rows             # seconds per row of W on this machine
+    rows = int(max(probe_rows, min(wl.rows, budget_s / per_row)))
+    return make(rows), rows
+
+
+def cores_used():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max((d.get("num_threads", 1) for d in threadpool_info()), default=1)
+        return int(n)
+    except Exception:
+        return len(os.sched_getaffinity(0))
+
+
+def time_oracle(wl, steps, warmup, budget_s):
+    step, rows = oracle_sample_setup(wl, budget_s)
+    for _ in range(warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    dt = (time.perf_counter() - t0) / steps
+    full = dt * wl.rows / rows                                    # cost is linear in the rows of W
+    sample = (f"oracle sfb_step on rows [0,{rows}) of W ({rows}/{wl.rows} of the matrix), all K={wl.K} "
+              f"samples, full feature dim; time scaled by {wl.rows}/{rows}")
+    return wl.K / full, dt, sample
+
+
+# ----------------------------------------------------------------------------------------------------------
+def clocks_sampler(index):
+    f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+    q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+    try:
+        p = subprocess.Popen(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-lms", "50",
+                              "-i", str(index)], stdout=f, stderr=subprocess.DEVNULL)
+    except Exception:
+        return None, f
+    return p, f
+
+
+def clocks_summary(p, f):
+    out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+    if p is None:
+        return out
+    p.terminate()
+    try:
+        p.wait(timeout=5)
+    except Exception:
+        p.kill()
+    f.flush()
+    f.seek(0)
+    sm, mx, reasons = [], [], set()
+    names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+    for line in f.read().splitlines():
+        parts = [x.strip() for x in line.split(",")]
+        if len(parts) < 7:
+            continue
+        try:
+            sm.append(float(parts[0]))
+            mx.append(float(parts[1]))
+        except ValueError:
+            continue
+        for nme, v in zip(names, parts[3:7]):
+            if v.lower().startswith("active"):
+                reasons.add(nme)
+    f.close()
+    os.unlink(f.name)
+    if sm:
+        out["sm_mhz"] = float(np.median(sm))
+        out["sm_max_mhz"] = float(max(mx))
+        out["samples"] = len(sm)
+    out["reasons"] = sorted(reasons)
+    return out
+
+
+# ----------------------------------------------------------------------------------------------------------
+def run_reference(args, wl, rank):
+    if rank != 0:
+        return
+    budget = 150.0 / max(1, args.steps + args.warmup)
+    value, dt, sample = time_oracle(wl, args.steps, args.warmup, budget)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(wl, "f64"),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores_used(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(wl, dtype):
+    return {"workload": wl.name, "model": ["mlr", "dml", "sc"][wl.model], "rows": wl.rows, "cols": wl.cols,
+            "workers_P": wl.workers, "batch_B": wl.batch, "K": wl.K, "eta": wl.eta, "operands": dtype,
+            "master_W": "f32", "l2": "inputs_larger_than_l2" if wl.rows * wl.cols * 4 > 2 * 126e6
+            else "l2_flushed_between_steps"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="sfb", choices=["sfb", "reference"])
+    ap.add_argument("--precision", default="bf16", choices=["bf16", "fp32"])
+    ap.add_argument("--workload", default="mlr_large", choices=sorted(I.WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    wl = I.WORKLOADS[args.workload]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, wl, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_1409_5705_b200 as S
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the SFB path has no CPU fallback")
+    S.build()
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl")
+    dev = torch.device("cuda", local)
+    prec = S.PREC_BF16 if args.precision == "bf16" else S.PREC_FP32
+    peaks = load_peaks()
+
+    # ---- synthetic state: W ~ the workload's init distribution, drawn on the device; minibatches from the
+    # seeded input module (each rank its own step indices)
+    g = torch.Generator(device=dev)
+    g.manual_seed(1234 + rank)
+    W = torch.empty((wl.rows, wl.cols), dtype=torch.float32, device=dev)
+    std = {"normal": wl.w_std, "dml": 1.0 / math.sqrt(wl.cols), "zeros": 0.0, "unit_columns": 1.0}[wl.w_init]
+    for r0 in range(0, wl.rows, 65536):
+        blk = W[r0:r0 + 65536]
+        if std == 0.0:
+            blk.zero_()
+        else:
+            blk.normal_(0.0, std, generator=g)
+    L = 0.0
+    if wl.w_init == "unit_columns":
+        W /= W.norm(dim=0, keepdim=True)
+        L = float(torch.linalg.matrix_norm(W, 2) ** 2)
+    nb = 4
+    true_dict = I.sc_true_dictionary(wl) if wl.model == I.SC else None
+    batches = [I.step_inputs(wl, rank * 1000 + t, true_dict) for t in range(nb)]
+    dX = [torch.from_numpy(b.X).to(dev) for b in batches]
+    dY = [None if b.Y is None else torch.from_numpy(b.Y).to(dev) for b in batches]
+    dL = [None if b.labels is None else torch.from_numpy(b.labels).to(dev) for b in batches]
+    hX = [torch.from_numpy(b.X).pin_memory() for b in batches]
+    hY = [None if b.Y is None else torch.from_numpy(b.Y).pin_memory() for b in batches]
+    hL = [None if b.labels is None else torch.from_numpy(b.labels).pin_memory() for b in batches]
+
+    cfg = S.make_config(wl.model, wl.rows, wl.cols, wl.workers, wl.batch, wl.eta, prec, dml_margin=wl.dml_margin,
+                        sc_lambda=wl.sc_lambda, sc_ista_iters=wl.sc_iters, sc_lipschitz=L,
+                        sc_prox=1 if wl.model == I.SC else 0)
+    ctx = S.Context(cfg, W)
+    flusher = None
+    if wl.rows * wl.cols * 4 <= 2 * 126e6:
+        flusher = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def phased_step(i, ev=None):
+        k = i % nb
+        if flusher is not None:
+            flusher.zero_()
+        if ev is not None:
+            ev[0].record()
+        ctx.sfb_compute_factors(-1, dX[k], dY[k], dL[k])
+        if ev is not None:
+            ev[1].record()
+        ctx.sfb_gather_factors()
+        if ev is not None:
+            ev[2].record()
+        ctx.sfb_apply_update()
+        if ev is not None:
+            ev[3].record()
+
+    # ---- device-resident timing
+    for i in range(args.warmup):
+        phased_step(i)
+    launches0 = ctx.sfb_get_stats().kernel_launches
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    barrier()
+    sampler, sfile = clocks_sampler(local) if rank == 0 else (None, None)
+    t_start = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    for i in range(args.steps):
+        phased_step(i, evs[i])
+    t_end.record()
+    barrier()
+    clocks = clocks_summary(sampler, sfile) if rank == 0 else None
+    total_ms = t_start.elapsed_time(t_end)
+    launches = ctx.sfb_get_stats().kernel_launches - launches0
+    status = ctx.sfb_get_status()
+    ms_f = sum(e[0].elapsed_time(e[1]) for e in evs) / args.steps
+    ms_g = sum(e[1].elapsed_time(e[2]) for e in evs) / args.steps
+    ms_u = sum(e[2].elapsed_time(e[3]) for e in evs) / args.steps
+
+    # ---- end to end: host minibatch -> sfb_step_host -> loss back on the host, every step
+    for i in range(3):
+        ctx.sfb_step_host(hX[i % nb], hY[i % nb], hL[i % nb])
+    barrier()
+    e2e_steps = args.steps
+    t0 = time.perf_counter()
+    loss = 0.0
+    for i in range(e2e_steps):
+        loss, _ = ctx.sfb_step_host(hX[i % nb], hY[i % nb], hL[i % nb])
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+
+    tms = torch.tensor([total_ms, e2e_s * 1e3], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms = float(tms[0]), float(tms[1])
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    K = wl.K
+    value = world * K * args.steps / (total_ms * 1e-3)
+    e2e_value = world * K * e2e_steps / (e2e_ms * 1e-3)
+    h2d = K * wl.in_dim * 4 + (K * wl.cols * 4 if wl.model == I.DML else 0) + (K * 4 if wl.model != I.SC else 0)
+
+    # ---- roofline of the dominant kernel: the fused update  W += -eta U^T V  (one launch per step)
+    esz = 2 if prec == S.PREC_BF16 else 4
+    upd_flops = 2.0 * wl.rows * wl.cols * K
+    upd_bytes = 8.0 * wl.rows * wl.cols + K * (wl.rows + wl.cols) * esz       # W read + written, U and V read once
+    if prec == S.PREC_BF16 and wl.model == I.MLR:
+        upd_bytes += 2.0 * wl.rows * wl.cols                                  # bf16 copy of W for the next forward
+    if prec == S.PREC_BF16:
+        t_flop = upd_flops / (peaks["bf16_tflops_sustained"] * 1e12)
+        t_mem = upd_bytes / (peaks["hbm_gbs"] * 1e9)
+        if t_mem >= t_flop:
+            roof = {"bound": "hbm", "achieved": upd_bytes / (ms_u * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s"}
+        else:
+            roof = {"bound": "tensor", "achieved": upd_flops / (ms_u * 1e-3) / 1e12,
+                    "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s"}
+    else:
+        # fp32 FMA pipe: 148 SMs x 128 lanes x 2 flop x max SM clock
+        peak = 148 * 128 * 2 * (clocks.get("sm_max_mhz") or 1965.0) * 1e6 / 1e12
+        roof = {"bound": "alu", "achieved": upd_flops / (ms_u * 1e-3) / 1e12, "peak": peak, "unit": "TFLOP/s"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = None
+    roof["kernel"] = "fused rank-K update (sfb_apply_update)"
+    roof["ms"] = ms_u
+    roof["peaks"] = peaks["source"]
+    roof["update_tflops"] = upd_flops / (ms_u * 1e-3) / 1e12
+    roof["algorithmic_bytes"] = upd_bytes
+    roof["algorithmic_flops"] = upd_flops
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        v, dt, sample = time_oracle(wl, 1, 0, 15.0)
+        cpu = {"value": v, "unit": UNIT, "cores": cores_used(), "kind": "oracle", "sample": sample,
+               "sample_seconds": dt}
+
+    one_copy = K * (wl.rows + wl.cols) * esz
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if prec == S.PREC_BF16 else "f32",
+            "data": "synthetic", "config": workload_config(wl, "bf16" if prec == S.PREC_BF16 else "f32"),
+            "roofline": roof, "cpu_baseline": cpu,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 8,
+                    "ms_per_step": e2e_ms / e2e_steps, "last_loss": loss},
+            "gpu_launches": int(launches), "clocks": clocks,
+            "phases_ms": {"factors": ms_f, "gather": ms_g, "update": ms_u},
+            "bytes": {"sf_gather_one_copy": one_copy,
+                      "sf_broadcast_p2p": wl.workers * (wl.workers - 1) * wl.batch * (wl.rows + wl.cols) * esz,
+                      "dense_sync": wl.workers * wl.rows * wl.cols * 4,
+                      "dense_over_sf": wl.workers * wl.rows * wl.cols * 4 / one_copy},
+            "status_word": status}
+    print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,152 @@
+/*
+ * sfb.h -- C ABI of the B200 (sm_100a) Sufficient Factor Broadcasting step.
+ *
+ * One minibatch step of the paper's computation model (Section 3, Figure 1; mini-batch form in Section 3,
+ * "Mini-batch proximal SGD"): P logical workers hold B samples each; every worker turns its samples into
+ * sufficient-factor pairs (u_i, v_i) against the same parameter matrix W (bulk-synchronous consistency,
+ * Section 4.1); the K = P*B pairs are gathered into one buffer (the on-device form of the broadcast), and
+ * the reconstructed update is applied:   W <- prox( W - eta * sum_{i<K} u_i v_i^T ).
+ *
+ * Conventions that hold for every call:
+ *  - "dev" pointers are CUDA device pointers, "host" pointers are host memory.  All buffers are owned by
+ *    the caller; the library borrows them.  W is updated in place.  The context is freed only by
+ *    sfb_destroy.  The library allocates no device memory: everything it needs is carved from the
+ *    caller's workspace (size from sfb_workspace_bytes).
+ *  - W is fp32, row-major [rows][cols]:  MLR classes x features, DML latent x features, SC features x atoms.
+ *    cols must be a multiple of 4 and every device pointer 16-byte aligned.
+ *  - Samples are worker-major: global pair index i = p*B + b for sample b of worker p.
+ *  - All work is enqueued on config.stream.  Calls return 0 or a negative sfb_error; nothing aborts or traps.
+ *    Errors detected on the device (a class id out of range, a pipeline wait that ran out) set bits of a
+ *    device status word, read with sfb_get_status.
+ *  - One context per stream; calls on one context are not re-entrant.
+ */
+#ifndef SFB_H_
+#define SFB_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sfb_ctx sfb_ctx;
+
+enum sfb_model { SFB_MLR = 0, SFB_DML = 1, SFB_SC = 2 };
+
+/* Operand precision of the matrix products.  The master copy of W is fp32 in both modes.
+ * SFB_PREC_BF16: tensor-core products on bf16 operands with fp32 accumulation.
+ * SFB_PREC_FP32: fp32 operands, fp32 FMA accumulation. */
+enum sfb_precision { SFB_PREC_BF16 = 0, SFB_PREC_FP32 = 1 };
+
+enum sfb_error {
+  SFB_OK = 0,
+  SFB_ERR_ARG = -1,          /* null pointer, bad enum, non-positive size                      */
+  SFB_ERR_ALIGN = -2,        /* a pointer is not 16-byte aligned                               */
+  SFB_ERR_SHAPE = -3,        /* cols not a multiple of 4, worker index out of range, ...       */
+  SFB_ERR_WORKSPACE = -4,    /* workspace smaller than sfb_workspace_bytes reports             */
+  SFB_ERR_CUDA = -5,         /* a CUDA runtime call failed (see sfb_last_cuda_error)           */
+  SFB_ERR_ARCH = -6,         /* the current device is not compute capability 10.x              */
+  SFB_ERR_TIMEOUT = -7,      /* a bounded device-side wait gave up (status word)               */
+  SFB_ERR_LABEL_RANGE = -8,  /* a class id outside [0, rows) was skipped (status word)         */
+  SFB_ERR_STATE = -9,        /* call order: gather before all workers committed, ...           */
+  SFB_ERR_UNSUPPORTED = -10  /* this model / precision combination is not built                */
+};
+
+/* Bits of the device status word. */
+#define SFB_STATUS_LABEL_RANGE 0x1u
+#define SFB_STATUS_TIMEOUT     0x2u
+
+typedef struct sfb_config {
+  int32_t model;          /* enum sfb_model                                                            */
+  int32_t precision;      /* enum sfb_precision                                                        */
+  int64_t rows, cols;     /* shape of W                                                                */
+  int32_t workers;        /* P                                                                         */
+  int32_t batch;          /* B; K = P*B                                                                */
+  float   eta;            /* W <- W - eta * sum u v^T (a plain sum: fold 1/B or 1/K into eta)          */
+  float   dml_margin;     /* hinge margin of dissimilar pairs (Section 2, DML)                         */
+  float   sc_lambda;      /* l1 weight of the sparse coder                                             */
+  int32_t sc_ista_iters;  /* ISTA iterations per sample, from a = 0                                    */
+  float   sc_lipschitz;   /* step is 1/L; <= 0: the library estimates L = ||W||_2^2 by 50 power
+                             iterations at the start of every step                                     */
+  int32_t sc_prox;        /* 0 none | 1 rescale columns of norm > 1 to norm 1 (Figure 3)               */
+  void*   stream;         /* cudaStream_t                                                              */
+} sfb_config;
+
+typedef struct sfb_stats {
+  int64_t steps;              /* completed sfb_step / sfb_apply_update calls                           */
+  int64_t samples;            /* pairs applied                                                         */
+  double  flops;              /* matrix-product flops issued (2*m*n*k each)                            */
+  double  gather_bytes;       /* bytes of gathered factors, one copy: K*(rows+cols)*element size        */
+  double  gather_bytes_p2p;   /* the paper's peer-to-peer count: P*(P-1)*B*(rows+cols)*element size     */
+  double  dense_sync_bytes;   /* what full-matrix sync would move: P*rows*cols*4 (Section 5 cost table) */
+  float   ms_factors, ms_gather, ms_update;  /* device time of the last step's phases (CUDA events)     */
+  float   last_loss;          /* MLR: mean over the last step's K samples of -log p(y_i); else 0        */
+  float   sc_lipschitz;       /* SC: the L = ||W||_2^2 the coder used in the last step                  */
+  int64_t kernel_launches;    /* kernels this library has launched in this process                      */
+} sfb_stats;
+
+/* Bytes of device workspace a context with this config needs.  Host-only; no CUDA call. */
+int sfb_workspace_bytes(const sfb_config* cfg, size_t* out_bytes);
+
+/* Create a context over caller-owned W_dev [rows x cols] fp32 and workspace_dev.  Enqueues the set-up
+ * work (status word clear, bf16 shadow of W in bf16 mode) on cfg->stream.  Problem (P), Section 2. */
+int sfb_init(const sfb_config* cfg, float* W_dev, void* workspace_dev, size_t workspace_bytes, sfb_ctx** out);
+
+/* Sufficient factors of worker `worker` (0..P-1; X_dev is that worker's [B x in_dim] fp32 block), or of all
+ * P workers at once (worker = -1; X_dev is [K x in_dim]).  in_dim = cols (MLR, DML) or rows (SC).
+ *   MLR: labels_dev = int32 class ids;   u = softmax(W x) - onehot(y), v = x       (Sections 1, 2.1)
+ *   DML: Y_dev = pair partner, labels_dev = 1 similar / 0 dissimilar;
+ *        v = x - y, u = 2 W v (similar), -2 W v if ||W v||^2 < margin else 0       (Section 2, DML)
+ *   SC : v = a = ISTA code of x, u = W a - x                                        (Figure 3)
+ * Factors are written at the worker's row offset p*B of the gathered buffers. */
+int sfb_compute_factors(sfb_ctx* ctx, int32_t worker, const float* X_dev, const float* Y_dev,
+                        const int32_t* labels_dev);
+
+/* The broadcast of Section 3 as an on-device gather: after it, U [K x rows] and V [K x cols] of all P workers
+ * sit in one buffer in the operand layout of the update.  Fails with SFB_ERR_STATE unless every worker has
+ * computed its factors since the last update.  Accounts the bytes of Section 5's cost table. */
+int sfb_gather_factors(sfb_ctx* ctx);
+
+/* Reconstruct and apply:  W <- W - eta * U^T V  in one pass over W, then the proximal operator (SC, when
+ * sc_prox = 1).  Section 2.1 (proximal SGD) and Figure 1. */
+int sfb_apply_update(sfb_ctx* ctx);
+
+/* compute_factors(all workers) + gather + apply_update for K samples resident on the device. */
+int sfb_step(sfb_ctx* ctx, const float* X_dev, const float* Y_dev, const int32_t* labels_dev);
+
+/* The same step for callers whose minibatch lives in HOST memory (pinned memory recommended): copies
+ * X_host [K x in_dim] (and Y_host, labels_host when the model uses them) to staging buffers inside the
+ * workspace, runs the step, copies the step's mean loss (MLR; 0 otherwise) and the status word back, and
+ * waits for the stream.  loss_out and status_out may be NULL. */
+int sfb_step_host(sfb_ctx* ctx, const float* X_host, const float* Y_host, const int32_t* labels_host,
+                  float* loss_out, uint32_t* status_out);
+
+/* Full-matrix-synchronisation comparison path (Section 3 "SFB vs client-server", Section 5): every worker
+ * materialises its dense update U_p^T V_p in scratch, the P matrices are summed, and W <- W - eta * sum.
+ * scratch_dev: at least 2*rows*cols*4 bytes.  Same result as sfb_step up to summation order. */
+int sfb_dense_sync_step(sfb_ctx* ctx, const float* X_dev, const float* Y_dev, const int32_t* labels_dev,
+                        float* scratch_dev, size_t scratch_bytes);
+
+/* The gathered factor buffers of the last gather, for inspection.  dtype: 0 = fp32, 1 = bf16.
+ * layout: 0 = pair-major (U [K x ldu], V [K x ldv]); 1 = transposed (U^T [rows x ldu], V^T [cols x ldv]). */
+int sfb_get_factors(sfb_ctx* ctx, const void** U_dev, const void** V_dev, int32_t* dtype, int32_t* layout,
+                    int64_t* ldu, int64_t* ldv);
+
+/* Waits for the stream, then fills the counters. */
+int sfb_get_stats(sfb_ctx* ctx, sfb_stats* out);
+
+/* Waits for the stream, returns the device status word and clears it. */
+int sfb_get_status(sfb_ctx* ctx, uint32_t* status_out);
+
+const char* sfb_strerror(int code);
+
+/* The cudaError_t of the last failed CUDA call made through this context (0 if none). */
+int sfb_last_cuda_error(sfb_ctx* ctx);
+
+int sfb_destroy(sfb_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SFB_H_ */

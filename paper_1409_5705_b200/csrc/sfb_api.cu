@@ -1,0 +1,406 @@
+// C ABI of libsfb: argument checking, workspace carve-up, and the sequencing of one SFB step
+// (Section 3, Figure 1: compute factors -> broadcast/gather -> reconstruct and apply -> prox).
+#include <new>
+
+#include "sfb_internal.h"
+#include "sfb_tc.h"
+
+namespace sfb {
+
+int64_t g_kernel_launches = 0;
+
+static size_t up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+Layout make_layout(const sfb_config& c) {
+  Layout L{};
+  const size_t K = static_cast<size_t>(c.workers) * c.batch;
+  const size_t rows = c.rows, cols = c.cols;
+  const size_t in_dim = c.model == SFB_SC ? rows : cols;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += up(bytes); return o; };
+  L.status = take(sizeof(uint32_t));
+  L.scalars = take(sizeof(Scalars));
+  L.loss = take(K * 4);
+  L.stageX = take(K * in_dim * 4);
+  L.stageY = take(c.model == SFB_DML ? K * cols * 4 : 0);
+  L.stageL = take(K * 4);
+  L.colpart = take(c.model == SFB_SC ? static_cast<size_t>(kProxSlabs) * cols * 8 : 0);
+  L.pib = take(c.model == SFB_SC ? cols * 4 : 0);
+  L.piy = take(c.model == SFB_SC ? rows * 4 : 0);
+  L.Kp = static_cast<int64_t>(K);
+  L.colsb = static_cast<int64_t>(cols);
+  if (c.precision == SFB_PREC_FP32) {
+    L.V = take(K * cols * 4);
+    L.U = take(K * rows * 4);
+  } else {
+    tc_extend_layout(c, L, off);
+  }
+  L.total = off;
+  return L;
+}
+
+}  // namespace sfb
+
+using namespace sfb;
+
+#define CK(call)                                        \
+  do {                                                  \
+    cudaError_t e__ = (call);                           \
+    if (e__ != cudaSuccess) {                           \
+      ctx->last_cuda = static_cast<int>(e__);           \
+      return SFB_ERR_CUDA;                              \
+    }                                                   \
+  } while (0)
+
+static bool al16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int check_config(const sfb_config* c) {
+  if (!c) return SFB_ERR_ARG;
+  if (c->model < SFB_MLR || c->model > SFB_SC) return SFB_ERR_ARG;
+  if (c->precision != SFB_PREC_BF16 && c->precision != SFB_PREC_FP32) return SFB_ERR_ARG;
+  if (c->rows <= 0 || c->cols <= 0 || c->workers <= 0 || c->batch <= 0) return SFB_ERR_ARG;
+  if (c->workers > 64) return SFB_ERR_SHAPE;
+  if (c->cols % 4 != 0) return SFB_ERR_SHAPE;
+  if (c->rows > (1LL << 30) || c->cols > (1LL << 30)) return SFB_ERR_SHAPE;
+  if (static_cast<int64_t>(c->workers) * c->batch > (1 << 20)) return SFB_ERR_SHAPE;
+  if (c->model == SFB_SC && c->sc_ista_iters < 0) return SFB_ERR_ARG;
+  if (c->model == SFB_SC && !(c->sc_lambda >= 0.f)) return SFB_ERR_ARG;
+  if (c->sc_prox < 0 || c->sc_prox > 1) return SFB_ERR_ARG;
+  return SFB_OK;
+}
+
+extern "C" int sfb_workspace_bytes(const sfb_config* cfg, size_t* out_bytes) {
+  if (!out_bytes) return SFB_ERR_ARG;
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  *out_bytes = make_layout(*cfg).total;
+  return SFB_OK;
+}
+
+extern "C" int sfb_init(const sfb_config* cfg, float* W_dev, void* workspace_dev, size_t workspace_bytes,
+                        sfb_ctx** out) {
+  if (!out) return SFB_ERR_ARG;
+  *out = nullptr;
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  if (!W_dev || !workspace_dev) return SFB_ERR_ARG;
+  if (!al16(W_dev) || (reinterpret_cast<uintptr_t>(workspace_dev) & (kAlign - 1)) != 0) return SFB_ERR_ALIGN;
+  Layout lay = make_layout(*cfg);
+  if (workspace_bytes < lay.total) return SFB_ERR_WORKSPACE;
+  int dev = 0, major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return SFB_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return SFB_ERR_CUDA;
+  if (major != 10) return SFB_ERR_ARCH;
+
+  sfb_ctx* ctx = new (std::nothrow) sfb_ctx();
+  if (!ctx) return SFB_ERR_ARG;
+  ctx->cfg = *cfg;
+  ctx->lay = lay;
+  ctx->W = W_dev;
+  ctx->ws = static_cast<char*>(workspace_dev);
+  ctx->stream = static_cast<cudaStream_t>(cfg->stream);
+  ctx->K = static_cast<int64_t>(cfg->workers) * cfg->batch;
+  ctx->in_dim = cfg->model == SFB_SC ? cfg->rows : cfg->cols;
+  ctx->committed = 0;
+  ctx->gathered = false;
+  ctx->last_cuda = 0;
+  ctx->stats = sfb_stats{};
+  ctx->tc = nullptr;
+  for (auto& e : ctx->ev) e = nullptr;
+  for (auto& e : ctx->ev) {
+    cudaError_t ce = cudaEventCreate(&e);
+    if (ce != cudaSuccess) { sfb_destroy(ctx); return SFB_ERR_CUDA; }
+  }
+  // status word, scalars and per-sample losses are the first three (contiguous) regions
+  cudaError_t ce = cudaMemsetAsync(ctx->ws + lay.status, 0, lay.stageX - lay.status, ctx->stream);
+  if (ce != cudaSuccess) { sfb_destroy(ctx); return SFB_ERR_CUDA; }
+  if (cfg->model == SFB_SC && cfg->sc_lipschitz > 0.f) {
+    ce = set_lipschitz(ctx->stream, ctx->at<Scalars>(lay.scalars), cfg->sc_lipschitz);
+    if (ce != cudaSuccess) { sfb_destroy(ctx); return SFB_ERR_CUDA; }
+  }
+  if (cfg->precision == SFB_PREC_BF16) {
+    rc = tc_init(ctx);
+    if (rc) { sfb_destroy(ctx); return rc; }
+  }
+  *out = ctx;
+  return SFB_OK;
+}
+
+extern "C" int sfb_destroy(sfb_ctx* ctx) {
+  if (!ctx) return SFB_ERR_ARG;
+  for (auto& e : ctx->ev)
+    if (e) cudaEventDestroy(e);
+  tc_destroy(ctx);
+  delete ctx;
+  return SFB_OK;
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// fp32-operand path
+// ---------------------------------------------------------------------------------------------------------
+static int factors_fp32(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float* Y,
+                        const int32_t* labels) {
+  const sfb_config& c = ctx->cfg;
+  const int64_t rows = c.rows, cols = c.cols;
+  float* V = ctx->at<float>(ctx->lay.V) + off * cols;
+  float* U = ctx->at<float>(ctx->lay.U) + off * rows;
+  Scalars* sc = ctx->at<Scalars>(ctx->lay.scalars);
+  uint32_t* status = ctx->at<uint32_t>(ctx->lay.status);
+  cudaStream_t s = ctx->stream;
+  EpiArgs e{};
+  if (c.model == SFB_MLR || c.model == SFB_DML) {
+    CK(pack_copy(s, V, X, c.model == SFB_DML ? Y : nullptr, n * cols));                 // v = x | x - y
+    e.C = U; e.ldc = rows;
+    CK(sgemm(s, true, true, EPI_STORE, n, rows, cols, V, cols, ctx->W, cols, e));       // z_i = W v_i
+    ctx->stats.flops += 2.0 * n * rows * cols;
+    if (c.model == SFB_MLR)
+      CK(mlr_softmax_rows(s, U, n, rows, labels, ctx->at<float>(ctx->lay.loss) + off, status));
+    else
+      CK(dml_scale_rows(s, U, n, rows, labels, c.dml_margin));
+    return SFB_OK;
+  }
+  // sparse coding: ISTA from a = 0, then u = W a - x, v = a
+  CK(fill_zero(s, V, n * cols));
+  for (int it = 0; it <= c.sc_ista_iters; ++it) {
+    e = EpiArgs{};
+    e.C = U; e.ldc = rows; e.aux = X;
+    CK(sgemm(s, true, true, EPI_SUB, n, rows, cols, V, cols, ctx->W, cols, e));         // r = W a - x
+    ctx->stats.flops += 2.0 * n * rows * cols;
+    if (it == c.sc_ista_iters) break;
+    e = EpiArgs{};
+    e.C = V; e.ldc = cols; e.sc = sc; e.lam = c.sc_lambda;
+    CK(sgemm(s, true, false, EPI_ISTA, n, cols, rows, U, rows, ctx->W, cols, e));       // a <- soft(a - W^T r / L)
+    ctx->stats.flops += 2.0 * n * rows * cols;
+  }
+  return SFB_OK;
+}
+
+static int update_fp32(sfb_ctx* ctx) {
+  const sfb_config& c = ctx->cfg;
+  EpiArgs e{};
+  e.C = ctx->W; e.ldc = c.cols; e.alpha = -c.eta;
+  CK(sgemm(ctx->stream, false, false, EPI_RMW, c.rows, c.cols, ctx->K, ctx->at<float>(ctx->lay.U), c.rows,
+           ctx->at<float>(ctx->lay.V), c.cols, e));
+  return SFB_OK;
+}
+
+// ---------------------------------------------------------------------------------------------------------
+static int check_inputs(sfb_ctx* ctx, const float* X, const float* Y, const int32_t* labels) {
+  if (!ctx || !X) return SFB_ERR_ARG;
+  if (ctx->cfg.model == SFB_DML && (!Y || !labels)) return SFB_ERR_ARG;
+  if (ctx->cfg.model == SFB_MLR && !labels) return SFB_ERR_ARG;
+  if (!al16(X) || (Y && !al16(Y))) return SFB_ERR_ALIGN;
+  return SFB_OK;
+}
+
+extern "C" int sfb_compute_factors(sfb_ctx* ctx, int32_t worker, const float* X_dev, const float* Y_dev,
+                                   const int32_t* labels_dev) {
+  int rc = check_inputs(ctx, X_dev, Y_dev, labels_dev);
+  if (rc) return rc;
+  const sfb_config& c = ctx->cfg;
+  if (worker < -1 || worker >= c.workers) return SFB_ERR_SHAPE;
+  const int64_t off = worker < 0 ? 0 : static_cast<int64_t>(worker) * c.batch;
+  const int64_t n = worker < 0 ? ctx->K : c.batch;
+  if (ctx->committed == 0) {
+    CK(cudaEventRecord(ctx->ev[0], ctx->stream));
+    // the coder's step size comes from the W every worker sees at the start of the step (BSP)
+    if (c.model == SFB_SC && !(c.sc_lipschitz > 0.f))
+      CK(estimate_lipschitz(ctx->stream, ctx->W, c.rows, c.cols, ctx->at<float>(ctx->lay.pib),
+                            ctx->at<float>(ctx->lay.piy), ctx->at<float>(ctx->lay.colpart),
+                            ctx->at<Scalars>(ctx->lay.scalars), 50));
+  }
+  rc = c.precision == SFB_PREC_FP32 ? factors_fp32(ctx, off, n, X_dev, Y_dev, labels_dev)
+                                    : tc_factors(ctx, off, n, X_dev, Y_dev, labels_dev);
+  if (rc) return rc;
+  const uint64_t all = c.workers == 64 ? ~0ull : ((1ull << c.workers) - 1);
+  ctx->committed |= worker < 0 ? all : (1ull << worker);
+  ctx->gathered = false;
+  return SFB_OK;
+}
+
+extern "C" int sfb_gather_factors(sfb_ctx* ctx) {
+  if (!ctx) return SFB_ERR_ARG;
+  const sfb_config& c = ctx->cfg;
+  const uint64_t all = c.workers == 64 ? ~0ull : ((1ull << c.workers) - 1);
+  if (ctx->committed != all) return SFB_ERR_STATE;
+  CK(cudaEventRecord(ctx->ev[1], ctx->stream));
+  // Every worker wrote its pairs at row offset p*B of the shared buffers, so the gathered operands are
+  // complete; what remains is the per-step read-out over all K pairs.
+  if (c.precision == SFB_PREC_BF16) {
+    int rc = tc_gather(ctx);
+    if (rc) return rc;
+  }
+  if (c.model == SFB_MLR)
+    CK(mean_of(ctx->stream, ctx->at<float>(ctx->lay.loss), ctx->K,
+               &ctx->at<Scalars>(ctx->lay.scalars)->loss_mean));
+  const double esz = c.precision == SFB_PREC_FP32 ? 4.0 : 2.0;
+  const double pair = static_cast<double>(c.rows + c.cols) * esz;
+  ctx->stats.gather_bytes += static_cast<double>(ctx->K) * pair;
+  ctx->stats.gather_bytes_p2p += static_cast<double>(c.workers) * (c.workers - 1) * c.batch * pair;
+  ctx->stats.dense_sync_bytes += static_cast<double>(c.workers) * c.rows * c.cols * 4.0;
+  ctx->gathered = true;
+  CK(cudaEventRecord(ctx->ev[2], ctx->stream));
+  return SFB_OK;
+}
+
+static int apply_prox(sfb_ctx* ctx) {
+  const sfb_config& c = ctx->cfg;
+  if (c.model == SFB_SC && c.sc_prox == 1)
+    CK(prox_unit_columns(ctx->stream, ctx->W, c.rows, c.cols, ctx->at<float>(ctx->lay.colpart)));
+  return SFB_OK;
+}
+
+extern "C" int sfb_apply_update(sfb_ctx* ctx) {
+  if (!ctx) return SFB_ERR_ARG;
+  if (!ctx->gathered) return SFB_ERR_STATE;
+  const sfb_config& c = ctx->cfg;
+  int rc = c.precision == SFB_PREC_FP32 ? update_fp32(ctx) : tc_update(ctx);
+  if (rc) return rc;
+  ctx->stats.flops += 2.0 * c.rows * c.cols * ctx->K;
+  rc = apply_prox(ctx);
+  if (rc) return rc;
+  if (c.precision == SFB_PREC_BF16) {
+    rc = tc_after_update(ctx);
+    if (rc) return rc;
+  }
+  CK(cudaEventRecord(ctx->ev[3], ctx->stream));
+  ctx->committed = 0;
+  ctx->gathered = false;
+  ctx->stats.steps += 1;
+  ctx->stats.samples += ctx->K;
+  return SFB_OK;
+}
+
+extern "C" int sfb_step(sfb_ctx* ctx, const float* X_dev, const float* Y_dev, const int32_t* labels_dev) {
+  if (!ctx) return SFB_ERR_ARG;
+  ctx->committed = 0;
+  int rc = sfb_compute_factors(ctx, -1, X_dev, Y_dev, labels_dev);
+  if (rc) return rc;
+  rc = sfb_gather_factors(ctx);
+  if (rc) return rc;
+  return sfb_apply_update(ctx);
+}
+
+extern "C" int sfb_step_host(sfb_ctx* ctx, const float* X_host, const float* Y_host, const int32_t* labels_host,
+                             float* loss_out, uint32_t* status_out) {
+  if (!ctx || !X_host) return SFB_ERR_ARG;
+  const sfb_config& c = ctx->cfg;
+  if (c.model == SFB_DML && (!Y_host || !labels_host)) return SFB_ERR_ARG;
+  if (c.model == SFB_MLR && !labels_host) return SFB_ERR_ARG;
+  float* Xs = ctx->at<float>(ctx->lay.stageX);
+  float* Ys = ctx->at<float>(ctx->lay.stageY);
+  int32_t* Ls = ctx->at<int32_t>(ctx->lay.stageL);
+  CK(cudaMemcpyAsync(Xs, X_host, static_cast<size_t>(ctx->K) * ctx->in_dim * 4, cudaMemcpyHostToDevice, ctx->stream));
+  if (c.model == SFB_DML)
+    CK(cudaMemcpyAsync(Ys, Y_host, static_cast<size_t>(ctx->K) * c.cols * 4, cudaMemcpyHostToDevice, ctx->stream));
+  if (c.model != SFB_SC)
+    CK(cudaMemcpyAsync(Ls, labels_host, static_cast<size_t>(ctx->K) * 4, cudaMemcpyHostToDevice, ctx->stream));
+  int rc = sfb_step(ctx, Xs, c.model == SFB_DML ? Ys : nullptr, c.model != SFB_SC ? Ls : nullptr);
+  if (rc) return rc;
+  float loss = 0.f;
+  uint32_t st = 0;
+  CK(cudaMemcpyAsync(&loss, &ctx->at<Scalars>(ctx->lay.scalars)->loss_mean, 4, cudaMemcpyDeviceToHost, ctx->stream));
+  CK(cudaMemcpyAsync(&st, ctx->at<uint32_t>(ctx->lay.status), 4, cudaMemcpyDeviceToHost, ctx->stream));
+  CK(cudaStreamSynchronize(ctx->stream));
+  if (loss_out) *loss_out = loss;
+  if (status_out) *status_out = st;
+  return SFB_OK;
+}
+
+extern "C" int sfb_dense_sync_step(sfb_ctx* ctx, const float* X_dev, const float* Y_dev, const int32_t* labels_dev,
+                                   float* scratch_dev, size_t scratch_bytes) {
+  if (!ctx || !scratch_dev) return SFB_ERR_ARG;
+  const sfb_config& c = ctx->cfg;
+  if (c.precision != SFB_PREC_FP32) return SFB_ERR_UNSUPPORTED;
+  if (!al16(scratch_dev)) return SFB_ERR_ALIGN;
+  const size_t mat = static_cast<size_t>(c.rows) * c.cols;
+  if (scratch_bytes < 2 * mat * 4) return SFB_ERR_WORKSPACE;
+  ctx->committed = 0;
+  int rc = sfb_compute_factors(ctx, -1, X_dev, Y_dev, labels_dev);
+  if (rc) return rc;
+  rc = sfb_gather_factors(ctx);   // loss read-out and byte accounting; the factors stay per worker below
+  if (rc) return rc;
+  float* sum = scratch_dev;
+  float* one = scratch_dev + mat;
+  const float* U = ctx->at<float>(ctx->lay.U);
+  const float* V = ctx->at<float>(ctx->lay.V);
+  for (int p = 0; p < c.workers; ++p) {
+    // worker p's dense update matrix, as it would be sent to the server
+    EpiArgs e{};
+    e.C = p == 0 ? sum : one; e.ldc = c.cols;
+    CK(sgemm(ctx->stream, false, false, EPI_STORE, c.rows, c.cols, c.batch, U + static_cast<int64_t>(p) * c.batch * c.rows,
+             c.rows, V + static_cast<int64_t>(p) * c.batch * c.cols, c.cols, e));
+    if (p > 0) CK(axpy(ctx->stream, sum, one, 1.f, static_cast<int64_t>(mat)));          // server-side aggregation
+  }
+  CK(axpy(ctx->stream, ctx->W, sum, -c.eta, static_cast<int64_t>(mat)));                 // W <- W - eta * sum_p dW_p
+  ctx->stats.flops += 2.0 * c.rows * c.cols * ctx->K;
+  rc = apply_prox(ctx);
+  if (rc) return rc;
+  CK(cudaEventRecord(ctx->ev[3], ctx->stream));
+  ctx->committed = 0;
+  ctx->gathered = false;
+  ctx->stats.steps += 1;
+  ctx->stats.samples += ctx->K;
+  return SFB_OK;
+}
+
+extern "C" int sfb_get_factors(sfb_ctx* ctx, const void** U_dev, const void** V_dev, int32_t* dtype, int32_t* layout,
+                               int64_t* ldu, int64_t* ldv) {
+  if (!ctx) return SFB_ERR_ARG;
+  if (ctx->cfg.precision == SFB_PREC_FP32) {
+    if (U_dev) *U_dev = ctx->at<float>(ctx->lay.U);
+    if (V_dev) *V_dev = ctx->at<float>(ctx->lay.V);
+    if (dtype) *dtype = 0;
+    if (layout) *layout = 0;
+    if (ldu) *ldu = ctx->cfg.rows;
+    if (ldv) *ldv = ctx->cfg.cols;
+    return SFB_OK;
+  }
+  return tc_get_factors(ctx, U_dev, V_dev, dtype, layout, ldu, ldv);
+}
+
+extern "C" int sfb_get_stats(sfb_ctx* ctx, sfb_stats* out) {
+  if (!ctx || !out) return SFB_ERR_ARG;
+  CK(cudaStreamSynchronize(ctx->stream));
+  if (ctx->stats.steps > 0) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, ctx->ev[0], ctx->ev[1]) == cudaSuccess) ctx->stats.ms_factors = ms;
+    if (cudaEventElapsedTime(&ms, ctx->ev[1], ctx->ev[2]) == cudaSuccess) ctx->stats.ms_gather = ms;
+    if (cudaEventElapsedTime(&ms, ctx->ev[2], ctx->ev[3]) == cudaSuccess) ctx->stats.ms_update = ms;
+    cudaGetLastError();
+    Scalars h{};
+    CK(cudaMemcpy(&h, ctx->at<Scalars>(ctx->lay.scalars), sizeof(h), cudaMemcpyDeviceToHost));
+    ctx->stats.last_loss = h.loss_mean;
+    ctx->stats.sc_lipschitz = h.L;
+  }
+  ctx->stats.kernel_launches = g_kernel_launches;
+  *out = ctx->stats;
+  return SFB_OK;
+}
+
+extern "C" int sfb_get_status(sfb_ctx* ctx, uint32_t* status_out) {
+  if (!ctx || !status_out) return SFB_ERR_ARG;
+  CK(cudaMemcpyAsync(status_out, ctx->at<uint32_t>(ctx->lay.status), 4, cudaMemcpyDeviceToHost, ctx->stream));
+  CK(cudaMemsetAsync(ctx->at<uint32_t>(ctx->lay.status), 0, 4, ctx->stream));
+  CK(cudaStreamSynchronize(ctx->stream));
+  return SFB_OK;
+}
+
+extern "C" int sfb_last_cuda_error(sfb_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }
+
+extern "C" const char* sfb_strerror(int code) {
+  switch (code) {
+    case SFB_OK: return "ok";
+    case SFB_ERR_ARG: return "invalid argument";
+    case SFB_ERR_ALIGN: return "pointer not 16-byte aligned";
+    case SFB_ERR_SHAPE: return "unsupported shape";
+    case SFB_ERR_WORKSPACE: return "workspace or scratch too small";
+    case SFB_ERR_CUDA: return "CUDA runtime error";
+    case SFB_ERR_ARCH: return "device is not compute capability 10.x";
+    case SFB_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+    case SFB_ERR_LABEL_RANGE: return "class id out of range";
+    case SFB_ERR_STATE: return "call out of order";
+    case SFB_ERR_UNSUPPORTED: return "model/precision combination not built";
+    default: return "unknown error";
+  }
+}

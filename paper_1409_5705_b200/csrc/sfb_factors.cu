@@ -1,0 +1,371 @@
+// Bandwidth-bound kernels of the SFB step in fp32: factor packing, the row softmax of multiclass logistic
+// regression, the pair residual of distance metric learning, the column-norm prox of sparse coding and the
+// power iteration that estimates the coder's step size.
+#include "sfb_internal.h"
+
+namespace sfb {
+namespace {
+
+constexpr int kThreads = 256;
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// Block-wide sum in a fixed order (warp shuffles, then warp 0 over the per-warp values).
+template <int NTHREADS>
+__device__ __forceinline__ float block_sum(float v, float* sh) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  v = warp_sum(v);
+  __syncthreads();
+  if (lane == 0) sh[w] = v;
+  __syncthreads();
+  float r = (threadIdx.x < NTHREADS / 32) ? sh[threadIdx.x] : 0.f;
+  if (w == 0) r = warp_sum(r);
+  if (threadIdx.x == 0) sh[0] = r;
+  __syncthreads();
+  return sh[0];
+}
+template <int NTHREADS>
+__device__ __forceinline__ float block_max(float v, float* sh) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  v = warp_max(v);
+  __syncthreads();
+  if (lane == 0) sh[w] = v;
+  __syncthreads();
+  float r = (threadIdx.x < NTHREADS / 32) ? sh[threadIdx.x] : -INFINITY;
+  if (w == 0) r = warp_max(r);
+  if (threadIdx.x == 0) sh[0] = r;
+  __syncthreads();
+  return sh[0];
+}
+
+// v = x (MLR) or v = x - y (DML pair difference, Section 2), 16-byte vectors with a scalar tail.
+__global__ void pack_kernel(float* __restrict__ dst, const float* __restrict__ x, const float* __restrict__ y,
+                            int64_t n4, int64_t n) {
+  const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+  for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < n4; i += stride) {
+    float4 a = reinterpret_cast<const float4*>(x)[i];
+    if (y) {
+      const float4 b = reinterpret_cast<const float4*>(y)[i];
+      a.x -= b.x; a.y -= b.y; a.z -= b.z; a.w -= b.w;
+    }
+    reinterpret_cast<float4*>(dst)[i] = a;
+  }
+  for (int64_t i = n4 * 4 + blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < n; i += stride)
+    dst[i] = y ? x[i] - y[i] : x[i];
+}
+
+__global__ void zero_kernel(float* __restrict__ dst, int64_t n) {
+  const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+  for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < n; i += stride) dst[i] = 0.f;
+}
+
+__global__ void axpy_kernel(float* __restrict__ y, const float* __restrict__ x, float alpha, int64_t n) {
+  const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+  for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < n; i += stride)
+    y[i] = fmaf(alpha, x[i], y[i]);
+}
+
+// One block per sample: u = softmax(z) - onehot(y) in place over the sample's row of Z [nsamp x rows]
+// (Section 1: u is the prediction vector; Section 2.1: u = d f / d (W a)).  A class id outside [0, rows)
+// sets a status bit and subtracts nothing.  loss = log sum exp z - z_y.
+template <int NTHREADS>
+__global__ void __launch_bounds__(NTHREADS) mlr_softmax_kernel(float* __restrict__ Z, int64_t rows,
+                                                               const int32_t* __restrict__ labels,
+                                                               float* __restrict__ loss, uint32_t* status) {
+  __shared__ float sh[32];
+  float* z = Z + static_cast<int64_t>(blockIdx.x) * rows;
+  float m = -INFINITY;
+  for (int64_t j = threadIdx.x; j < rows; j += NTHREADS) m = fmaxf(m, z[j]);
+  m = block_max<NTHREADS>(m, sh);
+  float s = 0.f;
+  for (int64_t j = threadIdx.x; j < rows; j += NTHREADS) s += expf(z[j] - m);
+  s = block_sum<NTHREADS>(s, sh);
+  const float inv = 1.f / s;
+  const int32_t y = labels[blockIdx.x];
+  const bool ok = y >= 0 && y < rows;
+  if (threadIdx.x == 0) {
+    if (!ok) atomicOr(status, SFB_STATUS_LABEL_RANGE);
+    loss[blockIdx.x] = ok ? (m + logf(s)) - z[y] : 0.f;
+  }
+  __syncthreads();
+  for (int64_t j = threadIdx.x; j < rows; j += NTHREADS) {
+    float u = expf(z[j] - m) * inv;
+    if (ok && j == y) u -= 1.f;
+    z[j] = u;
+  }
+}
+
+// One block per pair: q = ||z||^2; similar: u = 2z; dissimilar: u = -2z if q < margin else 0 (Section 2, DML).
+template <int NTHREADS>
+__global__ void __launch_bounds__(NTHREADS) dml_scale_kernel(float* __restrict__ Z, int64_t rows,
+                                                             const int32_t* __restrict__ similar, float margin) {
+  __shared__ float sh[32];
+  float* z = Z + static_cast<int64_t>(blockIdx.x) * rows;
+  float q = 0.f;
+  for (int64_t j = threadIdx.x; j < rows; j += NTHREADS) q = fmaf(z[j], z[j], q);
+  q = block_sum<NTHREADS>(q, sh);
+  const float c = similar[blockIdx.x] != 0 ? 2.f : (q < margin ? -2.f : 0.f);
+  for (int64_t j = threadIdx.x; j < rows; j += NTHREADS) z[j] = c * z[j];
+}
+
+__global__ void mean_kernel(const float* __restrict__ v, int64_t n, float* out) {
+  __shared__ float sh[32];
+  float s = 0.f;
+  for (int64_t i = threadIdx.x; i < n; i += 256) s += v[i];
+  s = block_sum<256>(s, sh);
+  if (threadIdx.x == 0) *out = s / static_cast<float>(n);
+}
+
+// Column reductions over W [rows x cols] in a fixed order: block (slab, column group of 128) sums
+// w^2 (MODE 0) or w * yvec[row] (MODE 1) over its row slab into part[slab][col].
+template <int MODE>
+__global__ void __launch_bounds__(kThreads) col_partial_kernel(const float* __restrict__ W, int64_t rows,
+                                                               int64_t cols, const float* __restrict__ yvec,
+                                                               float* __restrict__ part, int64_t slab_rows) {
+  __shared__ float sh[8][128];
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const int64_t c0 = static_cast<int64_t>(blockIdx.x) * 128 + tx * 4;
+  const int64_t r0 = static_cast<int64_t>(blockIdx.y) * slab_rows;
+  const int64_t r1 = min(rows, r0 + slab_rows);
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (c0 < cols) {                       // cols is a multiple of 4, so a quad is in range as a whole
+    for (int64_t r = r0 + ty; r < r1; r += 8) {
+      const float4 w = *reinterpret_cast<const float4*>(W + r * cols + c0);
+      if (MODE == 0) {
+        acc.x = fmaf(w.x, w.x, acc.x); acc.y = fmaf(w.y, w.y, acc.y);
+        acc.z = fmaf(w.z, w.z, acc.z); acc.w = fmaf(w.w, w.w, acc.w);
+      } else {
+        const float yv = yvec[r];
+        acc.x = fmaf(w.x, yv, acc.x); acc.y = fmaf(w.y, yv, acc.y);
+        acc.z = fmaf(w.z, yv, acc.z); acc.w = fmaf(w.w, yv, acc.w);
+      }
+    }
+  }
+  *reinterpret_cast<float4*>(&sh[ty][tx * 4]) = acc;
+  __syncthreads();
+  if (threadIdx.x < 128) {
+    const int64_t c = static_cast<int64_t>(blockIdx.x) * 128 + threadIdx.x;
+    if (c < cols) {
+      float s = 0.f;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) s += sh[k][threadIdx.x];
+      part[static_cast<int64_t>(blockIdx.y) * cols + c] = s;
+    }
+  }
+}
+
+// Column sums of squares in fp64 (the prox must resolve norms to far better than fp32's 6e-8, because the
+// rescaling multiplies every entry of W while the step's update is ~1e-3 of ||W||).
+__global__ void __launch_bounds__(kThreads) col_sumsq_kernel(const float* __restrict__ W, int64_t rows, int64_t cols,
+                                                             double* __restrict__ part, int64_t slab_rows) {
+  __shared__ double sh[8][128];
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const int64_t c0 = static_cast<int64_t>(blockIdx.x) * 128 + tx * 4;
+  const int64_t r0 = static_cast<int64_t>(blockIdx.y) * slab_rows;
+  const int64_t r1 = min(rows, r0 + slab_rows);
+  double a0 = 0., a1 = 0., a2 = 0., a3 = 0.;
+  if (c0 < cols) {
+    for (int64_t r = r0 + ty; r < r1; r += 8) {
+      const float4 w = *reinterpret_cast<const float4*>(W + r * cols + c0);
+      a0 = fma(static_cast<double>(w.x), static_cast<double>(w.x), a0);
+      a1 = fma(static_cast<double>(w.y), static_cast<double>(w.y), a1);
+      a2 = fma(static_cast<double>(w.z), static_cast<double>(w.z), a2);
+      a3 = fma(static_cast<double>(w.w), static_cast<double>(w.w), a3);
+    }
+  }
+  sh[ty][tx * 4 + 0] = a0; sh[ty][tx * 4 + 1] = a1; sh[ty][tx * 4 + 2] = a2; sh[ty][tx * 4 + 3] = a3;
+  __syncthreads();
+  if (threadIdx.x < 128) {
+    const int64_t c = static_cast<int64_t>(blockIdx.x) * 128 + threadIdx.x;
+    if (c < cols) {
+      double s = 0.;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) s += sh[k][threadIdx.x];
+      part[static_cast<int64_t>(blockIdx.y) * cols + c] = s;
+    }
+  }
+}
+
+// Prox of Figure 3: b <- b / ||b|| for the columns with ||b|| > 1, others untouched (bit-identical).
+__global__ void __launch_bounds__(kThreads) prox_scale_kernel(float* __restrict__ W, int64_t rows, int64_t cols,
+                                                              const double* __restrict__ part, int nslabs,
+                                                              int64_t slab_rows) {
+  __shared__ double scale[128];
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  if (threadIdx.x < 128) {
+    const int64_t c = static_cast<int64_t>(blockIdx.x) * 128 + threadIdx.x;
+    double s = 0.;
+    if (c < cols)
+      for (int k = 0; k < nslabs; ++k) s += part[static_cast<int64_t>(k) * cols + c];
+    scale[threadIdx.x] = s > 1. ? 1. / sqrt(s) : 1.;
+  }
+  __syncthreads();
+  const int64_t c0 = static_cast<int64_t>(blockIdx.x) * 128 + tx * 4;
+  if (c0 >= cols) return;
+  const double s0 = scale[tx * 4], s1 = scale[tx * 4 + 1], s2 = scale[tx * 4 + 2], s3 = scale[tx * 4 + 3];
+  if (s0 == 1. && s1 == 1. && s2 == 1. && s3 == 1.) return;
+  const int64_t r0 = static_cast<int64_t>(blockIdx.y) * slab_rows;
+  const int64_t r1 = min(rows, r0 + slab_rows);
+  for (int64_t r = r0 + ty; r < r1; r += 8) {
+    float4* p = reinterpret_cast<float4*>(W + r * cols + c0);
+    float4 w = *p;
+    if (s0 != 1.) w.x = static_cast<float>(static_cast<double>(w.x) * s0);
+    if (s1 != 1.) w.y = static_cast<float>(static_cast<double>(w.y) * s1);
+    if (s2 != 1.) w.z = static_cast<float>(static_cast<double>(w.z) * s2);
+    if (s3 != 1.) w.w = static_cast<float>(static_cast<double>(w.w) * s3);
+    *p = w;
+  }
+}
+
+// y = W b : one warp per row.
+__global__ void __launch_bounds__(kThreads) matvec_rows_kernel(const float* __restrict__ W, int64_t rows,
+                                                               int64_t cols, const float* __restrict__ b,
+                                                               float* __restrict__ y) {
+  const int64_t r = static_cast<int64_t>(blockIdx.x) * (kThreads / 32) + (threadIdx.x >> 5);
+  if (r >= rows) return;
+  const int lane = threadIdx.x & 31;
+  float s = 0.f;
+  for (int64_t c = lane * 4; c < cols; c += 128) {
+    const float4 w = *reinterpret_cast<const float4*>(W + r * cols + c);
+    const float4 v = *reinterpret_cast<const float4*>(b + c);
+    s = fmaf(w.x, v.x, s); s = fmaf(w.y, v.y, s); s = fmaf(w.z, v.z, s); s = fmaf(w.w, v.w, s);
+  }
+  s = warp_sum(s);
+  if (lane == 0) y[r] = s;
+}
+
+// One block: c = sum of the slab partials; b = c / ||c||.
+__global__ void __launch_bounds__(1024) pi_normalise_kernel(const float* __restrict__ part, int nslabs, int64_t cols,
+                                                            float* __restrict__ b) {
+  __shared__ float sh[32];
+  float ss = 0.f;
+  for (int64_t c = threadIdx.x; c < cols; c += 1024) {
+    float s = 0.f;
+    for (int k = 0; k < nslabs; ++k) s += part[static_cast<int64_t>(k) * cols + c];
+    b[c] = s;
+    ss = fmaf(s, s, ss);
+  }
+  ss = block_sum<1024>(ss, sh);
+  const float inv = rsqrtf(ss);
+  for (int64_t c = threadIdx.x; c < cols; c += 1024) b[c] *= inv;
+}
+
+__global__ void __launch_bounds__(1024) pi_init_kernel(float* __restrict__ b, int64_t cols) {
+  const float v = rsqrtf(static_cast<float>(cols));
+  for (int64_t c = threadIdx.x; c < cols; c += 1024) b[c] = v;
+}
+
+// L = ||W b||^2 (Rayleigh quotient of W^T W at the unit vector b).
+__global__ void __launch_bounds__(1024) pi_rayleigh_kernel(const float* __restrict__ y, int64_t rows, Scalars* sc) {
+  __shared__ float sh[32];
+  float ss = 0.f;
+  for (int64_t r = threadIdx.x; r < rows; r += 1024) ss = fmaf(y[r], y[r], ss);
+  ss = block_sum<1024>(ss, sh);
+  if (threadIdx.x == 0) { sc->L = ss; sc->invL = 1.f / ss; }
+}
+
+__global__ void set_L_kernel(Scalars* sc, float L) { sc->L = L; sc->invL = 1.f / L; }
+
+inline unsigned grid_for(int64_t n, int per_block) {
+  int64_t g = (n + per_block - 1) / per_block;
+  if (g < 1) g = 1;
+  const int64_t cap = 148 * 16;
+  return static_cast<unsigned>(g > cap ? cap : g);
+}
+
+inline int64_t slab_rows_for(int64_t rows) { return (rows + kProxSlabs - 1) / kProxSlabs; }
+
+}  // namespace
+
+cudaError_t pack_copy(cudaStream_t s, float* dst, const float* x, const float* y, int64_t n) {
+  if (n <= 0) return cudaSuccess;
+  pack_kernel<<<grid_for(n / 4 + 1, kThreads), kThreads, 0, s>>>(dst, x, y, n / 4, n);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t fill_zero(cudaStream_t s, float* dst, int64_t n) {
+  if (n <= 0) return cudaSuccess;
+  zero_kernel<<<grid_for(n, kThreads), kThreads, 0, s>>>(dst, n);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t axpy(cudaStream_t s, float* y, const float* x, float alpha, int64_t n) {
+  if (n <= 0) return cudaSuccess;
+  axpy_kernel<<<grid_for(n, kThreads), kThreads, 0, s>>>(y, x, alpha, n);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t mlr_softmax_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows, const int32_t* labels,
+                             float* loss, uint32_t* status) {
+  if (nsamp <= 0) return cudaSuccess;
+  mlr_softmax_kernel<512><<<static_cast<unsigned>(nsamp), 512, 0, s>>>(Z, rows, labels, loss, status);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t dml_scale_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows, const int32_t* similar,
+                           float margin) {
+  if (nsamp <= 0) return cudaSuccess;
+  dml_scale_kernel<256><<<static_cast<unsigned>(nsamp), 256, 0, s>>>(Z, rows, similar, margin);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t mean_of(cudaStream_t s, const float* v, int64_t n, float* out) {
+  mean_kernel<<<1, 256, 0, s>>>(v, n, out);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t prox_unit_columns(cudaStream_t s, float* W, int64_t rows, int64_t cols, float* colpart) {
+  const int64_t sr = slab_rows_for(rows);
+  dim3 grid(static_cast<unsigned>((cols + 127) / 128), kProxSlabs);
+  double* part = reinterpret_cast<double*>(colpart);
+  col_sumsq_kernel<<<grid, kThreads, 0, s>>>(W, rows, cols, part, sr);
+  count_launch();
+  prox_scale_kernel<<<grid, kThreads, 0, s>>>(W, rows, cols, part, kProxSlabs, sr);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t estimate_lipschitz(cudaStream_t s, const float* W, int64_t rows, int64_t cols, float* b, float* y,
+                               float* colpart, Scalars* sc, int iters) {
+  const int64_t sr = slab_rows_for(rows);
+  dim3 cgrid(static_cast<unsigned>((cols + 127) / 128), kProxSlabs);
+  const unsigned rgrid = static_cast<unsigned>((rows + kThreads / 32 - 1) / (kThreads / 32));
+  pi_init_kernel<<<1, 1024, 0, s>>>(b, cols);
+  count_launch();
+  for (int it = 0; it < iters; ++it) {
+    matvec_rows_kernel<<<rgrid, kThreads, 0, s>>>(W, rows, cols, b, y);
+    count_launch();
+    col_partial_kernel<1><<<cgrid, kThreads, 0, s>>>(W, rows, cols, y, colpart, sr);
+    count_launch();
+    pi_normalise_kernel<<<1, 1024, 0, s>>>(colpart, kProxSlabs, cols, b);
+    count_launch();
+  }
+  matvec_rows_kernel<<<rgrid, kThreads, 0, s>>>(W, rows, cols, b, y);
+  count_launch();
+  pi_rayleigh_kernel<<<1, 1024, 0, s>>>(y, rows, sc);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t set_lipschitz(cudaStream_t s, Scalars* sc, float L) {
+  set_L_kernel<<<1, 1, 0, s>>>(sc, L);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace sfb

@@ -1,0 +1,96 @@
+// Internal declarations shared by the translation units of libsfb (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "sfb.h"
+
+namespace sfb {
+
+extern int64_t g_kernel_launches;     // kernels launched by this library in this process
+inline void count_launch(int n = 1) { g_kernel_launches += n; }
+
+// ---------------------------------------------------------------------------------------------------------
+// Workspace carve-up.  Every offset is a multiple of 1024 bytes so that any sub-buffer can be a TMA base.
+// ---------------------------------------------------------------------------------------------------------
+constexpr size_t kAlign = 1024;
+constexpr int kProxSlabs = 64;        // row slabs of the deterministic column reductions
+
+struct Layout {
+  size_t status, scalars, loss, V, U, colpart, pib, piy, stageX, stageY, stageL;
+  // bf16 tensor-core mode
+  size_t Wb, Xb, VT, ZT, UT, part;
+  int64_t Kp;                         // K rounded up to the contraction block of the update product
+  int64_t colsb;                      // cols rounded up to the contraction block of the forward product
+  size_t total;
+};
+
+Layout make_layout(const sfb_config& c);
+
+struct Scalars {                      // device-resident scalars
+  float loss_mean;
+  float L;                            // ||W||_2^2 used by the coder
+  float invL;
+  float tmp;
+};
+
+}  // namespace sfb
+
+struct sfb_ctx {
+  sfb_config cfg;
+  sfb::Layout lay;
+  float* W;
+  char* ws;
+  cudaStream_t stream;
+  int64_t K;
+  int64_t in_dim;
+  uint64_t committed;                 // bit p set: worker p has written its factors since the last update
+  bool gathered;
+  int last_cuda;
+  cudaEvent_t ev[4];
+  sfb_stats stats;
+  void* tc;                           // tensor-core path state (tensor maps), owned
+
+  template <typename T>
+  T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
+};
+
+namespace sfb {
+
+// ---------------------------------------------------------------------------------------------------------
+// fp32 FMA matrix products:  C (M x N) = sum_k A(m,k) * B(n,k)  followed by an epilogue.
+// A_KC: A(m,k) at A[m*lda + k] (k contiguous), else at A[k*lda + m].  Same for B with n.
+// ---------------------------------------------------------------------------------------------------------
+enum Epilogue { EPI_STORE = 0, EPI_SUB = 1, EPI_RMW = 2, EPI_ISTA = 3 };
+
+struct EpiArgs {
+  float* C;            // output, row-major [M x ldc]
+  int64_t ldc;
+  const float* aux;    // EPI_SUB: the matrix subtracted, same shape and ld as C
+  float alpha;         // EPI_RMW: C += alpha * acc
+  const Scalars* sc;   // EPI_ISTA: reads invL
+  float lam;           // EPI_ISTA: C = soft(C - acc*invL, lam*invL)
+};
+
+cudaError_t sgemm(cudaStream_t s, bool a_kc, bool b_kc, Epilogue epi, int64_t M, int64_t N, int64_t Kc,
+                  const float* A, int64_t lda, const float* B, int64_t ldb, const EpiArgs& e);
+
+// ---------------------------------------------------------------------------------------------------------
+// Factor kernels (pack, softmax, pair residual, prox, power iteration)
+// ---------------------------------------------------------------------------------------------------------
+cudaError_t pack_copy(cudaStream_t s, float* dst, const float* x, const float* y_or_null, int64_t n);
+cudaError_t fill_zero(cudaStream_t s, float* dst, int64_t n);
+cudaError_t mlr_softmax_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows, const int32_t* labels,
+                             float* loss_per_sample, uint32_t* status);
+cudaError_t dml_scale_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows, const int32_t* similar,
+                           float margin);
+cudaError_t mean_of(cudaStream_t s, const float* v, int64_t n, float* out);
+cudaError_t prox_unit_columns(cudaStream_t s, float* W, int64_t rows, int64_t cols, float* colpart);
+cudaError_t estimate_lipschitz(cudaStream_t s, const float* W, int64_t rows, int64_t cols, float* b, float* y,
+                               float* colpart, Scalars* sc, int iters);
+cudaError_t set_lipschitz(cudaStream_t s, Scalars* sc, float L);
+cudaError_t axpy(cudaStream_t s, float* y, const float* x, float alpha, int64_t n);  // y += alpha*x
+
+}  // namespace sfb

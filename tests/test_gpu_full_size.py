@@ -1,0 +1,76 @@
+"""Parity at the full sizes of the five workloads, one step each, in the launch configuration the bench times.
+The paper-scale MLR shape is checked on sampled rows of W (every label row, random rows, the last rows),
+which the oracle computes from the exact log-partition of every sample."""
+import numpy as np
+import pytest
+
+import paper_1409_5705_b200 as S
+import sfb_inputs as I
+from oracle import sfb_oracle as O
+from _parity import TOL, step_tol, config_for, entries_ok, oracle_step, rel_err, to_dev
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+
+PRECS = [pytest.param(S.PREC_FP32, id="fp32"), pytest.param(S.PREC_BF16, id="bf16")]
+
+
+@pytest.mark.parametrize("prec", PRECS)
+@pytest.mark.parametrize("name", ["mlr_mid", "dml", "sc"])
+def test_full_size_step(name, prec):
+    wl = I.WORKLOADS[name]
+    W0 = I.initial_W(wl)
+    inp = I.step_inputs(wl, 0)
+    L = float(np.float32(O.lipschitz_power_iteration(W0))) if wl.model == I.SC else 0.0
+    W = to_dev(W0, torch)
+    ctx = S.Context(config_for(wl, prec, L), W)
+    ctx.sfb_step(to_dev(inp.X, torch), to_dev(inp.Y, torch), to_dev(inp.labels, torch))
+    assert ctx.sfb_get_status() == 0
+    Wg = W.cpu().numpy()
+    ctx.close()
+    del W
+    torch.cuda.empty_cache()
+    ref = oracle_step(wl, W0, inp, L=L)
+    err = rel_err(Wg, ref, W0)
+    assert err <= step_tol(wl, prec, ref, W0), err
+    # rows that carry no label and the ragged last tile must be right on their own, not hidden by the norm
+    tail = slice(wl.rows - wl.rows % 128 if wl.rows % 128 else wl.rows - 128, wl.rows)
+    if wl.model != I.MLR:
+        assert rel_err(Wg[tail], ref[tail], W0[tail]) <= 2 * step_tol(wl, prec, ref, W0)
+    else:
+        assert entries_ok(Wg[tail], ref[tail], W0[tail], TOL[prec])
+        bulk = np.setdiff1d(np.arange(wl.rows), inp.labels)
+        assert entries_ok(Wg[bulk], ref[bulk], W0[bulk], TOL[prec])
+
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_mlr_large_sampled_rows(prec):
+    wl = I.WORKLOADS["mlr_large"]
+    W0 = I.initial_W(wl, threads=16)
+    inp = I.step_inputs(wl, 0)
+    W = torch.empty((wl.rows, wl.cols), dtype=torch.float32, device="cuda")
+    chunk = 32768
+    for r0 in range(0, wl.rows, chunk):
+        W[r0:r0 + chunk].copy_(torch.from_numpy(W0[r0:r0 + chunk]))
+    ctx = S.Context(config_for(wl, prec), W)
+    ctx.sfb_step(to_dev(inp.X, torch), None, to_dev(inp.labels, torch))
+    assert ctx.sfb_get_status() == 0
+    loss = ctx.sfb_get_stats().last_loss
+    rng = np.random.default_rng(7)
+    label_rows = np.unique(inp.labels)
+    rows = np.unique(np.concatenate([label_rows, rng.integers(0, wl.rows, 4096),
+                                     np.arange(wl.rows - 136, wl.rows)]))
+    Wg = W[torch.from_numpy(rows).cuda()].cpu().numpy()
+    ctx.close()
+    del W
+    torch.cuda.empty_cache()
+    lse = O.mlr_log_partition(W0, inp.X)
+    ref = O.mlr_updated_rows(W0[rows], rows, inp.X, inp.labels, lse, wl.eta)
+    W0r = W0[rows]
+    assert rel_err(Wg, ref, W0r) <= TOL[prec]
+    is_label = np.isin(rows, label_rows)
+    assert entries_ok(Wg[~is_label], ref[~is_label], W0r[~is_label], TOL[prec])
+    last = rows >= wl.rows - 136
+    assert entries_ok(Wg[last], ref[last], W0r[last], TOL[prec])
+    zy = np.einsum("kd,kd->k", inp.X.astype(np.float64), W0[inp.labels].astype(np.float64))
+    assert abs(loss - float((lse - zy).mean())) < 1e-3
