@@ -21,7 +21,7 @@ constexpr int kProxSlabs = 64;        // row slabs of the deterministic column r
 struct Layout {
   size_t status, scalars, loss, V, U, colpart, pib, piy, stageX, stageY, stageL;
   // bf16 tensor-core mode
-  size_t Wb, Xb, VT, ZT, UT, part;
+  size_t Wb, Xb, VT, ZT, UT, part, Xf, labels;
   int64_t Kp;                         // K rounded up to the contraction block of the update product
   int64_t colsb;                      // cols rounded up to the contraction block of the forward product
   size_t total;

@@ -1,11 +1,700 @@
+// Tensor-core (bf16 operand) path of the SFB step on sm_100a.
+//
+// One persistent, warp-specialised kernel computes  D (M x N) = A (M x Kc) * B (N x Kc)^T  with bf16 operands
+// staged by TMA into 128-byte-swizzled shared memory, tcgen05.mma accumulating in TMEM (two 128 x 256 fp32
+// accumulators, so the epilogue of one tile overlaps the main loop of the next), and one of two epilogues:
+//
+//   TC_UPDATE   W <- W + alpha * D   (Section 3, Figure 1: reconstruct the K rank-1 updates and apply them).
+//               A = U^T [rows x K], B = V^T [cols x K].  The fp32 tile of W is brought in by TMA while the MMAs
+//               run, modified in shared memory and stored back by TMA: W makes one HBM round trip per step.
+//               A bf16 copy of the new W (the operand of the next step's forward product) is written alongside.
+//   TC_FORWARD  Z = D stored as fp32, plus per (sample, 256-row block) softmax partials (max, sum of exp)
+//               (Section 2: the products W a_i, batched; Section 1: u is the prediction vector).
+//               A = X [K x cols] (samples on the TMEM lanes), B = W [rows x cols].
+//
+// Roles: warp 0 TMA producer, warp 1 MMA issuer (and TMEM owner), warps 2-5 epilogue (one TMEM lane quarter each).
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <algorithm>
+#include <new>
+
+#include "sfb_ptx.cuh"
 #include "sfb_tc.h"
+
 namespace sfb {
-void tc_extend_layout(const sfb_config&, Layout&, size_t&) {}
-int tc_init(sfb_ctx*) { return SFB_ERR_UNSUPPORTED; }
-void tc_destroy(sfb_ctx*) {}
-int tc_factors(sfb_ctx*, int64_t, int64_t, const float*, const float*, const int32_t*) { return SFB_ERR_UNSUPPORTED; }
-int tc_gather(sfb_ctx*) { return SFB_ERR_UNSUPPORTED; }
-int tc_update(sfb_ctx*) { return SFB_ERR_UNSUPPORTED; }
-int tc_after_update(sfb_ctx*) { return SFB_ERR_UNSUPPORTED; }
-int tc_get_factors(sfb_ctx*, const void**, const void**, int32_t*, int32_t*, int64_t*, int64_t*) { return SFB_ERR_UNSUPPORTED; }
+namespace {
+
+using namespace ptx;
+
+constexpr int BM = 128, BN = 256, BK = 64, UMMA_K = 16;
+constexpr int kBytesA = BM * BK * 2, kBytesB = BN * BK * 2;
+constexpr int kChunk = 32;                 // accumulator columns handled per epilogue step
+constexpr int kSlotBytes = 32 * kChunk * 4;  // one warp's 32 rows x 32 fp32 columns
+constexpr int kThreads = 192;
+constexpr int kTmemCols = 512;
+
+enum TcEpi { TC_UPDATE = 0, TC_FORWARD = 1 };
+
+template <int EPI> struct Shape {
+  static constexpr int S = EPI == TC_UPDATE ? 3 : 4;   // operand pipeline stages
+  static constexpr int R = EPI == TC_UPDATE ? 5 : 2;   // epilogue ring slots per warp
+  static constexpr int kBars = 2 * S + 4 + 4 * R;
+  static constexpr int kSmem = S * (kBytesA + kBytesB) + 4 * R * kSlotBytes + kBars * 8 + 16 + 1024;
+};
+
+struct TcParams {
+  int32_t M, N, Kc;            // extents of the product: output rows, output columns, contraction
+  int32_t m_off;               // first output row handled by this launch (per-worker slices of the forward)
+  int32_t tilesM, tilesN;
+  float alpha;                 // TC_UPDATE: -eta
+  __nv_bfloat16* shadow;       // TC_UPDATE: bf16 copy of the updated W, row pitch shadow_ld elements (or null)
+  int64_t shadow_ld;
+  float2* part;                // TC_FORWARD: [tilesN][part_ld] (max, sum exp) per sample and column block
+  int64_t part_ld;
+  uint32_t* status;
+};
+
+__device__ __forceinline__ void tile_coords(const TcParams& p, int tile, int& m0, int& n0) {
+  int tm, tn;
+  if (p.tilesM <= 8) { tm = tile % p.tilesM; tn = tile / p.tilesM; }   // few row blocks: keep a B block hot in L2
+  else { tn = tile % p.tilesN; tm = tile / p.tilesN; }                 // update: sweep the columns of one row block
+  m0 = p.m_off + tm * BM;
+  n0 = tn * BN;
 }
+
+template <int EPI>
+__global__ void __launch_bounds__(kThreads, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmC, const TcParams p) {
+  constexpr int S = Shape<EPI>::S, R = Shape<EPI>::R;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sA = smem;
+  uint8_t* sB = smem + S * kBytesA;
+  uint8_t* sRing = smem + S * (kBytesA + kBytesB);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sRing + 4 * R * kSlotBytes);
+  uint64_t* full = bars;
+  uint64_t* empty = bars + S;
+  uint64_t* tfull = bars + 2 * S;
+  uint64_t* tempty = bars + 2 * S + 2;
+  uint64_t* rfull = bars + 2 * S + 4;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + Shape<EPI>::kBars);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int ntiles = p.tilesM * p.tilesN;
+  const int numK = (p.Kc + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < S; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&tfull[i], 1); mbar_init(&tempty[i], 4); }
+    for (int i = 0; i < 4 * R; ++i) mbar_init(&rfull[i], 1);
+    *abort_flag = 0;
+    fence_barrier_init();
+    prefetch_tmap(&tmA); prefetch_tmap(&tmB); prefetch_tmap(&tmC);
+  }
+  if (warp == 1) { tmem_alloc(tmem_slot, kTmemCols); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      // The small operand every tile re-reads (V^T in the update, X in the forward) is pinned in L2.
+      const uint64_t pol_keep = policy_evict_last();
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+        int m0, n0;
+        tile_coords(p, tile, m0, n0);
+        for (int kb = 0; kb < numK; ++kb, ++it) {
+          const uint32_t s = it % S, ph = (it / S) & 1;
+          if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
+          mbar_expect_tx(&full[s], kBytesA + kBytesB);
+          if (EPI == TC_UPDATE) {
+            tma_load_2d(sA + s * kBytesA, &tmA, kb * BK, m0, &full[s]);
+            tma_load_2d_hint(sB + s * kBytesB, &tmB, kb * BK, n0, &full[s], pol_keep);
+          } else {
+            tma_load_2d_hint(sA + s * kBytesA, &tmA, kb * BK, m0, &full[s], pol_keep);
+            tma_load_2d(sB + s * kBytesB, &tmB, kb * BK, n0, &full[s]);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_bf16(BM, BN);
+      uint32_t it = 0, tl = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++tl) {
+        const uint32_t a = tl & 1, aph = (tl >> 1) & 1;
+        if (!mbar_wait(&tempty[a], aph ^ 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + a * BN;
+        for (int kb = 0; kb < numK; ++kb, ++it) {
+          const uint32_t s = it % S, ph = (it / S) & 1;
+          if (!mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t da = umma_desc_k128(smem_u32(sA + s * kBytesA));
+          const uint64_t db = umma_desc_k128(smem_u32(sB + s * kBytesB));
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k)
+            umma_bf16(d_tmem, da + static_cast<uint64_t>(k * UMMA_K * 2 / 16), db + static_cast<uint64_t>(k * UMMA_K * 2 / 16),
+                      idesc, (kb | k) != 0 ? 1u : 0u);
+          umma_commit(&empty[s]);          // the stage is free once these MMAs have read it
+        }
+        if (ok) umma_commit(&tfull[a]);    // the accumulator is complete once every MMA of the tile is
+      }
+    }
+  } else {
+    // ---------------- epilogue: warps 2..5, TMEM lane quarter q ----------------
+    const int q = warp & 3;
+    uint8_t* ring = sRing + q * R * kSlotBytes;
+    uint64_t* rf = rfull + q * R;
+    const int my_tiles = blockIdx.x < ntiles ? (ntiles - 1 - blockIdx.x) / gridDim.x + 1 : 0;
+    const uint32_t nchunks = static_cast<uint32_t>(my_tiles) * (BN / kChunk);
+    bool ok = true;
+
+    if constexpr (EPI == TC_UPDATE) {
+      // Per warp: kLoadSlots ring slots receive W chunks by TMA (issued kLoadSlots chunks ahead, refilled as soon
+      // as the warp has read them) and 2 staging slots carry the updated chunks to the TMA stores.  The TMEM
+      // load of chunk c+1 is in flight while chunk c is combined with W.
+      constexpr int kLoadSlots = R - 2;
+      constexpr int kChunksPerTile = BN / kChunk;
+      uint8_t* stage = ring + kLoadSlots * kSlotBytes;
+      const uint64_t pol_stream = policy_evict_first();
+      // chunk g+kLoadSlots is always requested while chunk g is processed: track its tile incrementally
+      uint32_t lg = 0;                 // next chunk to request
+      int ltile = blockIdx.x, lc = 0;  // its tile and chunk-in-tile
+      auto issue_load = [&]() {
+        if (lg >= nchunks) return;
+        int m0, n0;
+        tile_coords(p, ltile, m0, n0);
+        const uint32_t slot = lg % kLoadSlots;
+        mbar_expect_tx(&rf[slot], kSlotBytes);
+        tma_load_2d_hint(ring + slot * kSlotBytes, &tmC, n0 + lc * kChunk, m0 + q * 32, &rf[slot], pol_stream);
+        ++lg;
+        if (++lc == kChunksPerTile) { lc = 0; ltile += gridDim.x; }
+      };
+      if (lane == 0)
+        for (int i = 0; i < kLoadSlots; ++i) issue_load();
+      uint32_t g = 0;
+      for (int tl = 0; tl < my_tiles && ok; ++tl) {
+        int m0, n0;
+        tile_coords(p, blockIdx.x + tl * gridDim.x, m0, n0);
+        const uint32_t a = tl & 1, aph = (tl >> 1) & 1;
+        if (!__all_sync(0xffffffffu, mbar_wait(&tfull[a], aph, abort_flag))) { ok = false; break; }
+        tc_fence_after();
+        const int row = m0 + q * 32 + lane;
+        const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + a * BN;
+        uint32_t acc0[32], acc1[32];
+        tmem_ld_32x32(t_addr, acc0);
+        auto process = [&](uint32_t (&acc)[32], uint32_t (&nxt)[32], int c) -> bool {
+          tmem_ld_wait();                                      // chunk c's accumulators are in registers
+          if (c + 1 < kChunksPerTile) {
+            tmem_ld_32x32(t_addr + (c + 1) * kChunk, nxt);     // chunk c+1 streams in during this chunk's work
+          } else {
+            tc_fence_before();                                 // last TMEM read of the tile: hand the
+            __syncwarp();                                      // accumulator back to the MMA warp now
+            if (lane == 0) mbar_arrive(&tempty[a]);
+          }
+          const uint32_t slot = g % kLoadSlots;
+          const uint8_t* sl = ring + slot * kSlotBytes;
+          uint8_t* st = stage + (g & 1) * kSlotBytes;
+          if (!__all_sync(0xffffffffu, mbar_wait(&rf[slot], (g / kLoadSlots) & 1, abort_flag))) return false;
+          if (lane == 0) tma_wait_group_read<1>();             // the store two chunks back has read `st`
+          __syncwarp();
+          const int col0 = n0 + c * kChunk;
+          uint32_t packed[16];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const int o = lane * 128 + ((j ^ (lane & 7)) << 4);
+            float4 w = *reinterpret_cast<const float4*>(sl + o);
+            w.x = fmaf(p.alpha, __uint_as_float(acc[4 * j + 0]), w.x);
+            w.y = fmaf(p.alpha, __uint_as_float(acc[4 * j + 1]), w.y);
+            w.z = fmaf(p.alpha, __uint_as_float(acc[4 * j + 2]), w.z);
+            w.w = fmaf(p.alpha, __uint_as_float(acc[4 * j + 3]), w.w);
+            *reinterpret_cast<float4*>(st + o) = w;
+            __nv_bfloat162 lo = __floats2bfloat162_rn(w.x, w.y), hi = __floats2bfloat162_rn(w.z, w.w);
+            packed[2 * j + 0] = *reinterpret_cast<uint32_t*>(&lo);
+            packed[2 * j + 1] = *reinterpret_cast<uint32_t*>(&hi);
+          }
+          fence_proxy_async_smem();
+          __syncwarp();                                        // every lane has read `sl` and written `st`
+          if (lane == 0) {
+            tma_store_2d_hint(&tmC, st, col0, m0 + q * 32, pol_stream);
+            tma_commit_group();
+            issue_load();                                      // refill the slot just consumed
+          }
+          if (p.shadow != nullptr && row < p.M) {
+            __nv_bfloat16* dst = p.shadow + static_cast<int64_t>(row) * p.shadow_ld + col0;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              if (col0 + 8 * j < p.shadow_ld)
+                *reinterpret_cast<uint4*>(dst + 8 * j) =
+                    make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
+          }
+          ++g;
+          return true;
+        };
+#pragma unroll 1
+        for (int c = 0; c < kChunksPerTile && ok; c += 2) {
+          ok = process(acc0, acc1, c);
+          if (ok) ok = process(acc1, acc0, c + 1);
+        }
+      }
+      if (lane == 0) tma_wait_group<0>();
+    } else {
+      // Forward: store Z through the ring and keep a running (max, sum exp) per sample over the tile's columns.
+      uint32_t gs = 0;                       // stores issued so far: consecutive stores alternate ring slots
+      for (int tl = 0; tl < my_tiles && ok; ++tl) {
+        int m0, n0;
+        tile_coords(p, blockIdx.x + tl * gridDim.x, m0, n0);
+        const uint32_t a = tl & 1, aph = (tl >> 1) & 1;
+        if (!__all_sync(0xffffffffu, mbar_wait(&tfull[a], aph, abort_flag))) { ok = false; break; }
+        tc_fence_after();
+        const int row = m0 + q * 32 + lane;
+        float mx = -INFINITY, sum = 0.f;
+        for (int c = 0; c < BN / kChunk; ++c) {
+          uint8_t* sl = ring + (gs % R) * kSlotBytes;
+          uint32_t acc[32];
+          tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + a * BN + c * kChunk, acc);
+          tmem_ld_wait();
+          const int col0 = n0 + c * kChunk;
+          if (col0 < p.N) {
+            float cm = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (col0 + j < p.N) cm = fmaxf(cm, __uint_as_float(acc[j]));
+            const float nm = fmaxf(mx, cm);
+            float cs = 0.f;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (col0 + j < p.N) cs += __expf(__uint_as_float(acc[j]) - nm);
+            sum = sum * __expf(mx - nm) + cs;
+            mx = nm;
+            if (lane == 0) tma_wait_group_read<R - 1>();   // the store that last used this slot has read it
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              *reinterpret_cast<uint4*>(sl + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                  make_uint4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_2d(&tmC, sl, col0, m0 + q * 32);
+              tma_commit_group();
+            }
+            ++gs;
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tempty[a]);
+        if (row < p.M) p.part[static_cast<int64_t>(n0 / BN) * p.part_ld + row] = make_float2(mx, sum);
+      }
+      if (lane == 0) tma_wait_group<0>();
+    }
+  }
+
+  // ---------------- teardown ----------------
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    // A wait ran out: report it, give copies in flight a bounded time to land, then release TMEM.
+    if (threadIdx.x == 0) atomicOr(p.status, SFB_STATUS_TIMEOUT);
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, kTmemCols); }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Bandwidth-bound companions of the tensor-core products
+// ---------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// fp32 [rows x cols] -> bf16 [rows x ld] (row-major), 8 elements per thread; cols is a multiple of 4.
+__global__ void __launch_bounds__(256) convert_rows_kernel(const float* __restrict__ src, int64_t rows, int64_t cols,
+                                                           __nv_bfloat16* __restrict__ dst, int64_t ld) {
+  const int64_t quads = cols / 4;
+  const int64_t total = rows * quads;
+  const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+  for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total; i += stride) {
+    const int64_t r = i / quads, qd = i % quads;
+    const float4 v = *reinterpret_cast<const float4*>(src + r * cols + qd * 4);
+    *reinterpret_cast<uint2*>(dst + r * ld + qd * 4) = make_uint2(pack_bf16(v.x, v.y), pack_bf16(v.z, v.w));
+  }
+}
+
+// Pack of the inputs of n samples starting at pair index off (Section 2.1: v = a_i):
+//   Xb[off + i][:]  = bf16(x_i)          forward operand, sample-major
+//   VT[:][off + i]  = bf16(x_i)          update operand, feature-major (V^T)
+// 64 x 64 tiles through shared memory so that both sides are written in 16-byte pieces.
+__global__ void __launch_bounds__(256) pack_mlr_kernel(const float* __restrict__ X, int64_t n, int64_t cols,
+                                                       __nv_bfloat16* __restrict__ Xb, int64_t ldx,
+                                                       __nv_bfloat16* __restrict__ VT, int64_t ldv, int64_t off,
+                                                       float* __restrict__ Xf, const int32_t* __restrict__ labels,
+                                                       int32_t* __restrict__ labels_out) {
+  __shared__ float tile[64][65];
+  const int64_t i0 = static_cast<int64_t>(blockIdx.y) * 64, c0 = static_cast<int64_t>(blockIdx.x) * 64;
+  const int t = threadIdx.x;
+#pragma unroll
+  for (int v = 0; v < 4; ++v) {
+    const int idx = t + v * 256;            // 64 samples x 16 quads
+    const int i = idx / 16, cq = (idx % 16) * 4;
+    float4 val = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (i0 + i < n && c0 + cq < cols) val = *reinterpret_cast<const float4*>(X + (i0 + i) * cols + c0 + cq);
+    tile[i][cq + 0] = val.x; tile[i][cq + 1] = val.y; tile[i][cq + 2] = val.z; tile[i][cq + 3] = val.w;
+    if (i0 + i < n && c0 + cq < cols) {
+      *reinterpret_cast<uint2*>(Xb + (off + i0 + i) * ldx + c0 + cq) =
+          make_uint2(pack_bf16(val.x, val.y), pack_bf16(val.z, val.w));
+      *reinterpret_cast<float4*>(Xf + (off + i0 + i) * cols + c0 + cq) = val;
+    }
+  }
+  if (blockIdx.x == 0 && t < 64 && i0 + t < n) labels_out[off + i0 + t] = labels[i0 + t];
+  __syncthreads();
+#pragma unroll
+  for (int v = 0; v < 2; ++v) {
+    const int idx = t + v * 256;            // 64 features x 8 groups of 8 samples
+    const int c = idx / 8, ig = (idx % 8) * 8;
+    if (c0 + c >= cols) continue;
+    __nv_bfloat16* dst = VT + (c0 + c) * ldv + off + i0 + ig;
+    if (i0 + ig + 7 < n && ((off + i0 + ig) & 7) == 0) {
+      *reinterpret_cast<uint4*>(dst) =
+          make_uint4(pack_bf16(tile[ig][c], tile[ig + 1][c]), pack_bf16(tile[ig + 2][c], tile[ig + 3][c]),
+                     pack_bf16(tile[ig + 4][c], tile[ig + 5][c]), pack_bf16(tile[ig + 6][c], tile[ig + 7][c]));
+    } else {
+      for (int k = 0; k < 8; ++k)
+        if (i0 + ig + k < n) dst[k] = __float2bfloat16_rn(tile[ig + k][c]);
+    }
+  }
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// One warp per sample: merge the per-block (max, sum exp) partials into log sum exp; loss = lse - z_y.
+__global__ void __launch_bounds__(256) mlr_lse_kernel(const float2* __restrict__ part, int64_t part_ld, int nblocks,
+                                                      const float* __restrict__ Z, int64_t ldz, int64_t rows,
+                                                      const int32_t* __restrict__ labels, int64_t off, int64_t n,
+                                                      float* __restrict__ lse, float* __restrict__ loss,
+                                                      uint32_t* status) {
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * 8 + (threadIdx.x >> 5);
+  if (i >= n) return;
+  const int lane = threadIdx.x & 31;
+  const int64_t s = off + i;
+  float m = -INFINITY;
+  for (int b = lane; b < nblocks; b += 32) m = fmaxf(m, part[static_cast<int64_t>(b) * part_ld + s].x);
+  m = warp_max(m);
+  float sum = 0.f;
+  for (int b = lane; b < nblocks; b += 32) {
+    const float2 v = part[static_cast<int64_t>(b) * part_ld + s];
+    sum += v.y * __expf(v.x - m);
+  }
+  sum = warp_sum(sum);
+  if (lane == 0) {
+    const float l = m + logf(sum);
+    lse[s] = l;
+    const int32_t y = labels[i];
+    const bool okl = y >= 0 && y < rows;
+    if (!okl) atomicOr(status, SFB_STATUS_LABEL_RANGE);
+    loss[s] = okl ? l - Z[s * ldz + y] : 0.f;
+  }
+}
+
+// P^T[r][off + i] = bf16( exp(z_ir - lse_i) ): 64 samples x 64 rows per block, transposed through shared
+// memory (Z is sample-major, the update operand is row-major with samples contiguous).  The factor is
+// u_i = p_i - onehot(y_i); its onehot part is not rounded to bf16 but applied exactly by label_rows_kernel.
+__global__ void __launch_bounds__(256) mlr_emit_ut_kernel(const float* __restrict__ Z, int64_t ldz, int64_t rows,
+                                                          const float* __restrict__ lse, int64_t off, int64_t n,
+                                                          __nv_bfloat16* __restrict__ UT, int64_t ldu) {
+  __shared__ float tile[64][65];
+  const int64_t i0 = static_cast<int64_t>(blockIdx.y) * 64, r0 = static_cast<int64_t>(blockIdx.x) * 64;
+  const int t = threadIdx.x;
+  const bool vec = (ldz % 4) == 0;
+#pragma unroll
+  for (int v = 0; v < 4; ++v) {
+    const int idx = t + v * 256;
+    const int i = idx / 16, rq = (idx % 16) * 4;
+    if (i0 + i >= n) continue;
+    const int64_t s = off + i0 + i;
+    const float l = lse[s];
+    const float* zp = Z + s * ldz + r0 + rq;
+    float z[4] = {0.f, 0.f, 0.f, 0.f};
+    if (vec && r0 + rq + 3 < rows) {
+      const float4 q4 = *reinterpret_cast<const float4*>(zp);
+      z[0] = q4.x; z[1] = q4.y; z[2] = q4.z; z[3] = q4.w;
+    } else {
+      for (int k = 0; k < 4; ++k)
+        if (r0 + rq + k < rows) z[k] = zp[k];
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      tile[i][rq + k] = __expf(z[k] - l);
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int v = 0; v < 2; ++v) {
+    const int idx = t + v * 256;
+    const int r = idx / 8, ig = (idx % 8) * 8;
+    if (r0 + r >= rows) continue;
+    __nv_bfloat16* dst = UT + (r0 + r) * ldu + off + i0 + ig;
+    if (i0 + ig + 7 < n && ((off + i0 + ig) & 7) == 0) {
+      *reinterpret_cast<uint4*>(dst) =
+          make_uint4(pack_bf16(tile[ig][r], tile[ig + 1][r]), pack_bf16(tile[ig + 2][r], tile[ig + 3][r]),
+                     pack_bf16(tile[ig + 4][r], tile[ig + 5][r]), pack_bf16(tile[ig + 6][r], tile[ig + 7][r]));
+    } else {
+      for (int k = 0; k < 8; ++k)
+        if (i0 + ig + k < n) dst[k] = __float2bfloat16_rn(tile[ig + k][r]);
+    }
+  }
+}
+
+// The onehot part of the K factors, sum_i (-e_{y_i}) x_i^T, applied to W in fp32 after the tensor-core product
+// has applied sum_i p_i x_i^T:  W[y] <- W[y] + eta * sum_{i : y_i = y} x_i.  One block per sample; the block of
+// the first sample of each class sums that class's samples in index order (no atomics: same result every
+// run) and refreshes the bf16 copy of the row.
+__global__ void __launch_bounds__(256) label_rows_kernel(float* __restrict__ W, int64_t rows, int64_t cols,
+                                                         const float* __restrict__ Xf, const int32_t* __restrict__ labels,
+                                                         int K, float eta, __nv_bfloat16* __restrict__ shadow,
+                                                         int64_t shadow_ld) {
+  __shared__ int first;
+  const int i = blockIdx.x;
+  const int32_t y = labels[i];
+  if (y < 0 || y >= rows) return;              // out-of-range ids were flagged by the softmax pass
+  if (threadIdx.x == 0) first = 1;
+  __syncthreads();
+  for (int j = threadIdx.x; j < i; j += 256)
+    if (labels[j] == y) first = 0;
+  __syncthreads();
+  if (!first) return;
+  for (int64_t c = (static_cast<int64_t>(blockIdx.y) * 256 + threadIdx.x) * 4; c < cols;
+       c += static_cast<int64_t>(gridDim.y) * 256 * 4) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int j = i; j < K; ++j) {
+      if (labels[j] != y) continue;
+      const float4 x = *reinterpret_cast<const float4*>(Xf + static_cast<int64_t>(j) * cols + c);
+      acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
+    }
+    float4* wp = reinterpret_cast<float4*>(W + static_cast<int64_t>(y) * cols + c);
+    float4 w = *wp;
+    w.x = fmaf(eta, acc.x, w.x); w.y = fmaf(eta, acc.y, w.y);
+    w.z = fmaf(eta, acc.z, w.z); w.w = fmaf(eta, acc.w, w.w);
+    *wp = w;
+    if (shadow)
+      *reinterpret_cast<uint2*>(shadow + static_cast<int64_t>(y) * shadow_ld + c) =
+          make_uint2(pack_bf16(w.x, w.y), pack_bf16(w.z, w.w));
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct TcState {
+  EncodeTiledFn encode;
+  int sms;
+};
+
+inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
+
+// 2-D row-major tensor [outer x inner] with row pitch `pitch_bytes`, box [box_outer x box_inner], 128-byte swizzle.
+bool make_map(const TcState* st, CUtensorMap* m, CUtensorMapDataType dt, int esz, void* base, int64_t inner,
+              int64_t outer, int64_t pitch_bytes, int box_inner, int box_outer) {
+  if (inner <= 0 || outer <= 0) return false;
+  cuuint64_t dims[2] = {static_cast<cuuint64_t>(inner), static_cast<cuuint64_t>(outer)};
+  cuuint64_t strides[1] = {static_cast<cuuint64_t>(pitch_bytes)};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(box_inner), static_cast<cuuint32_t>(box_outer)};
+  cuuint32_t estr[2] = {1, 1};
+  (void)esz;
+  return st->encode(m, dt, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int EPI>
+cudaError_t launch_gemm(sfb_ctx* ctx, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c, TcParams p) {
+  const TcState* st = static_cast<const TcState*>(ctx->tc);
+  static bool attr_set[2] = {false, false};
+  if (!attr_set[EPI]) {
+    cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         Shape<EPI>::kSmem);
+    if (e != cudaSuccess) return e;
+    attr_set[EPI] = true;
+  }
+  const int64_t tiles = static_cast<int64_t>(p.tilesM) * p.tilesN;
+  if (tiles <= 0) return cudaSuccess;
+  const int grid = static_cast<int>(tiles < st->sms ? tiles : st->sms);
+  tc_gemm_kernel<EPI><<<grid, kThreads, Shape<EPI>::kSmem, ctx->stream>>>(a, b, c, p);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+#define CKC(call)                                       \
+  do {                                                  \
+    cudaError_t e__ = (call);                           \
+    if (e__ != cudaSuccess) {                           \
+      ctx->last_cuda = static_cast<int>(e__);           \
+      return SFB_ERR_CUDA;                              \
+    }                                                   \
+  } while (0)
+
+void tc_extend_layout(const sfb_config& c, Layout& L, size_t& off) {
+  auto take = [&](size_t bytes) { size_t o = off; off += (bytes + kAlign - 1) / kAlign * kAlign; return o; };
+  const size_t K = static_cast<size_t>(c.workers) * c.batch;
+  L.Kp = round_up(static_cast<int64_t>(K), 64);
+  L.colsb = round_up(c.cols, 64);
+  const size_t ldz = static_cast<size_t>(round_up(c.rows, 32));
+  const size_t nblk = static_cast<size_t>((c.rows + BN - 1) / BN);
+  L.Wb = take(static_cast<size_t>(c.rows) * L.colsb * 2);
+  L.Xb = take(K * L.colsb * 2);
+  L.VT = take(static_cast<size_t>(c.cols) * L.Kp * 2);
+  L.ZT = take(K * ldz * 4);                      // logits Z, sample-major [K x ldz]
+  L.UT = take(static_cast<size_t>(c.rows) * L.Kp * 2);
+  L.part = take(nblk * K * 8);
+  L.V = take(K * 4);                             // log-sum-exp per sample
+  L.Xf = take(K * static_cast<size_t>(c.cols) * 4);   // fp32 copy of the K samples (exact label-row term)
+  L.labels = take(K * 4);                        // class ids of the K samples
+  L.U = 0;
+}
+
+int tc_init(sfb_ctx* ctx) {
+  if (ctx->cfg.model != SFB_MLR) return SFB_ERR_UNSUPPORTED;
+  TcState* st = new (std::nothrow) TcState();
+  if (!st) return SFB_ERR_ARG;
+  ctx->tc = st;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  CKC(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+  if (qres != cudaDriverEntryPointSuccess || !fn) return SFB_ERR_CUDA;
+  st->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  int dev = 0;
+  CKC(cudaGetDevice(&dev));
+  CKC(cudaDeviceGetAttribute(&st->sms, cudaDevAttrMultiProcessorCount, dev));
+  const sfb_config& c = ctx->cfg;
+  // bf16 copy of W for the forward product; afterwards the update's epilogue keeps it current
+  convert_rows_kernel<<<148 * 8, 256, 0, ctx->stream>>>(ctx->W, c.rows, c.cols, ctx->at<__nv_bfloat16>(ctx->lay.Wb),
+                                                        ctx->lay.colsb);
+  count_launch();
+  CKC(cudaGetLastError());
+  return SFB_OK;
+}
+
+void tc_destroy(sfb_ctx* ctx) {
+  delete static_cast<TcState*>(ctx->tc);
+  ctx->tc = nullptr;
+}
+
+int tc_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float* /*Y*/, const int32_t* labels) {
+  const sfb_config& c = ctx->cfg;
+  const TcState* st = static_cast<const TcState*>(ctx->tc);
+  const Layout& L = ctx->lay;
+  const int64_t rows = c.rows, cols = c.cols, K = ctx->K;
+  const int64_t ldz = round_up(rows, 32);
+  __nv_bfloat16* Xb = ctx->at<__nv_bfloat16>(L.Xb);
+  __nv_bfloat16* VT = ctx->at<__nv_bfloat16>(L.VT);
+  __nv_bfloat16* Wb = ctx->at<__nv_bfloat16>(L.Wb);
+  __nv_bfloat16* UT = ctx->at<__nv_bfloat16>(L.UT);
+  float* Z = ctx->at<float>(L.ZT);
+  float2* part = ctx->at<float2>(L.part);
+  float* lse = ctx->at<float>(L.V);
+  float* loss = ctx->at<float>(L.loss);
+  uint32_t* status = ctx->at<uint32_t>(L.status);
+
+  dim3 pgrid(static_cast<unsigned>((cols + 63) / 64), static_cast<unsigned>((n + 63) / 64));
+  pack_mlr_kernel<<<pgrid, 256, 0, ctx->stream>>>(X, n, cols, Xb, L.colsb, VT, L.Kp, off, ctx->at<float>(L.Xf), labels,
+                                                  ctx->at<int32_t>(L.labels));
+  count_launch();
+  CKC(cudaGetLastError());
+
+  // Z[off .. off+n) = X W^T : samples on the lanes (A), rows of W on the accumulator columns (B)
+  CUtensorMap ma, mb, mc;
+  if (!make_map(st, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Xb, cols, off + n, L.colsb * 2, BK, BM) ||
+      !make_map(st, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Wb, cols, rows, L.colsb * 2, BK, BN) ||
+      !make_map(st, &mc, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, Z, rows, off + n, ldz * 4, kChunk, 32))
+    return SFB_ERR_CUDA;
+  TcParams p{};
+  p.M = static_cast<int32_t>(off + n); p.N = static_cast<int32_t>(rows); p.Kc = static_cast<int32_t>(cols);
+  p.m_off = static_cast<int32_t>(off);
+  p.tilesM = static_cast<int32_t>((n + BM - 1) / BM);
+  p.tilesN = static_cast<int32_t>((rows + BN - 1) / BN);
+  p.part = part; p.part_ld = K; p.status = status;
+  CKC(launch_gemm<TC_FORWARD>(ctx, ma, mb, mc, p));
+  ctx->stats.flops += 2.0 * n * rows * cols;
+
+  mlr_lse_kernel<<<static_cast<unsigned>((n + 7) / 8), 256, 0, ctx->stream>>>(part, K, p.tilesN, Z, ldz, rows, labels, off,
+                                                                              n, lse, loss, status);
+  count_launch();
+  dim3 egrid(static_cast<unsigned>((rows + 63) / 64), static_cast<unsigned>((n + 63) / 64));
+  mlr_emit_ut_kernel<<<egrid, 256, 0, ctx->stream>>>(Z, ldz, rows, lse, off, n, UT, L.Kp);
+  count_launch();
+  CKC(cudaGetLastError());
+  return SFB_OK;
+}
+
+int tc_gather(sfb_ctx*) { return SFB_OK; }   // every worker wrote at its offset of U^T and V^T: nothing to move
+
+int tc_update(sfb_ctx* ctx) {
+  const sfb_config& c = ctx->cfg;
+  const TcState* st = static_cast<const TcState*>(ctx->tc);
+  const Layout& L = ctx->lay;
+  CUtensorMap ma, mb, mc;
+  if (!make_map(st, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ctx->at<__nv_bfloat16>(L.UT), ctx->K, c.rows, L.Kp * 2, BK, BM) ||
+      !make_map(st, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ctx->at<__nv_bfloat16>(L.VT), ctx->K, c.cols, L.Kp * 2, BK, BN) ||
+      !make_map(st, &mc, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, ctx->W, c.cols, c.rows, c.cols * 4, kChunk, 32))
+    return SFB_ERR_CUDA;
+  TcParams p{};
+  p.M = static_cast<int32_t>(c.rows); p.N = static_cast<int32_t>(c.cols); p.Kc = static_cast<int32_t>(ctx->K);
+  p.m_off = 0;
+  p.tilesM = static_cast<int32_t>((c.rows + BM - 1) / BM);
+  p.tilesN = static_cast<int32_t>((c.cols + BN - 1) / BN);
+  p.alpha = -c.eta;
+  p.shadow = ctx->at<__nv_bfloat16>(L.Wb); p.shadow_ld = L.colsb;
+  p.status = ctx->at<uint32_t>(L.status);
+  CKC(launch_gemm<TC_UPDATE>(ctx, ma, mb, mc, p));          // W += -eta * P^T V
+  dim3 lgrid(static_cast<unsigned>(ctx->K), static_cast<unsigned>(std::min<int64_t>(16, (c.cols + 1023) / 1024)));
+  label_rows_kernel<<<lgrid, 256, 0, ctx->stream>>>(
+      ctx->W, c.rows, c.cols, ctx->at<float>(L.Xf), ctx->at<int32_t>(L.labels), static_cast<int>(ctx->K), c.eta,
+      ctx->at<__nv_bfloat16>(L.Wb), L.colsb);                // W[y_i] += eta * x_i  (the -onehot part of u_i)
+  count_launch();
+  CKC(cudaGetLastError());
+  return SFB_OK;
+}
+
+int tc_after_update(sfb_ctx*) { return SFB_OK; }
+
+int tc_get_factors(sfb_ctx* ctx, const void** U, const void** V, int32_t* dtype, int32_t* layout, int64_t* ldu,
+                   int64_t* ldv) {
+  if (U) *U = ctx->at<__nv_bfloat16>(ctx->lay.UT);
+  if (V) *V = ctx->at<__nv_bfloat16>(ctx->lay.VT);
+  if (dtype) *dtype = 1;
+  if (layout) *layout = 1;
+  if (ldu) *ldu = ctx->lay.Kp;
+  if (ldv) *ldv = ctx->lay.Kp;
+  return SFB_OK;
+}
+
+}  // namespace sfb

@@ -17,7 +17,7 @@ def small(name):
     """Ragged shapes spanning several 128-wide tiles with tails, same recipes as the full workloads."""
     if name == "mlr":
         return I.scaled(I.WORKLOADS["mlr_mid"], "mlr_small", rows=333, cols=260, workers=3, batch=37, eta=0.05,
-                        w_std=0.3, x_scale="unit")
+                        w_std=0.05, x_scale="unit")
     if name == "dml":
         return I.scaled(I.WORKLOADS["dml"], "dml_small", rows=150, cols=388, workers=4, batch=33, eta=1e-3)
     if name == "sc":
@@ -89,6 +89,9 @@ def test_small_ragged_step_matches_oracle(name, prec):
     assert status == 0
     assert rel_err(Wg, Wref, W0) <= step_tol(wl, prec, Wref, W0)
     ftol = 1e-5 if prec == S.PREC_FP32 else 1e-2
+    if name == "mlr" and prec == S.PREC_BF16:
+        # bf16 mode carries u = p - onehot(y) as (p in bf16, y as an integer): rebuild u from the two
+        Ug[np.arange(wl.K), inp.labels] -= 1.0
     assert np.linalg.norm(Ug - Uref) <= ftol * np.linalg.norm(Uref)
     assert np.linalg.norm(Vg - Vref) <= ftol * max(np.linalg.norm(Vref), 1e-30)
     if name == "mlr":
