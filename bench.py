@@ -179,9 +179,13 @@ def main():
     ap.add_argument("--precision", default="bf16", choices=["bf16", "fp32"])
     ap.add_argument("--workload", default="mlr_large", choices=sorted(I.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--rows", type=int, default=0,
+                    help="run a slab of the workload with this many rows of W (small cases for profiler captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     wl = I.WORKLOADS[args.workload]
+    if args.rows > 0:
+        wl = I.scaled(wl, f"{wl.name}_rows{args.rows}", rows=args.rows)
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))

@@ -35,7 +35,10 @@ typedef struct sfb_ctx sfb_ctx;
 enum sfb_model { SFB_MLR = 0, SFB_DML = 1, SFB_SC = 2 };
 
 /* Operand precision of the matrix products.  The master copy of W is fp32 in both modes.
- * SFB_PREC_BF16: tensor-core products on bf16 operands with fp32 accumulation.
+ * SFB_PREC_BF16: tensor-core products on bf16 operands with fp32 accumulation.  MLR: forward and update
+ *                products on single bf16 operands.  DML, SC: the factors are computed on fp32 operands (u is a
+ *                residual that cancels); the update product runs on the tensor cores with every factor value
+ *                carried as a (hi, lo) pair of bf16, three bf16 products per term.
  * SFB_PREC_FP32: fp32 operands, fp32 FMA accumulation. */
 enum sfb_precision { SFB_PREC_BF16 = 0, SFB_PREC_FP32 = 1 };
 
@@ -130,6 +133,7 @@ int sfb_dense_sync_step(sfb_ctx* ctx, const float* X_dev, const float* Y_dev, co
 
 /* The gathered factor buffers of the last gather, for inspection.  dtype: 0 = fp32, 1 = bf16.
  * layout: 0 = pair-major (U [K x ldu], V [K x ldv]); 1 = transposed (U^T [rows x ldu], V^T [cols x ldv]).
+ * DML and SC return their fp32 pair-major factors in both modes.
  * MLR in bf16 mode keeps u_i = p_i - onehot(y_i) as the pair (p_i in bf16, y_i as int32): the buffer holds the
  * softmax probabilities p_i, and the onehot part is applied to W exactly in fp32 from the class ids. */
 int sfb_get_factors(sfb_ctx* ctx, const void** U_dev, const void** V_dev, int32_t* dtype, int32_t* layout,

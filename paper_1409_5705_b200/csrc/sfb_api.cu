@@ -209,8 +209,10 @@ extern "C" int sfb_compute_factors(sfb_ctx* ctx, int32_t worker, const float* X_
                             ctx->at<float>(ctx->lay.piy), ctx->at<float>(ctx->lay.colpart),
                             ctx->at<Scalars>(ctx->lay.scalars), 50));
   }
-  rc = c.precision == SFB_PREC_FP32 ? factors_fp32(ctx, off, n, X_dev, Y_dev, labels_dev)
-                                    : tc_factors(ctx, off, n, X_dev, Y_dev, labels_dev);
+  // bf16 mode: MLR runs its forward product on the tensor cores; DML and SC need fp32-class factors (their u
+  // comes from a cancelling residual), so only their update product does
+  rc = (c.precision == SFB_PREC_FP32 || c.model != SFB_MLR) ? factors_fp32(ctx, off, n, X_dev, Y_dev, labels_dev)
+                                                            : tc_factors(ctx, off, n, X_dev, Y_dev, labels_dev);
   if (rc) return rc;
   const uint64_t all = c.workers == 64 ? ~0ull : ((1ull << c.workers) - 1);
   ctx->committed |= worker < 0 ? all : (1ull << worker);
@@ -233,7 +235,8 @@ extern "C" int sfb_gather_factors(sfb_ctx* ctx) {
   if (c.model == SFB_MLR)
     CK(mean_of(ctx->stream, ctx->at<float>(ctx->lay.loss), ctx->K,
                &ctx->at<Scalars>(ctx->lay.scalars)->loss_mean));
-  const double esz = c.precision == SFB_PREC_FP32 ? 4.0 : 2.0;
+  // bytes per gathered value: fp32, bf16, or a (hi, lo) pair of bf16 for the split operands of DML and SC
+  const double esz = (c.precision == SFB_PREC_FP32 || c.model != SFB_MLR) ? 4.0 : 2.0;
   const double pair = static_cast<double>(c.rows + c.cols) * esz;
   ctx->stats.gather_bytes += static_cast<double>(ctx->K) * pair;
   ctx->stats.gather_bytes_p2p += static_cast<double>(c.workers) * (c.workers - 1) * c.batch * pair;

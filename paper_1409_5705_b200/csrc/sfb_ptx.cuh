@@ -51,13 +51,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Polls until the phase with this parity has completed.  Gives up (returns false) after kMaxPolls polls
-// or as soon as *abort is set by another role of the CTA.
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Polls until the phase with this parity has completed.  Gives up (returns false) after kMaxWaitNs of wall
+// time or kMaxPolls polls, whichever comes first, or as soon as *abort is set by another role of the CTA.
 constexpr uint32_t kMaxPolls = 1u << 24;
+constexpr uint64_t kMaxWaitNs = 2000000000ull;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
   for (uint32_t i = 0; i < kMaxPolls; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 255u) == 255u && *abort) return false;
+    if ((i & 63u) == 63u) {
+      if (*abort) return false;
+      if (global_timer_ns() - t0 > kMaxWaitNs) break;
+    }
   }
   *abort = 1;
   return false;

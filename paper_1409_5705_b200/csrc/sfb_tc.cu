@@ -47,6 +47,11 @@ struct TcParams {
   int32_t M, N, Kc;            // extents of the product: output rows, output columns, contraction
   int32_t m_off;               // first output row handled by this launch (per-worker slices of the forward)
   int32_t tilesM, tilesN;
+  // The contraction runs over nseg segments of kseg k-blocks; segment s reads A from column a_off[s] and B from
+  // column b_off[s] of their tensors.  One segment is the plain product; three segments over [hi | lo] operand
+  // halves form the split-bf16 product  hi*hi + hi*lo + lo*hi.
+  int32_t nseg, kseg;
+  int32_t a_off[3], b_off[3];
   float alpha;                 // TC_UPDATE: -eta
   __nv_bfloat16* shadow;       // TC_UPDATE: bf16 copy of the updated W, row pitch shadow_ld elements (or null)
   int64_t shadow_ld;
@@ -84,7 +89,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int ntiles = p.tilesM * p.tilesN;
-  const int numK = (p.Kc + BK - 1) / BK;
+  const int numK = p.nseg * p.kseg;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < S; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
@@ -110,16 +115,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
         int m0, n0;
         tile_coords(p, tile, m0, n0);
-        for (int kb = 0; kb < numK; ++kb, ++it) {
-          const uint32_t s = it % S, ph = (it / S) & 1;
-          if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
-          mbar_expect_tx(&full[s], kBytesA + kBytesB);
-          if (EPI == TC_UPDATE) {
-            tma_load_2d(sA + s * kBytesA, &tmA, kb * BK, m0, &full[s]);
-            tma_load_2d_hint(sB + s * kBytesB, &tmB, kb * BK, n0, &full[s], pol_keep);
-          } else {
-            tma_load_2d_hint(sA + s * kBytesA, &tmA, kb * BK, m0, &full[s], pol_keep);
-            tma_load_2d(sB + s * kBytesB, &tmB, kb * BK, n0, &full[s]);
+        for (int seg = 0; seg < p.nseg && ok; ++seg) {
+          for (int kl = 0; kl < p.kseg; ++kl, ++it) {
+            const uint32_t s = it % S, ph = (it / S) & 1;
+            if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
+            mbar_expect_tx(&full[s], kBytesA + kBytesB);
+            const int xa = p.a_off[seg] + kl * BK, xb = p.b_off[seg] + kl * BK;
+            if (EPI == TC_UPDATE) {
+              tma_load_2d(sA + s * kBytesA, &tmA, xa, m0, &full[s]);
+              tma_load_2d_hint(sB + s * kBytesB, &tmB, xb, n0, &full[s], pol_keep);
+            } else {
+              tma_load_2d_hint(sA + s * kBytesA, &tmA, xa, m0, &full[s], pol_keep);
+              tma_load_2d(sB + s * kBytesB, &tmB, xb, n0, &full[s]);
+            }
           }
         }
       }
@@ -379,6 +387,52 @@ __global__ void __launch_bounds__(256) pack_mlr_kernel(const float* __restrict__
   }
 }
 
+// Gathered fp32 factors F [n x dim] (pair-major) -> the split-bf16 operand of the update product,
+// FT [dim x 2*Kp] (samples contiguous): FT[c][i] = hi(F[i][c]), FT[c][Kp + i] = lo(F[i][c]) with
+// hi = bf16(f), lo = bf16(f - hi); samples n..Kp-1 are written as zeros.  64 x 64 tiles through shared memory.
+__global__ void __launch_bounds__(256) pack_split_t_kernel(const float* __restrict__ F, int64_t n, int64_t dim,
+                                                           __nv_bfloat16* __restrict__ FT, int64_t Kp) {
+  __shared__ float tile[64][65];
+  const int64_t i0 = static_cast<int64_t>(blockIdx.y) * 64, c0 = static_cast<int64_t>(blockIdx.x) * 64;
+  const int t = threadIdx.x;
+  const bool vec = (dim % 4) == 0;
+#pragma unroll
+  for (int v = 0; v < 4; ++v) {
+    const int idx = t + v * 256;            // 64 samples x 16 quads
+    const int i = idx / 16, cq = (idx % 16) * 4;
+    float f[4] = {0.f, 0.f, 0.f, 0.f};
+    if (i0 + i < n) {
+      const float* src = F + (i0 + i) * dim + c0 + cq;
+      if (vec && c0 + cq + 3 < dim) {
+        const float4 q4 = *reinterpret_cast<const float4*>(src);
+        f[0] = q4.x; f[1] = q4.y; f[2] = q4.z; f[3] = q4.w;
+      } else {
+        for (int k = 0; k < 4; ++k)
+          if (c0 + cq + k < dim) f[k] = src[k];
+      }
+    }
+    tile[i][cq + 0] = f[0]; tile[i][cq + 1] = f[1]; tile[i][cq + 2] = f[2]; tile[i][cq + 3] = f[3];
+  }
+  __syncthreads();
+#pragma unroll
+  for (int v = 0; v < 2; ++v) {
+    const int idx = t + v * 256;            // 64 features x 8 groups of 8 samples
+    const int c = idx / 8, ig = (idx % 8) * 8;
+    if (c0 + c >= dim) continue;
+    uint32_t hi[4], lo[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const float f0 = tile[ig + 2 * k][c], f1 = tile[ig + 2 * k + 1][c];
+      const __nv_bfloat16 h0 = __float2bfloat16_rn(f0), h1 = __float2bfloat16_rn(f1);
+      hi[k] = static_cast<uint32_t>(__bfloat16_as_ushort(h0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(h1)) << 16);
+      lo[k] = pack_bf16(f0 - __bfloat162float(h0), f1 - __bfloat162float(h1));
+    }
+    __nv_bfloat16* dst = FT + (c0 + c) * 2 * Kp + i0 + ig;     // Kp is a multiple of 64: 16-byte aligned
+    *reinterpret_cast<uint4*>(dst) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+    *reinterpret_cast<uint4*>(dst + Kp) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+  }
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -567,6 +621,14 @@ void tc_extend_layout(const sfb_config& c, Layout& L, size_t& off) {
   const size_t K = static_cast<size_t>(c.workers) * c.batch;
   L.Kp = round_up(static_cast<int64_t>(K), 64);
   L.colsb = round_up(c.cols, 64);
+  if (c.model != SFB_MLR) {
+    // fp32 factors as the workers write them, and their split-bf16 transposes for the update product
+    L.V = take(K * static_cast<size_t>(c.cols) * 4);
+    L.U = take(K * static_cast<size_t>(c.rows) * 4);
+    L.UT = take(static_cast<size_t>(c.rows) * 2 * L.Kp * 2);
+    L.VT = take(static_cast<size_t>(c.cols) * 2 * L.Kp * 2);
+    return;
+  }
   const size_t ldz = static_cast<size_t>(round_up(c.rows, 32));
   const size_t nblk = static_cast<size_t>((c.rows + BN - 1) / BN);
   L.Wb = take(static_cast<size_t>(c.rows) * L.colsb * 2);
@@ -582,7 +644,6 @@ void tc_extend_layout(const sfb_config& c, Layout& L, size_t& off) {
 }
 
 int tc_init(sfb_ctx* ctx) {
-  if (ctx->cfg.model != SFB_MLR) return SFB_ERR_UNSUPPORTED;
   TcState* st = new (std::nothrow) TcState();
   if (!st) return SFB_ERR_ARG;
   ctx->tc = st;
@@ -595,6 +656,7 @@ int tc_init(sfb_ctx* ctx) {
   CKC(cudaGetDevice(&dev));
   CKC(cudaDeviceGetAttribute(&st->sms, cudaDevAttrMultiProcessorCount, dev));
   const sfb_config& c = ctx->cfg;
+  if (c.model != SFB_MLR) return SFB_OK;        // the forward products of DML and SC run on fp32 operands
   // bf16 copy of W for the forward product; afterwards the update's epilogue keeps it current
   convert_rows_kernel<<<148 * 8, 256, 0, ctx->stream>>>(ctx->W, c.rows, c.cols, ctx->at<__nv_bfloat16>(ctx->lay.Wb),
                                                         ctx->lay.colsb);
@@ -642,6 +704,7 @@ int tc_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float
   p.tilesM = static_cast<int32_t>((n + BM - 1) / BM);
   p.tilesN = static_cast<int32_t>((rows + BN - 1) / BN);
   p.part = part; p.part_ld = K; p.status = status;
+  p.nseg = 1; p.kseg = (p.Kc + BK - 1) / BK;
   CKC(launch_gemm<TC_FORWARD>(ctx, ma, mb, mc, p));
   ctx->stats.flops += 2.0 * n * rows * cols;
 
@@ -655,15 +718,33 @@ int tc_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float
   return SFB_OK;
 }
 
-int tc_gather(sfb_ctx*) { return SFB_OK; }   // every worker wrote at its offset of U^T and V^T: nothing to move
+// MLR: every worker wrote at its offset of U^T and V^T, nothing to move.  DML, SC: the workers' fp32 factors
+// are transposed into the split-bf16 operands of the update product.
+int tc_gather(sfb_ctx* ctx) {
+  const sfb_config& c = ctx->cfg;
+  if (c.model == SFB_MLR) return SFB_OK;
+  const Layout& L = ctx->lay;
+  const unsigned gy = static_cast<unsigned>(L.Kp / 64);
+  pack_split_t_kernel<<<dim3(static_cast<unsigned>((c.rows + 63) / 64), gy), 256, 0, ctx->stream>>>(
+      ctx->at<float>(L.U), ctx->K, c.rows, ctx->at<__nv_bfloat16>(L.UT), L.Kp);
+  count_launch();
+  pack_split_t_kernel<<<dim3(static_cast<unsigned>((c.cols + 63) / 64), gy), 256, 0, ctx->stream>>>(
+      ctx->at<float>(L.V), ctx->K, c.cols, ctx->at<__nv_bfloat16>(L.VT), L.Kp);
+  count_launch();
+  CKC(cudaGetLastError());
+  return SFB_OK;
+}
 
 int tc_update(sfb_ctx* ctx) {
   const sfb_config& c = ctx->cfg;
   const TcState* st = static_cast<const TcState*>(ctx->tc);
   const Layout& L = ctx->lay;
+  const bool split = c.model != SFB_MLR;
+  const int64_t kw = split ? 2 * L.Kp : ctx->K;       // operand width in elements; pitch is Kp or 2*Kp
+  const int64_t pitch = (split ? 2 * L.Kp : L.Kp) * 2;
   CUtensorMap ma, mb, mc;
-  if (!make_map(st, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ctx->at<__nv_bfloat16>(L.UT), ctx->K, c.rows, L.Kp * 2, BK, BM) ||
-      !make_map(st, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ctx->at<__nv_bfloat16>(L.VT), ctx->K, c.cols, L.Kp * 2, BK, BN) ||
+  if (!make_map(st, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ctx->at<__nv_bfloat16>(L.UT), kw, c.rows, pitch, BK, BM) ||
+      !make_map(st, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ctx->at<__nv_bfloat16>(L.VT), kw, c.cols, pitch, BK, BN) ||
       !make_map(st, &mc, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, ctx->W, c.cols, c.rows, c.cols * 4, kChunk, 32))
     return SFB_ERR_CUDA;
   TcParams p{};
@@ -672,8 +753,19 @@ int tc_update(sfb_ctx* ctx) {
   p.tilesM = static_cast<int32_t>((c.rows + BM - 1) / BM);
   p.tilesN = static_cast<int32_t>((c.cols + BN - 1) / BN);
   p.alpha = -c.eta;
-  p.shadow = ctx->at<__nv_bfloat16>(L.Wb); p.shadow_ld = L.colsb;
+  p.kseg = static_cast<int32_t>(L.Kp / BK);
   p.status = ctx->at<uint32_t>(L.status);
+  if (split) {
+    // U^T V = Uhi Vhi + Uhi Vlo + Ulo Vhi (+ Ulo Vlo, dropped: 2^-16 of the product)
+    p.nseg = 3;
+    p.a_off[0] = 0; p.a_off[1] = 0; p.a_off[2] = static_cast<int32_t>(L.Kp);
+    p.b_off[0] = 0; p.b_off[1] = static_cast<int32_t>(L.Kp); p.b_off[2] = 0;
+    p.shadow = nullptr; p.shadow_ld = 0;
+    CKC(launch_gemm<TC_UPDATE>(ctx, ma, mb, mc, p));
+    return SFB_OK;
+  }
+  p.nseg = 1;
+  p.shadow = ctx->at<__nv_bfloat16>(L.Wb); p.shadow_ld = L.colsb;
   CKC(launch_gemm<TC_UPDATE>(ctx, ma, mb, mc, p));          // W += -eta * P^T V
   dim3 lgrid(static_cast<unsigned>(ctx->K), static_cast<unsigned>(std::min<int64_t>(16, (c.cols + 1023) / 1024)));
   label_rows_kernel<<<lgrid, 256, 0, ctx->stream>>>(
@@ -688,6 +780,15 @@ int tc_after_update(sfb_ctx*) { return SFB_OK; }
 
 int tc_get_factors(sfb_ctx* ctx, const void** U, const void** V, int32_t* dtype, int32_t* layout, int64_t* ldu,
                    int64_t* ldv) {
+  if (ctx->cfg.model != SFB_MLR) {   // the workers' fp32 factors, pair-major
+    if (U) *U = ctx->at<float>(ctx->lay.U);
+    if (V) *V = ctx->at<float>(ctx->lay.V);
+    if (dtype) *dtype = 0;
+    if (layout) *layout = 0;
+    if (ldu) *ldu = ctx->cfg.rows;
+    if (ldv) *ldv = ctx->cfg.cols;
+    return SFB_OK;
+  }
   if (U) *U = ctx->at<__nv_bfloat16>(ctx->lay.UT);
   if (V) *V = ctx->at<__nv_bfloat16>(ctx->lay.VT);
   if (dtype) *dtype = 1;

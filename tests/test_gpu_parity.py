@@ -107,7 +107,7 @@ def test_small_ragged_step_matches_oracle(name, prec):
         assert (norms <= 1 + 1e-6).all()
         assert abs(stats.sc_lipschitz - L) <= 1e-6 * L
     # the byte report of the cost table
-    esz = 4 if prec == S.PREC_FP32 else 2
+    esz = 2 if (prec == S.PREC_BF16 and name == "mlr") else 4     # DML, SC: fp32 or a (hi, lo) bf16 pair
     one, p2p, fms = O.comm_values(wl.rows, wl.cols, wl.workers, wl.batch)
     assert stats.gather_bytes == one * esz and stats.gather_bytes_p2p == p2p * esz
     assert stats.dense_sync_bytes == fms * 4
