@@ -1,17 +1,11 @@
-// Tensor-core (bf16 operand) path of the SFB step on sm_100a.
+// Tensor-core (bf16 operand) path of the SFB step on sm_100a: sufficient-factor computation for multiclass
+// logistic regression (Sections 1 and 2: u = softmax(W x) - onehot(y), v = x) and the operand packing of the
+// update product.  The update product itself is in sfb_update.cu.
 //
-// One persistent, warp-specialised kernel computes  D (M x N) = A (M x Kc) * B (N x Kc)^T  with bf16 operands
-// staged by TMA into 128-byte-swizzled shared memory, tcgen05.mma accumulating in TMEM (two 128 x 256 fp32
-// accumulators, so the epilogue of one tile overlaps the main loop of the next), and one of two epilogues:
-//
-//   TC_UPDATE   W <- W + alpha * D   (Section 3, Figure 1: reconstruct the K rank-1 updates and apply them).
-//               A = U^T [rows x K], B = V^T [cols x K].  The fp32 tile of W is brought in by TMA while the MMAs
-//               run, modified in shared memory and stored back by TMA: W makes one HBM round trip per step.
-//               A bf16 copy of the new W (the operand of the next step's forward product) is written alongside.
-//   TC_FORWARD  Z = D stored as fp32, plus per (sample, 256-row block) softmax partials (max, sum of exp)
-//               (Section 2: the products W a_i, batched; Section 1: u is the prediction vector).
-//               A = X [K x cols] (samples on the TMEM lanes), B = W [rows x cols].
-//
+// Forward product: one persistent, warp-specialised kernel computes  Z (K x rows) = X (K x cols) * W^T  with bf16
+// operands staged by TMA into 128-byte-swizzled shared memory, tcgen05.mma accumulating in TMEM (two 128 x 256
+// fp32 accumulators, so the epilogue of one tile overlaps the main loop of the next).  The epilogue stores Z as
+// fp32 and, per (sample, 256-row block), the softmax partials (max, sum of exp).
 // Roles: warp 0 TMA producer, warp 1 MMA issuer (and TMEM owner), warps 2-5 epilogue (one TMEM lane quarter each).
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -31,48 +25,34 @@ constexpr int BM = 128, BN = 256, BK = 64, UMMA_K = 16;
 constexpr int kBytesA = BM * BK * 2, kBytesB = BN * BK * 2;
 constexpr int kChunk = 32;                 // accumulator columns handled per epilogue step
 constexpr int kSlotBytes = 32 * kChunk * 4;  // one warp's 32 rows x 32 fp32 columns
-constexpr int kThreads = 192;
 constexpr int kTmemCols = 512;
-
-enum TcEpi { TC_UPDATE = 0, TC_FORWARD = 1 };
-
-template <int EPI> struct Shape {
-  static constexpr int S = EPI == TC_UPDATE ? 3 : 4;   // operand pipeline stages
-  static constexpr int R = EPI == TC_UPDATE ? 5 : 2;   // epilogue ring slots per warp
-  static constexpr int kBars = 2 * S + 4 + 4 * R;
-  static constexpr int kSmem = S * (kBytesA + kBytesB) + 4 * R * kSlotBytes + kBars * 8 + 16 + 1024;
-};
+constexpr int S = 4;                      // operand pipeline stages
+constexpr int R = 2;                      // epilogue ring slots per warp
+constexpr int kEpiWarps = 4;
+constexpr int kThreads = 64 + 32 * kEpiWarps;
+constexpr int kBars = 2 * S + 4;
+constexpr int kSmem = S * (kBytesA + kBytesB) + kEpiWarps * R * kSlotBytes + kBars * 8 + 16 + 1024;
 
 struct TcParams {
-  int32_t M, N, Kc;            // extents of the product: output rows, output columns, contraction
-  int32_t m_off;               // first output row handled by this launch (per-worker slices of the forward)
+  int32_t M, N, Kc;            // extents of the product: samples, rows of W, features
+  int32_t m_off;               // first sample handled by this launch (per-worker slices)
   int32_t tilesM, tilesN;
-  // The contraction runs over nseg segments of kseg k-blocks; segment s reads A from column a_off[s] and B from
-  // column b_off[s] of their tensors.  One segment is the plain product; three segments over [hi | lo] operand
-  // halves form the split-bf16 product  hi*hi + hi*lo + lo*hi.
-  int32_t nseg, kseg;
-  int32_t a_off[3], b_off[3];
-  float alpha;                 // TC_UPDATE: -eta
-  __nv_bfloat16* shadow;       // TC_UPDATE: bf16 copy of the updated W, row pitch shadow_ld elements (or null)
-  int64_t shadow_ld;
-  float2* part;                // TC_FORWARD: [tilesN][part_ld] (max, sum exp) per sample and column block
+  float2* part;                // [tilesN][part_ld] (max, sum exp) per sample and 256-row block
   int64_t part_ld;
   uint32_t* status;
 };
 
+// Tiles are numbered with the sample block fastest: consecutive tiles (which run on different SMs at the same
+// time) share one block of W, which therefore stays hot in L2 while all K samples are swept past it.
 __device__ __forceinline__ void tile_coords(const TcParams& p, int tile, int& m0, int& n0) {
-  int tm, tn;
-  if (p.tilesM <= 8) { tm = tile % p.tilesM; tn = tile / p.tilesM; }   // few row blocks: keep a B block hot in L2
-  else { tn = tile % p.tilesN; tm = tile / p.tilesN; }                 // update: sweep the columns of one row block
+  const int tm = tile % p.tilesM, tn = tile / p.tilesM;
   m0 = p.m_off + tm * BM;
   n0 = tn * BN;
 }
 
-template <int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
-tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+forward_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmC, const TcParams p) {
-  constexpr int S = Shape<EPI>::S, R = Shape<EPI>::R;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sA = smem;
@@ -83,18 +63,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   uint64_t* empty = bars + S;
   uint64_t* tfull = bars + 2 * S;
   uint64_t* tempty = bars + 2 * S + 2;
-  uint64_t* rfull = bars + 2 * S + 4;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + Shape<EPI>::kBars);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kBars);
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int ntiles = p.tilesM * p.tilesN;
-  const int numK = p.nseg * p.kseg;
+  const int numK = (p.Kc + BK - 1) / BK;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < S; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&tfull[i], 1); mbar_init(&tempty[i], 4); }
-    for (int i = 0; i < 4 * R; ++i) mbar_init(&rfull[i], 1);
     *abort_flag = 0;
     fence_barrier_init();
     prefetch_tmap(&tmA); prefetch_tmap(&tmB); prefetch_tmap(&tmC);
@@ -108,27 +86,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
-      // The small operand every tile re-reads (V^T in the update, X in the forward) is pinned in L2.
+      // A (the K samples) is the small operand every tile re-reads: pinned in L2.
       const uint64_t pol_keep = policy_evict_last();
       uint32_t it = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
         int m0, n0;
         tile_coords(p, tile, m0, n0);
-        for (int seg = 0; seg < p.nseg && ok; ++seg) {
-          for (int kl = 0; kl < p.kseg; ++kl, ++it) {
-            const uint32_t s = it % S, ph = (it / S) & 1;
-            if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
-            mbar_expect_tx(&full[s], kBytesA + kBytesB);
-            const int xa = p.a_off[seg] + kl * BK, xb = p.b_off[seg] + kl * BK;
-            if (EPI == TC_UPDATE) {
-              tma_load_2d(sA + s * kBytesA, &tmA, xa, m0, &full[s]);
-              tma_load_2d_hint(sB + s * kBytesB, &tmB, xb, n0, &full[s], pol_keep);
-            } else {
-              tma_load_2d_hint(sA + s * kBytesA, &tmA, xa, m0, &full[s], pol_keep);
-              tma_load_2d(sB + s * kBytesB, &tmB, xb, n0, &full[s]);
-            }
-          }
+        for (int kb = 0; kb < numK; ++kb, ++it) {
+          const uint32_t s = it % S, ph = (it / S) & 1;
+          if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
+          mbar_expect_tx(&full[s], kBytesA + kBytesB);
+          tma_load_2d_hint(sA + s * kBytesA, &tmA, kb * BK, m0, &full[s], pol_keep);
+          tma_load_2d(sB + s * kBytesB, &tmB, kb * BK, n0, &full[s]);
         }
       }
     }
@@ -162,101 +132,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // ---------------- epilogue: warps 2..5, TMEM lane quarter q ----------------
     const int q = warp & 3;
     uint8_t* ring = sRing + q * R * kSlotBytes;
-    uint64_t* rf = rfull + q * R;
     const int my_tiles = blockIdx.x < ntiles ? (ntiles - 1 - blockIdx.x) / gridDim.x + 1 : 0;
-    const uint32_t nchunks = static_cast<uint32_t>(my_tiles) * (BN / kChunk);
     bool ok = true;
 
-    if constexpr (EPI == TC_UPDATE) {
-      // Per warp: kLoadSlots ring slots receive W chunks by TMA (issued kLoadSlots chunks ahead, refilled as soon
-      // as the warp has read them) and 2 staging slots carry the updated chunks to the TMA stores.  The TMEM
-      // load of chunk c+1 is in flight while chunk c is combined with W.
-      constexpr int kLoadSlots = R - 2;
-      constexpr int kChunksPerTile = BN / kChunk;
-      uint8_t* stage = ring + kLoadSlots * kSlotBytes;
-      const uint64_t pol_stream = policy_evict_first();
-      // chunk g+kLoadSlots is always requested while chunk g is processed: track its tile incrementally
-      uint32_t lg = 0;                 // next chunk to request
-      int ltile = blockIdx.x, lc = 0;  // its tile and chunk-in-tile
-      auto issue_load = [&]() {
-        if (lg >= nchunks) return;
-        int m0, n0;
-        tile_coords(p, ltile, m0, n0);
-        const uint32_t slot = lg % kLoadSlots;
-        mbar_expect_tx(&rf[slot], kSlotBytes);
-        tma_load_2d_hint(ring + slot * kSlotBytes, &tmC, n0 + lc * kChunk, m0 + q * 32, &rf[slot], pol_stream);
-        ++lg;
-        if (++lc == kChunksPerTile) { lc = 0; ltile += gridDim.x; }
-      };
-      if (lane == 0)
-        for (int i = 0; i < kLoadSlots; ++i) issue_load();
-      uint32_t g = 0;
-      for (int tl = 0; tl < my_tiles && ok; ++tl) {
-        int m0, n0;
-        tile_coords(p, blockIdx.x + tl * gridDim.x, m0, n0);
-        const uint32_t a = tl & 1, aph = (tl >> 1) & 1;
-        if (!__all_sync(0xffffffffu, mbar_wait(&tfull[a], aph, abort_flag))) { ok = false; break; }
-        tc_fence_after();
-        const int row = m0 + q * 32 + lane;
-        const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + a * BN;
-        uint32_t acc0[32], acc1[32];
-        tmem_ld_32x32(t_addr, acc0);
-        auto process = [&](uint32_t (&acc)[32], uint32_t (&nxt)[32], int c) -> bool {
-          tmem_ld_wait();                                      // chunk c's accumulators are in registers
-          if (c + 1 < kChunksPerTile) {
-            tmem_ld_32x32(t_addr + (c + 1) * kChunk, nxt);     // chunk c+1 streams in during this chunk's work
-          } else {
-            tc_fence_before();                                 // last TMEM read of the tile: hand the
-            __syncwarp();                                      // accumulator back to the MMA warp now
-            if (lane == 0) mbar_arrive(&tempty[a]);
-          }
-          const uint32_t slot = g % kLoadSlots;
-          const uint8_t* sl = ring + slot * kSlotBytes;
-          uint8_t* st = stage + (g & 1) * kSlotBytes;
-          if (!__all_sync(0xffffffffu, mbar_wait(&rf[slot], (g / kLoadSlots) & 1, abort_flag))) return false;
-          if (lane == 0) tma_wait_group_read<1>();             // the store two chunks back has read `st`
-          __syncwarp();
-          const int col0 = n0 + c * kChunk;
-          uint32_t packed[16];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const int o = lane * 128 + ((j ^ (lane & 7)) << 4);
-            float4 w = *reinterpret_cast<const float4*>(sl + o);
-            w.x = fmaf(p.alpha, __uint_as_float(acc[4 * j + 0]), w.x);
-            w.y = fmaf(p.alpha, __uint_as_float(acc[4 * j + 1]), w.y);
-            w.z = fmaf(p.alpha, __uint_as_float(acc[4 * j + 2]), w.z);
-            w.w = fmaf(p.alpha, __uint_as_float(acc[4 * j + 3]), w.w);
-            *reinterpret_cast<float4*>(st + o) = w;
-            __nv_bfloat162 lo = __floats2bfloat162_rn(w.x, w.y), hi = __floats2bfloat162_rn(w.z, w.w);
-            packed[2 * j + 0] = *reinterpret_cast<uint32_t*>(&lo);
-            packed[2 * j + 1] = *reinterpret_cast<uint32_t*>(&hi);
-          }
-          fence_proxy_async_smem();
-          __syncwarp();                                        // every lane has read `sl` and written `st`
-          if (lane == 0) {
-            tma_store_2d_hint(&tmC, st, col0, m0 + q * 32, pol_stream);
-            tma_commit_group();
-            issue_load();                                      // refill the slot just consumed
-          }
-          if (p.shadow != nullptr && row < p.M) {
-            __nv_bfloat16* dst = p.shadow + static_cast<int64_t>(row) * p.shadow_ld + col0;
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-              if (col0 + 8 * j < p.shadow_ld)
-                *reinterpret_cast<uint4*>(dst + 8 * j) =
-                    make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
-          }
-          ++g;
-          return true;
-        };
-#pragma unroll 1
-        for (int c = 0; c < kChunksPerTile && ok; c += 2) {
-          ok = process(acc0, acc1, c);
-          if (ok) ok = process(acc1, acc0, c + 1);
-        }
-      }
-      if (lane == 0) tma_wait_group<0>();
-    } else {
+    {
       // Forward: store Z through the ring and keep a running (max, sum exp) per sample over the tile's columns.
       uint32_t gs = 0;                       // stores issued so far: consecutive stores alternate ring slots
       for (int tl = 0; tl < my_tiles && ok; ++tl) {
@@ -522,85 +401,21 @@ __global__ void __launch_bounds__(256) mlr_emit_ut_kernel(const float* __restric
   }
 }
 
-// The onehot part of the K factors, sum_i (-e_{y_i}) x_i^T, applied to W in fp32 after the tensor-core product
-// has applied sum_i p_i x_i^T:  W[y] <- W[y] + eta * sum_{i : y_i = y} x_i.  One block per sample; the block of
-// the first sample of each class sums that class's samples in index order (no atomics: same result every
-// run) and refreshes the bf16 copy of the row.
-__global__ void __launch_bounds__(256) label_rows_kernel(float* __restrict__ W, int64_t rows, int64_t cols,
-                                                         const float* __restrict__ Xf, const int32_t* __restrict__ labels,
-                                                         int K, float eta, __nv_bfloat16* __restrict__ shadow,
-                                                         int64_t shadow_ld) {
-  __shared__ int first;
-  const int i = blockIdx.x;
-  const int32_t y = labels[i];
-  if (y < 0 || y >= rows) return;              // out-of-range ids were flagged by the softmax pass
-  if (threadIdx.x == 0) first = 1;
-  __syncthreads();
-  for (int j = threadIdx.x; j < i; j += 256)
-    if (labels[j] == y) first = 0;
-  __syncthreads();
-  if (!first) return;
-  for (int64_t c = (static_cast<int64_t>(blockIdx.y) * 256 + threadIdx.x) * 4; c < cols;
-       c += static_cast<int64_t>(gridDim.y) * 256 * 4) {
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int j = i; j < K; ++j) {
-      if (labels[j] != y) continue;
-      const float4 x = *reinterpret_cast<const float4*>(Xf + static_cast<int64_t>(j) * cols + c);
-      acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
-    }
-    float4* wp = reinterpret_cast<float4*>(W + static_cast<int64_t>(y) * cols + c);
-    float4 w = *wp;
-    w.x = fmaf(eta, acc.x, w.x); w.y = fmaf(eta, acc.y, w.y);
-    w.z = fmaf(eta, acc.z, w.z); w.w = fmaf(eta, acc.w, w.w);
-    *wp = w;
-    if (shadow)
-      *reinterpret_cast<uint2*>(shadow + static_cast<int64_t>(y) * shadow_ld + c) =
-          make_uint2(pack_bf16(w.x, w.y), pack_bf16(w.z, w.w));
-  }
-}
-
 // ---------------------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-struct TcState {
-  EncodeTiledFn encode;
-  int sms;
-};
-
-inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
-
-// 2-D row-major tensor [outer x inner] with row pitch `pitch_bytes`, box [box_outer x box_inner], 128-byte swizzle.
-bool make_map(const TcState* st, CUtensorMap* m, CUtensorMapDataType dt, int esz, void* base, int64_t inner,
-              int64_t outer, int64_t pitch_bytes, int box_inner, int box_outer) {
-  if (inner <= 0 || outer <= 0) return false;
-  cuuint64_t dims[2] = {static_cast<cuuint64_t>(inner), static_cast<cuuint64_t>(outer)};
-  cuuint64_t strides[1] = {static_cast<cuuint64_t>(pitch_bytes)};
-  cuuint32_t box[2] = {static_cast<cuuint32_t>(box_inner), static_cast<cuuint32_t>(box_outer)};
-  cuuint32_t estr[2] = {1, 1};
-  (void)esz;
-  return st->encode(m, dt, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-template <int EPI>
-cudaError_t launch_gemm(sfb_ctx* ctx, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c, TcParams p) {
+cudaError_t launch_forward(sfb_ctx* ctx, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c, TcParams p) {
   const TcState* st = static_cast<const TcState*>(ctx->tc);
-  static bool attr_set[2] = {false, false};
-  if (!attr_set[EPI]) {
-    cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         Shape<EPI>::kSmem);
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
-    attr_set[EPI] = true;
+    attr_set = true;
   }
   const int64_t tiles = static_cast<int64_t>(p.tilesM) * p.tilesN;
   if (tiles <= 0) return cudaSuccess;
   const int grid = static_cast<int>(tiles < st->sms ? tiles : st->sms);
-  tc_gemm_kernel<EPI><<<grid, kThreads, Shape<EPI>::kSmem, ctx->stream>>>(a, b, c, p);
+  forward_kernel<<<grid, kThreads, kSmem, ctx->stream>>>(a, b, c, p);
   count_launch();
   return cudaGetLastError();
 }
@@ -655,6 +470,10 @@ int tc_init(sfb_ctx* ctx) {
   int dev = 0;
   CKC(cudaGetDevice(&dev));
   CKC(cudaDeviceGetAttribute(&st->sms, cudaDevAttrMultiProcessorCount, dev));
+  {
+    const int rc = tc_update_init(ctx, st);
+    if (rc) return rc;
+  }
   const sfb_config& c = ctx->cfg;
   if (c.model != SFB_MLR) return SFB_OK;        // the forward products of DML and SC run on fp32 operands
   // bf16 copy of W for the forward product; afterwards the update's epilogue keeps it current
@@ -694,9 +513,9 @@ int tc_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float
 
   // Z[off .. off+n) = X W^T : samples on the lanes (A), rows of W on the accumulator columns (B)
   CUtensorMap ma, mb, mc;
-  if (!make_map(st, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Xb, cols, off + n, L.colsb * 2, BK, BM) ||
-      !make_map(st, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Wb, cols, rows, L.colsb * 2, BK, BN) ||
-      !make_map(st, &mc, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, Z, rows, off + n, ldz * 4, kChunk, 32))
+  if (!make_map(st, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, Xb, cols, off + n, L.colsb * 2, BK, BM) ||
+      !make_map(st, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, Wb, cols, rows, L.colsb * 2, BK, BN) ||
+      !make_map(st, &mc, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, Z, rows, off + n, ldz * 4, kChunk, 32))
     return SFB_ERR_CUDA;
   TcParams p{};
   p.M = static_cast<int32_t>(off + n); p.N = static_cast<int32_t>(rows); p.Kc = static_cast<int32_t>(cols);
@@ -704,8 +523,7 @@ int tc_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float
   p.tilesM = static_cast<int32_t>((n + BM - 1) / BM);
   p.tilesN = static_cast<int32_t>((rows + BN - 1) / BN);
   p.part = part; p.part_ld = K; p.status = status;
-  p.nseg = 1; p.kseg = (p.Kc + BK - 1) / BK;
-  CKC(launch_gemm<TC_FORWARD>(ctx, ma, mb, mc, p));
+  CKC(launch_forward(ctx, ma, mb, mc, p));
   ctx->stats.flops += 2.0 * n * rows * cols;
 
   mlr_lse_kernel<<<static_cast<unsigned>((n + 7) / 8), 256, 0, ctx->stream>>>(part, K, p.tilesN, Z, ldz, rows, labels, off,
@@ -730,47 +548,6 @@ int tc_gather(sfb_ctx* ctx) {
   count_launch();
   pack_split_t_kernel<<<dim3(static_cast<unsigned>((c.cols + 63) / 64), gy), 256, 0, ctx->stream>>>(
       ctx->at<float>(L.V), ctx->K, c.cols, ctx->at<__nv_bfloat16>(L.VT), L.Kp);
-  count_launch();
-  CKC(cudaGetLastError());
-  return SFB_OK;
-}
-
-int tc_update(sfb_ctx* ctx) {
-  const sfb_config& c = ctx->cfg;
-  const TcState* st = static_cast<const TcState*>(ctx->tc);
-  const Layout& L = ctx->lay;
-  const bool split = c.model != SFB_MLR;
-  const int64_t kw = split ? 2 * L.Kp : ctx->K;       // operand width in elements; pitch is Kp or 2*Kp
-  const int64_t pitch = (split ? 2 * L.Kp : L.Kp) * 2;
-  CUtensorMap ma, mb, mc;
-  if (!make_map(st, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ctx->at<__nv_bfloat16>(L.UT), kw, c.rows, pitch, BK, BM) ||
-      !make_map(st, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ctx->at<__nv_bfloat16>(L.VT), kw, c.cols, pitch, BK, BN) ||
-      !make_map(st, &mc, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, ctx->W, c.cols, c.rows, c.cols * 4, kChunk, 32))
-    return SFB_ERR_CUDA;
-  TcParams p{};
-  p.M = static_cast<int32_t>(c.rows); p.N = static_cast<int32_t>(c.cols); p.Kc = static_cast<int32_t>(ctx->K);
-  p.m_off = 0;
-  p.tilesM = static_cast<int32_t>((c.rows + BM - 1) / BM);
-  p.tilesN = static_cast<int32_t>((c.cols + BN - 1) / BN);
-  p.alpha = -c.eta;
-  p.kseg = static_cast<int32_t>(L.Kp / BK);
-  p.status = ctx->at<uint32_t>(L.status);
-  if (split) {
-    // U^T V = Uhi Vhi + Uhi Vlo + Ulo Vhi (+ Ulo Vlo, dropped: 2^-16 of the product)
-    p.nseg = 3;
-    p.a_off[0] = 0; p.a_off[1] = 0; p.a_off[2] = static_cast<int32_t>(L.Kp);
-    p.b_off[0] = 0; p.b_off[1] = static_cast<int32_t>(L.Kp); p.b_off[2] = 0;
-    p.shadow = nullptr; p.shadow_ld = 0;
-    CKC(launch_gemm<TC_UPDATE>(ctx, ma, mb, mc, p));
-    return SFB_OK;
-  }
-  p.nseg = 1;
-  p.shadow = ctx->at<__nv_bfloat16>(L.Wb); p.shadow_ld = L.colsb;
-  CKC(launch_gemm<TC_UPDATE>(ctx, ma, mb, mc, p));          // W += -eta * P^T V
-  dim3 lgrid(static_cast<unsigned>(ctx->K), static_cast<unsigned>(std::min<int64_t>(16, (c.cols + 1023) / 1024)));
-  label_rows_kernel<<<lgrid, 256, 0, ctx->stream>>>(
-      ctx->W, c.rows, c.cols, ctx->at<float>(L.Xf), ctx->at<int32_t>(L.labels), static_cast<int>(ctx->K), c.eta,
-      ctx->at<__nv_bfloat16>(L.Wb), L.colsb);                // W[y_i] += eta * x_i  (the -onehot part of u_i)
   count_launch();
   CKC(cudaGetLastError());
   return SFB_OK;

@@ -1,5 +1,8 @@
-// Tensor-core (bf16 operand) path of the SFB step: hooks called by the C ABI layer.
+// Tensor-core (bf16 operand) path of the SFB step: hooks called by the C ABI layer, and the host-side helpers
+// the tensor-core translation units share (sfb_tc.cu: factors and forward product; sfb_update.cu: the update).
 #pragma once
+#include <cuda.h>
+
 #include "sfb_internal.h"
 
 namespace sfb {
@@ -14,5 +17,33 @@ int tc_update(sfb_ctx* ctx);
 int tc_after_update(sfb_ctx* ctx);
 int tc_get_factors(sfb_ctx* ctx, const void** U, const void** V, int32_t* dtype, int32_t* layout, int64_t* ldu,
                    int64_t* ldv);
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct TcState {
+  EncodeTiledFn encode;      // cuTensorMapEncodeTiled, obtained through the runtime's driver entry point query
+  int sms;                   // multiprocessors of the device
+  int max_pairs;             // CTA pairs (clusters of 2) of the update kernel that can be resident at once
+};
+
+inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
+
+// 2-D row-major tensor [outer x inner] with row pitch `pitch_bytes`, box [box_outer x box_inner], 128-byte swizzle.
+inline bool make_map(const TcState* st, CUtensorMap* m, CUtensorMapDataType dt, void* base, int64_t inner,
+                     int64_t outer, int64_t pitch_bytes, int box_inner, int box_outer) {
+  if (inner <= 0 || outer <= 0) return false;
+  cuuint64_t dims[2] = {static_cast<cuuint64_t>(inner), static_cast<cuuint64_t>(outer)};
+  cuuint64_t strides[1] = {static_cast<cuuint64_t>(pitch_bytes)};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(box_inner), static_cast<cuuint32_t>(box_outer)};
+  cuuint32_t estr[2] = {1, 1};
+  return st->encode(m, dt, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Fills st->max_pairs (occupancy query of the update kernel); defined beside that kernel.
+int tc_update_init(sfb_ctx* ctx, TcState* st);
 
 }  // namespace sfb
