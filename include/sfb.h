@@ -53,7 +53,8 @@ enum sfb_error {
   SFB_ERR_TIMEOUT = -7,      /* a bounded device-side wait gave up (status word)               */
   SFB_ERR_LABEL_RANGE = -8,  /* a class id outside [0, rows) was skipped (status word)         */
   SFB_ERR_STATE = -9,        /* call order: gather before all workers committed, ...           */
-  SFB_ERR_UNSUPPORTED = -10  /* this model / precision combination is not built                */
+  SFB_ERR_UNSUPPORTED = -10, /* this model / precision combination is not built                */
+  SFB_ERR_STATIC_LIMIT = -11 /* size beyond what the library's built-in scratch array can hold  */
 };
 
 /* Bits of the device status word. */
@@ -151,6 +152,32 @@ const char* sfb_strerror(int code);
 int sfb_last_cuda_error(sfb_ctx* ctx);
 
 int sfb_destroy(sfb_ctx* ctx);
+
+/* Largest column count sfb_prox_columns_noalloc accepts. */
+#define SFB_NOALLOC_MAX_COLS 16384
+
+/* The column prox of sparse coding on its own, for callers that may not allocate:
+ *     every column b of W_dev [rows x cols] (fp32, row-major) with ||b||_2 > 1 becomes b / ||b||_2,
+ * the same two kernels, in the same order, that sfb_apply_update runs for SFB_SC with sc_prox = 1.  (The paper
+ * has no counterpart of this entry point: it exists for the integration cases below, not for the method.)
+ *
+ * Who needs it: code that runs where a device allocation is off the table -- a plug-in living inside another
+ * program's fixed memory budget, a service whose device memory was carved up at start-up and is policed, or a
+ * latency-bound loop that cannot afford the device-wide synchronisation an allocation can bring with it.  Those
+ * callers cannot build an sfb_ctx either (it wants a workspace from them).  This call needs no context and no
+ * workspace: its only scratch, the per-slab column sums (64 x SFB_NOALLOC_MAX_COLS doubles, 8 MB), is an array
+ * built into the library.  Every GPU that loads the library holds those 8 MB until the process ends.
+ *
+ *  - It calls no allocating routine (no cudaMalloc / cudaFree, no library that allocates); the caller passes
+ *    W_dev (updated in place, 16-byte aligned, cols a multiple of 4) and the stream the work is enqueued on.
+ *  - cols > SFB_NOALLOC_MAX_COLS is refused with SFB_ERR_STATIC_LIMIT and nothing is launched.
+ *  - The first call on each device looks up the array's device address (once per device, with that device
+ *    current).  Make that first call outside any stream capture.
+ *  - All calls on one device share the one array.  Nothing in it has to start at zero -- each call overwrites
+ *    every entry it later reads -- but two calls whose kernels overlap on the GPU (different streams, no
+ *    ordering between them) race on it and both results are then undefined.  Order them on one stream or with
+ *    events. */
+int sfb_prox_columns_noalloc(float* W_dev, int64_t rows, int64_t cols, void* stream);
 
 #ifdef __cplusplus
 }

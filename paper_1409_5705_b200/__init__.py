@@ -17,7 +17,8 @@ STATUS_LABEL_RANGE, STATUS_TIMEOUT = 0x1, 0x2
 
 EXPORTS = ("sfb_workspace_bytes", "sfb_init", "sfb_compute_factors", "sfb_gather_factors", "sfb_apply_update",
            "sfb_step", "sfb_step_host", "sfb_dense_sync_step", "sfb_get_factors", "sfb_get_stats",
-           "sfb_get_status", "sfb_strerror", "sfb_last_cuda_error", "sfb_destroy")
+           "sfb_get_status", "sfb_strerror", "sfb_last_cuda_error", "sfb_destroy", "sfb_prox_columns_noalloc")
+NOALLOC_MAX_COLS = 16384
 
 
 class sfb_config(ctypes.Structure):
@@ -72,6 +73,7 @@ def lib() -> ctypes.CDLL:
         L.sfb_strerror.restype = ctypes.c_char_p
         L.sfb_last_cuda_error.argtypes = [vp]
         L.sfb_destroy.argtypes = [vp]
+        L.sfb_prox_columns_noalloc.argtypes = [vp, i64, i64, vp]
         for name in EXPORTS:
             if name != "sfb_strerror":
                 getattr(L, name).restype = ctypes.c_int
@@ -200,6 +202,18 @@ class Context:
             self.close()
         except Exception:
             pass
+
+
+def sfb_prox_columns_noalloc(W, stream=None):
+    """Column prox of sparse coding on a CUDA fp32 tensor ``W`` [rows x cols], in place, through the entry point
+    that allocates nothing (no context, no workspace: the scratch is an array built into the library).  Argument
+    marshalling only; raises SfbError with code -11 when cols exceeds NOALLOC_MAX_COLS."""
+    import torch
+    assert W.is_cuda and W.dtype == torch.float32 and W.is_contiguous() and W.dim() == 2
+    st = stream if stream is not None else torch.cuda.current_stream(W.device)
+    rc = lib().sfb_prox_columns_noalloc(W.data_ptr(), W.shape[0], W.shape[1], st.cuda_stream)
+    if rc:
+        raise SfbError(rc, "sfb_prox_columns_noalloc")
 
 
 def _host_ptr(a):

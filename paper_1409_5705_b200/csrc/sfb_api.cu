@@ -404,6 +404,7 @@ extern "C" const char* sfb_strerror(int code) {
     case SFB_ERR_LABEL_RANGE: return "class id out of range";
     case SFB_ERR_STATE: return "call out of order";
     case SFB_ERR_UNSUPPORTED: return "model/precision combination not built";
+    case SFB_ERR_STATIC_LIMIT: return "size beyond the library's built-in scratch array";
     default: return "unknown error";
   }
 }

@@ -369,3 +369,59 @@ cudaError_t set_lipschitz(cudaStream_t s, Scalars* sc, float L) {
 }
 
 }  // namespace sfb
+
+// ---------------------------------------------------------------------------------------------------------
+// Column prox without any allocation (sfb_prox_columns_noalloc in sfb.h)
+// ---------------------------------------------------------------------------------------------------------
+#include <mutex>
+
+namespace {
+
+constexpr int64_t kNoAllocMaxCols = SFB_NOALLOC_MAX_COLS;
+constexpr int kNoAllocMaxDevices = 64;
+
+// Per-slab column sums of squares of the no-allocation prox: kProxSlabs x kNoAllocMaxCols doubles (8 MB), resident
+// on every device that loads the library until the process exits.  Shared by all calls.
+static __device__ __align__(256) double g_noalloc_colpart[static_cast<size_t>(sfb::kProxSlabs) * kNoAllocMaxCols];
+
+std::mutex g_noalloc_mutex;
+double* g_noalloc_ptr[kNoAllocMaxDevices] = {};   // device address of the array above, per device ordinal
+
+// The array's name is only a handle on the host; the address a kernel can use comes from the runtime, and it
+// differs per device.  Looked up once per device, with that device current.
+cudaError_t noalloc_scratch(double** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kNoAllocMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  if (g_noalloc_ptr[dev] == nullptr) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_noalloc_colpart);
+    if (e != cudaSuccess) return e;
+    g_noalloc_ptr[dev] = static_cast<double*>(p);
+  }
+  *out = g_noalloc_ptr[dev];
+  return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" int sfb_prox_columns_noalloc(float* W_dev, int64_t rows, int64_t cols, void* stream) {
+  if (!W_dev || rows <= 0 || cols <= 0) return SFB_ERR_ARG;
+  if ((reinterpret_cast<uintptr_t>(W_dev) & 15u) != 0) return SFB_ERR_ALIGN;
+  if (cols % 4 != 0 || rows > (1LL << 30)) return SFB_ERR_SHAPE;
+  if (cols > kNoAllocMaxCols) return SFB_ERR_STATIC_LIMIT;
+  double* part = nullptr;
+  if (noalloc_scratch(&part) != cudaSuccess) return SFB_ERR_CUDA;
+  // Every partial that the second kernel reads is written by the first one in this call, so nothing has to start
+  // at zero and what an earlier call left in the array does not matter.
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int64_t sr = sfb::slab_rows_for(rows);
+  dim3 grid(static_cast<unsigned>((cols + 127) / 128), sfb::kProxSlabs);
+  sfb::col_sumsq_kernel<<<grid, sfb::kThreads, 0, s>>>(W_dev, rows, cols, part, sr);
+  sfb::count_launch();
+  sfb::prox_scale_kernel<<<grid, sfb::kThreads, 0, s>>>(W_dev, rows, cols, part, sfb::kProxSlabs, sr);
+  sfb::count_launch();
+  return cudaGetLastError() == cudaSuccess ? SFB_OK : SFB_ERR_CUDA;
+}
