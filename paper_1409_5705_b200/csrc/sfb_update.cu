@@ -192,7 +192,6 @@ update_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
       if (!__all_sync(0xffffffffu, mbar_wait(&tfull[a], aph, abort_flag))) { ok = false; break; }
       tc_fence_after();
       const int y0 = m0 + row_in_tile;
-      const int row = y0 + lane;
       const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + a * UN + h * (UN / 2);
       uint32_t acc0[32], acc1[32];
       tmem_ld_32x32(t_addr, acc0);
@@ -209,7 +208,6 @@ update_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         uint8_t* sl = ring + slot * kSlotBytes;
         if (!__all_sync(0xffffffffu, mbar_wait(&rf[slot], (g / kRing) & 1, abort_flag))) return false;
         const int x0 = n0 + h * (UN / 2) + c * kChunk;
-        uint32_t packed[16];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           float4* wp = reinterpret_cast<float4*>(sl + lane * 128 + ((j ^ (lane & 7)) << 4));
@@ -219,7 +217,6 @@ update_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
           w.z = fmaf(p.alpha, __uint_as_float(acc[4 * j + 2]), w.z);
           w.w = fmaf(p.alpha, __uint_as_float(acc[4 * j + 3]), w.w);
           *wp = w;
-          if (SHADOW) { packed[2 * j] = pack2(w.x, w.y); packed[2 * j + 1] = pack2(w.z, w.w); }
         }
         fence_proxy_async_smem();
         __syncwarp();                                        // every lane has rewritten its row of the slot
@@ -229,13 +226,19 @@ update_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
           if (g >= 1) tma_wait_group_read<1>();              // the store of chunk g-1 has read its slot:
           issue_load();                                      // refill it with chunk g + kRing - 1
         }
-        if (SHADOW && row < p.rows) {
-          __nv_bfloat16* dst = p.shadow + static_cast<int64_t>(row) * p.shadow_ld + x0;
+        if (SHADOW) {
+          // bf16 copy of the chunk, read back from the slot with 8 lanes per row (4 rows per pass): each row's
+          // 32 values leave as one 64-byte piece instead of 32 lanes storing 16 bytes to 32 different rows.
+          const int sub = lane >> 3, jj = lane & 7;
 #pragma unroll
-          for (int j = 0; j < 4; ++j)
-            if (x0 + 8 * j < p.shadow_ld)
-              *reinterpret_cast<uint4*>(dst + 8 * j) =
-                  make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
+          for (int r0 = 0; r0 < 32; r0 += 4) {
+            const int r = r0 + sub;
+            const float4 w = *reinterpret_cast<const float4*>(sl + r * 128 + ((jj ^ (r & 7)) << 4));
+            const int col = x0 + 4 * jj;
+            if (y0 + r < p.rows && col < p.shadow_ld)
+              *reinterpret_cast<uint2*>(p.shadow + static_cast<int64_t>(y0 + r) * p.shadow_ld + col) =
+                  make_uint2(pack2(w.x, w.y), pack2(w.z, w.w));
+          }
         }
         ++g;
         return true;
