@@ -98,20 +98,39 @@ def time_oracle(wl, steps, warmup, budget_s):
 
 
 # ----------------------------------------------------------------------------------------------------------
+def max_over_ranks(values, device, world):
+    """Element-wise maximum over all ranks of a list of floats (the job is as slow as its slowest rank)."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def aggregate_value(world, K, steps, total_ms):
+    """Whole-job samples/s: every rank steps its own replica on K samples per step (no exchange between them)."""
+    return world * K * steps / (total_ms * 1e-3)
+
+
 def clocks_sampler(index):
+    """Starts nvidia-smi sampling SM clock, power and throttle reasons every 20 ms (it needs a moment to start, so
+    it is launched before the warm-up); clocks_summary keeps the samples that fall inside the timed region."""
     f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
-    q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
     try:
-        p = subprocess.Popen(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-lms", "50",
+        p = subprocess.Popen(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-lms", "20",
                               "-i", str(index)], stdout=f, stderr=subprocess.DEVNULL)
     except Exception:
         return None, f
     return p, f
 
 
-def clocks_summary(p, f):
+def clocks_summary(p, f, t0, t1):
+    """Median SM clock and the throttle reasons seen between wall-clock times t0 and t1."""
+    import datetime
     out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
     if p is None:
         return out
@@ -122,18 +141,22 @@ def clocks_summary(p, f):
         p.kill()
     f.flush()
     f.seek(0)
-    sm, mx, reasons = [], [], set()
+    sm, mx, pw, reasons = [], [], [], set()
     names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
     for line in f.read().splitlines():
         parts = [x.strip() for x in line.split(",")]
-        if len(parts) < 7:
+        if len(parts) < 8:
             continue
         try:
-            sm.append(float(parts[0]))
-            mx.append(float(parts[1]))
+            ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+            if ts < t0 or ts > t1:
+                continue
+            sm.append(float(parts[1]))
+            mx.append(float(parts[2]))
+            pw.append(float(parts[3]))
         except ValueError:
             continue
-        for nme, v in zip(names, parts[3:7]):
+        for nme, v in zip(names, parts[4:8]):
             if v.lower().startswith("active"):
                 reasons.add(nme)
     f.close()
@@ -141,6 +164,7 @@ def clocks_summary(p, f):
     if sm:
         out["sm_mhz"] = float(np.median(sm))
         out["sm_max_mhz"] = float(max(mx))
+        out["power_w"] = float(np.median(pw))
         out["samples"] = len(sm)
     out["reasons"] = sorted(reasons)
     return out
@@ -163,6 +187,19 @@ def run_reference(args, wl, rank):
     print(json.dumps(line), flush=True)
 
 
+# DRAM bytes per launch of the update kernel from the ncu capture summarised in profiles/ (a slab of 16384 rows of
+# the paper-scale MLR shape; traffic is proportional to the rows, see that file).  None when the kernel or the
+# workload is not the captured one.
+NCU_UPDATE_TRAFFIC = {"rows": 16384, "cols": 10000, "K": 1024, "bytes": 719213312 + 933900032}
+
+
+def ncu_traffic_per_launch(wl, prec):
+    t = NCU_UPDATE_TRAFFIC
+    if t["bytes"] is None or wl.model != I.MLR or wl.cols != t["cols"] or wl.K != t["K"] or prec != 0:
+        return None
+    return t["bytes"] * wl.rows / t["rows"]
+
+
 def workload_config(wl, dtype):
     return {"workload": wl.name, "model": ["mlr", "dml", "sc"][wl.model], "rows": wl.rows, "cols": wl.cols,
             "workers_P": wl.workers, "batch_B": wl.batch, "K": wl.K, "eta": wl.eta, "operands": dtype,
@@ -173,7 +210,7 @@ def workload_config(wl, dtype):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="sfb", choices=["sfb", "reference"])
     ap.add_argument("--precision", default="bf16", choices=["bf16", "fp32"])
@@ -264,12 +301,13 @@ def main():
             ev[3].record()
 
     # ---- device-resident timing
+    sampler, sfile = clocks_sampler(local) if rank == 0 else (None, None)
     for i in range(args.warmup):
         phased_step(i)
     launches0 = ctx.sfb_get_stats().kernel_launches
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
     barrier()
-    sampler, sfile = clocks_sampler(local) if rank == 0 else (None, None)
+    wall0 = time.time()
     t_start = torch.cuda.Event(enable_timing=True)
     t_end = torch.cuda.Event(enable_timing=True)
     t_start.record()
@@ -277,7 +315,7 @@ def main():
         phased_step(i, evs[i])
     t_end.record()
     barrier()
-    clocks = clocks_summary(sampler, sfile) if rank == 0 else None
+    clocks = clocks_summary(sampler, sfile, wall0, time.time()) if rank == 0 else None
     total_ms = t_start.elapsed_time(t_end)
     launches = ctx.sfb_get_stats().kernel_launches - launches0
     status = ctx.sfb_get_status()
@@ -297,26 +335,27 @@ def main():
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
 
-    tms = torch.tensor([total_ms, e2e_s * 1e3], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms = float(tms[0]), float(tms[1])
+    total_ms, e2e_ms, ms_f, ms_g, ms_u = max_over_ranks([total_ms, e2e_s * 1e3, ms_f, ms_g, ms_u], dev, world)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
     K = wl.K
-    value = world * K * args.steps / (total_ms * 1e-3)
-    e2e_value = world * K * e2e_steps / (e2e_ms * 1e-3)
+    value = aggregate_value(world, K, args.steps, total_ms)
+    e2e_value = aggregate_value(world, K, e2e_steps, e2e_ms)
     h2d = K * wl.in_dim * 4 + (K * wl.cols * 4 if wl.model == I.DML else 0) + (K * 4 if wl.model != I.SC else 0)
 
-    # ---- roofline of the dominant kernel: the fused update  W += -eta U^T V  (one launch per step)
+    # ---- roofline of the dominant kernel: the fused update  W += -eta U^T V  (one launch per step).
+    # Algorithmic bytes per launch: W read and written once in fp32 plus U and V read once (what the method
+    # itself has to move).  The bf16 copy of W that this design writes alongside (the operand of the next forward
+    # product) is real traffic of the kernel and is reported beside it, not counted as algorithmic.
     esz = 2 if prec == S.PREC_BF16 else 4
+    if prec == S.PREC_BF16 and wl.model != I.MLR:
+        esz = 4                                                               # (hi, lo) pairs of bf16
     upd_flops = 2.0 * wl.rows * wl.cols * K
-    upd_bytes = 8.0 * wl.rows * wl.cols + K * (wl.rows + wl.cols) * esz       # W read + written, U and V read once
-    if prec == S.PREC_BF16 and wl.model == I.MLR:
-        upd_bytes += 2.0 * wl.rows * wl.cols                                  # bf16 copy of W for the next forward
+    upd_bytes = 8.0 * wl.rows * wl.cols + K * (wl.rows + wl.cols) * esz
+    shadow_bytes = 2.0 * wl.rows * wl.cols if (prec == S.PREC_BF16 and wl.model == I.MLR) else 0.0
     if prec == S.PREC_BF16:
         t_flop = upd_flops / (peaks["bf16_tflops_sustained"] * 1e12)
         t_mem = upd_bytes / (peaks["hbm_gbs"] * 1e9)
@@ -328,16 +367,19 @@ def main():
                     "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s"}
     else:
         # fp32 FMA pipe: 148 SMs x 128 lanes x 2 flop x max SM clock
-        peak = 148 * 128 * 2 * (clocks.get("sm_max_mhz") or 1965.0) * 1e6 / 1e12
+        peak = 148 * 128 * 2 * ((clocks or {}).get("sm_max_mhz") or 1965.0) * 1e6 / 1e12
         roof = {"bound": "alu", "achieved": upd_flops / (ms_u * 1e-3) / 1e12, "peak": peak, "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["traffic"] = None
-    roof["kernel"] = "fused rank-K update (sfb_apply_update)"
+    roof["traffic"] = ncu_traffic_per_launch(wl, prec)
+    roof["kernel"] = "update_pair_kernel + label_rows_kernel (sfb_apply_update)" if prec == S.PREC_BF16 \
+        else "sgemm_kernel EPI_RMW (sfb_apply_update)"
     roof["ms"] = ms_u
-    roof["peaks"] = peaks["source"]
+    roof["peaks"] = "of " + peaks["source"]
     roof["update_tflops"] = upd_flops / (ms_u * 1e-3) / 1e12
+    roof["tensor_frac_of_sustained"] = roof["update_tflops"] / peaks["bf16_tflops_sustained"]
     roof["algorithmic_bytes"] = upd_bytes
     roof["algorithmic_flops"] = upd_flops
+    roof["achieved_incl_bf16_copy_of_W"] = (upd_bytes + shadow_bytes) / (ms_u * 1e-3) / 1e9
 
     cpu = None
     if not args.no_cpu_baseline:
