@@ -10,9 +10,11 @@
 // 128 x 256 fp32 half of the W tile.
 // Warps of a CTA: 0 = TMA producer, 1 = MMA issuer (leader CTA only) and TMEM owner, 2..9 = epilogue.
 // Epilogue warp (q, h): TMEM lane quarter q (32 rows of W), column half h (128 columns), in four chunks of
-// 32 x 32.  Each warp owns a ring of four 4 KB slots: the W chunk lands there by TMA (three chunks in flight per
-// warp, 96 KB per SM, which is what it takes to keep HBM busy), is combined in place with the accumulator chunk
-// and goes back by TMA from the same slot; the bf16 copy of the new chunk is stored from registers.
+// 32 x 32.  Each warp owns a ring of three 4 KB slots: the W chunk lands there by TMA (two chunks in flight per
+// warp, 64 KB per SM), is combined in place with the accumulator chunk and goes back by TMA from the same slot;
+// the bf16 copy of the new chunk is read back from the slot and stored as 64-byte row pieces.  Shared memory is
+// the scarce resource: 4 operand stages (128 KB) + the rings (96 KB).  Measured: a fourth operand stage gains
+// more (the operand loads slow down when they share L2 with the stream of W) than a fourth ring slot.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -29,13 +31,14 @@ using namespace ptx;
 constexpr int UM = 128;                 // rows of W per CTA (256 per pair)
 constexpr int UN = 256;                 // columns of W per tile
 constexpr int UK = 64, UMMA_K = 16;
-constexpr int kStages = 3;
+constexpr int kStages = 4;
 constexpr int kBytesA = UM * UK * 2;          // 16 KB: this CTA's rows of U^T
 constexpr int kBytesB = (UN / 2) * UK * 2;    // 16 KB: this CTA's half of the V^T rows
 constexpr int kStageBytes = kBytesA + kBytesB;
 constexpr int kChunk = 32;
 constexpr int kSlotBytes = 32 * kChunk * 4;   // 4 KB
-constexpr int kRing = 4;                      // slots per epilogue warp
+constexpr int kRing = 3;                      // slots per epilogue warp
+constexpr int kPend = 1;                      // TMA stores of a warp that may still be reading their slots
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 64 + 32 * kEpiWarps;
 constexpr int kChunksPerWarp = (UN / 2) / kChunk;   // 4
@@ -183,7 +186,7 @@ update_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
       ++lg;
     };
     if (lane == 0)
-      for (int i = 0; i < kRing - 1; ++i) issue_load();
+      for (int i = 0; i < kRing - kPend; ++i) issue_load();
     uint32_t g = 0;
     for (int tl = 0; tl < my_tiles && ok; ++tl) {
       int m0, n0;
@@ -223,8 +226,8 @@ update_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         if (lane == 0) {
           if (x0 < p.cols && y0 < p.rows) tma_store_2d_hint(&tmC, sl, x0, y0, pol_w);
           tma_commit_group();
-          if (g >= 1) tma_wait_group_read<1>();              // the store of chunk g-1 has read its slot:
-          issue_load();                                      // refill it with chunk g + kRing - 1
+          if (g >= kPend) tma_wait_group_read<kPend>();      // the store of chunk g-kPend has read its slot:
+          issue_load();                                      // refill it with chunk g + kRing - kPend
         }
         if (SHADOW) {
           // bf16 copy of the chunk, read back from the slot with 8 lanes per row (4 rows per pass): each row's
