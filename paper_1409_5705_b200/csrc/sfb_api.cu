@@ -29,6 +29,7 @@ Layout make_layout(const sfb_config& c) {
   L.piy = take(c.model == SFB_SC ? rows * 4 : 0);
   L.Kp = static_cast<int64_t>(K);
   L.colsb = static_cast<int64_t>(cols);
+  L.ldu = static_cast<int64_t>(rows);
   if (c.precision == SFB_PREC_FP32) {
     L.V = take(K * cols * 4);
     L.U = take(K * rows * 4);
@@ -156,7 +157,7 @@ static int factors_fp32(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, co
     if (c.model == SFB_MLR)
       CK(mlr_softmax_rows(s, U, n, rows, labels, ctx->at<float>(ctx->lay.loss) + off, status));
     else
-      CK(dml_scale_rows(s, U, n, rows, labels, c.dml_margin));
+      CK(dml_scale_rows(s, U, n, rows, rows, labels, c.dml_margin));
     return SFB_OK;
   }
   // sparse coding: ISTA from a = 0, then u = W a - x, v = a
@@ -209,10 +210,10 @@ extern "C" int sfb_compute_factors(sfb_ctx* ctx, int32_t worker, const float* X_
                             ctx->at<float>(ctx->lay.piy), ctx->at<float>(ctx->lay.colpart),
                             ctx->at<Scalars>(ctx->lay.scalars), 50));
   }
-  // bf16 mode: MLR runs its forward product on the tensor cores; DML and SC need fp32-class factors (their u
-  // comes from a cancelling residual), so only their update product does
-  rc = (c.precision == SFB_PREC_FP32 || c.model != SFB_MLR) ? factors_fp32(ctx, off, n, X_dev, Y_dev, labels_dev)
-                                                            : tc_factors(ctx, off, n, X_dev, Y_dev, labels_dev);
+  // bf16 mode: every product runs on the tensor cores; DML and SC, whose u comes from a cancelling residual,
+  // carry each value as a (hi, lo) pair of bf16 (fp32-class products)
+  rc = c.precision == SFB_PREC_FP32 ? factors_fp32(ctx, off, n, X_dev, Y_dev, labels_dev)
+                                    : tc_factors(ctx, off, n, X_dev, Y_dev, labels_dev);
   if (rc) return rc;
   const uint64_t all = c.workers == 64 ? ~0ull : ((1ull << c.workers) - 1);
   ctx->committed |= worker < 0 ? all : (1ull << worker);

@@ -106,10 +106,10 @@ __global__ void __launch_bounds__(NTHREADS) mlr_softmax_kernel(float* __restrict
 
 // One block per pair: q = ||z||^2; similar: u = 2z; dissimilar: u = -2z if q < margin else 0 (Section 2, DML).
 template <int NTHREADS>
-__global__ void __launch_bounds__(NTHREADS) dml_scale_kernel(float* __restrict__ Z, int64_t rows,
+__global__ void __launch_bounds__(NTHREADS) dml_scale_kernel(float* __restrict__ Z, int64_t rows, int64_t ld,
                                                              const int32_t* __restrict__ similar, float margin) {
   __shared__ float sh[32];
-  float* z = Z + static_cast<int64_t>(blockIdx.x) * rows;
+  float* z = Z + static_cast<int64_t>(blockIdx.x) * ld;
   float q = 0.f;
   for (int64_t j = threadIdx.x; j < rows; j += NTHREADS) q = fmaf(z[j], z[j], q);
   q = block_sum<NTHREADS>(q, sh);
@@ -315,10 +315,10 @@ cudaError_t mlr_softmax_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t ro
   return cudaGetLastError();
 }
 
-cudaError_t dml_scale_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows, const int32_t* similar,
-                           float margin) {
+cudaError_t dml_scale_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows, int64_t ld,
+                           const int32_t* similar, float margin) {
   if (nsamp <= 0) return cudaSuccess;
-  dml_scale_kernel<256><<<static_cast<unsigned>(nsamp), 256, 0, s>>>(Z, rows, similar, margin);
+  dml_scale_kernel<256><<<static_cast<unsigned>(nsamp), 256, 0, s>>>(Z, rows, ld, similar, margin);
   count_launch();
   return cudaGetLastError();
 }

@@ -22,6 +22,10 @@ struct Layout {
   size_t status, scalars, loss, V, U, colpart, pib, piy, stageX, stageY, stageL;
   // bf16 tensor-core mode
   size_t Wb, Xb, VT, ZT, UT, part, Xf, labels;
+  // bf16 mode, DML and SC: (hi | lo) bf16 operands of the split products
+  size_t Ws, WTs, As, Rs;             // W by rows, W transposed, the A operand (v or the codes), the residual
+  int64_t ldu;                        // row pitch of the fp32 U buffer (rows rounded up to 4 in bf16 mode)
+  int64_t colsp, rowsp;               // cols, rows rounded up to 64
   int64_t Kp;                         // K rounded up to the contraction block of the update product
   int64_t colsb;                      // cols rounded up to the contraction block of the forward product
   size_t total;
@@ -84,8 +88,8 @@ cudaError_t pack_copy(cudaStream_t s, float* dst, const float* x, const float* y
 cudaError_t fill_zero(cudaStream_t s, float* dst, int64_t n);
 cudaError_t mlr_softmax_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows, const int32_t* labels,
                              float* loss_per_sample, uint32_t* status);
-cudaError_t dml_scale_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows, const int32_t* similar,
-                           float margin);
+cudaError_t dml_scale_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows, int64_t ld,
+                           const int32_t* similar, float margin);
 cudaError_t mean_of(cudaStream_t s, const float* v, int64_t n, float* out);
 cudaError_t prox_unit_columns(cudaStream_t s, float* W, int64_t rows, int64_t cols, float* colpart);
 cudaError_t estimate_lipschitz(cudaStream_t s, const float* W, int64_t rows, int64_t cols, float* b, float* y,

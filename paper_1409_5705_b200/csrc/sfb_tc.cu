@@ -33,12 +33,32 @@ constexpr int kThreads = 64 + 32 * kEpiWarps;
 constexpr int kBars = 2 * S + 4;
 constexpr int kSmem = S * (kBytesA + kBytesB) + kEpiWarps * R * kSlotBytes + kBars * 8 + 16 + 1024;
 
+// Epilogues of the product  D (samples x N) = A * B^T:
+//   F_SOFTMAX  store D as fp32 logits and the per (sample, 256-column block) softmax partials      (MLR)
+//   F_STORE    store D as fp32                                                                     (DML: z = W v)
+//   F_SUB      store D - aux as fp32 and as a (hi | lo) bf16 pair                                  (SC: r = W a - x)
+//   F_ISTA     C <- soft(C - D / L, lambda / L) in place, also as a (hi | lo) bf16 pair            (SC: ISTA step)
+enum FwdEpi { F_SOFTMAX = 0, F_STORE = 1, F_SUB = 2, F_ISTA = 3 };
+
 struct TcParams {
-  int32_t M, N, Kc;            // extents of the product: samples, rows of W, features
+  int32_t M, N, Kc;            // extents of the product: samples, output columns, contraction
   int32_t m_off;               // first sample handled by this launch (per-worker slices)
   int32_t tilesM, tilesN;
-  float2* part;                // [tilesN][part_ld] (max, sum exp) per sample and 256-row block
+  // The contraction runs over nseg segments of kseg k-blocks; segment s reads A from column a_off<s> and B from
+  // column b_off<s> of their tensors: one segment is the plain product, three segments over [hi | lo] operand
+  // halves form the split-bf16 product hi*hi + hi*lo + lo*hi.  (Scalars: an indexed array would send the whole
+  // parameter block to local memory.)
+  int32_t nseg, kseg;
+  int32_t a_off0, a_off1, a_off2, b_off0, b_off1, b_off2;
+  float2* part;                // F_SOFTMAX: [tilesN][part_ld] (max, sum exp) per sample and 256-row block
   int64_t part_ld;
+  const float* aux;            // F_SUB: the matrix subtracted, [M x ldaux]; F_ISTA: the matrix updated, [M x ldaux]
+  int64_t ldaux;
+  const Scalars* sc;           // F_ISTA: 1 / L
+  float lam;                   // F_ISTA: lambda
+  __nv_bfloat16* split;        // F_SUB, F_ISTA: [M x ld_split] receives hi at column n and lo at column split_half + n
+  int64_t ld_split;
+  int32_t split_half;          // padded N (a multiple of 64); columns N..split_half-1 are written as zeros
   uint32_t* status;
 };
 
@@ -50,6 +70,12 @@ __device__ __forceinline__ void tile_coords(const TcParams& p, int tile, int& m0
   n0 = tn * BN;
 }
 
+__device__ __forceinline__ float soft_threshold(float w, float t) {
+  const float a = fabsf(w) - t;
+  return a > 0.f ? copysignf(a, w) : 0.f;
+}
+
+template <int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
 forward_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmC, const TcParams p) {
@@ -68,7 +94,7 @@ forward_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int ntiles = p.tilesM * p.tilesN;
-  const int numK = (p.Kc + BK - 1) / BK;
+  const int numK = p.nseg * p.kseg;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < S; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
@@ -93,12 +119,16 @@ forward_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
         int m0, n0;
         tile_coords(p, tile, m0, n0);
-        for (int kb = 0; kb < numK; ++kb, ++it) {
-          const uint32_t s = it % S, ph = (it / S) & 1;
-          if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
-          mbar_expect_tx(&full[s], kBytesA + kBytesB);
-          tma_load_2d_hint(sA + s * kBytesA, &tmA, kb * BK, m0, &full[s], pol_keep);
-          tma_load_2d(sB + s * kBytesB, &tmB, kb * BK, n0, &full[s]);
+        for (int seg = 0; seg < p.nseg && ok; ++seg) {
+          const int xa0 = seg == 0 ? p.a_off0 : seg == 1 ? p.a_off1 : p.a_off2;
+          const int xb0 = seg == 0 ? p.b_off0 : seg == 1 ? p.b_off1 : p.b_off2;
+          for (int kl = 0; kl < p.kseg; ++kl, ++it) {
+            const uint32_t s = it % S, ph = (it / S) & 1;
+            if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
+            mbar_expect_tx(&full[s], kBytesA + kBytesB);
+            tma_load_2d_hint(sA + s * kBytesA, &tmA, xa0 + kl * BK, m0, &full[s], pol_keep);
+            tma_load_2d(sB + s * kBytesB, &tmB, xb0 + kl * BK, n0, &full[s]);
+          }
         }
       }
     }
@@ -136,7 +166,7 @@ forward_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     bool ok = true;
 
     {
-      // Forward: store Z through the ring and keep a running (max, sum exp) per sample over the tile's columns.
+      // The fp32 result goes out through the ring by TMA; F_SOFTMAX keeps a running (max, sum exp) per sample.
       uint32_t gs = 0;                       // stores issued so far: consecutive stores alternate ring slots
       for (int tl = 0; tl < my_tiles && ok; ++tl) {
         int m0, n0;
@@ -153,17 +183,64 @@ forward_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           tmem_ld_wait();
           const int col0 = n0 + c * kChunk;
           if (col0 < p.N) {
-            float cm = -INFINITY;
+            if constexpr (EPI == F_SOFTMAX) {
+              float cm = -INFINITY;
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (col0 + j < p.N) cm = fmaxf(cm, __uint_as_float(acc[j]));
-            const float nm = fmaxf(mx, cm);
-            float cs = 0.f;
+              for (int j = 0; j < 32; ++j)
+                if (col0 + j < p.N) cm = fmaxf(cm, __uint_as_float(acc[j]));
+              const float nm = fmaxf(mx, cm);
+              float cs = 0.f;
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (col0 + j < p.N) cs += __expf(__uint_as_float(acc[j]) - nm);
-            sum = sum * __expf(mx - nm) + cs;
-            mx = nm;
+              for (int j = 0; j < 32; ++j)
+                if (col0 + j < p.N) cs += __expf(__uint_as_float(acc[j]) - nm);
+              sum = sum * __expf(mx - nm) + cs;
+              mx = nm;
+            }
+            if constexpr (EPI == F_SUB || EPI == F_ISTA) {
+              // the sample's 32 values of aux (x, or the current code a) are contiguous: 128 bytes per lane
+              float xv[32];
+              const float* ap = p.aux + static_cast<int64_t>(row) * p.ldaux + col0;
+              const bool vec = row < p.M && col0 + 32 <= p.N && ((reinterpret_cast<uintptr_t>(ap) & 15u) == 0);
+              if (vec) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                  const float4 v4 = *reinterpret_cast<const float4*>(ap + 4 * j);
+                  xv[4 * j] = v4.x; xv[4 * j + 1] = v4.y; xv[4 * j + 2] = v4.z; xv[4 * j + 3] = v4.w;
+                }
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) xv[j] = (row < p.M && col0 + j < p.N) ? ap[j] : 0.f;
+              }
+              float invL = 0.f, thr = 0.f;
+              if (EPI == F_ISTA) { invL = p.sc->invL; thr = p.lam * invL; }
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                const float d = __uint_as_float(acc[j]);
+                const float v = EPI == F_SUB ? d - xv[j] : soft_threshold(fmaf(-d, invL, xv[j]), thr);
+                acc[j] = __float_as_uint((row < p.M && col0 + j < p.N) ? v : 0.f);
+              }
+              if (row < p.M) {
+                // (hi | lo) bf16 pair of the result: the operand of the next product
+                __nv_bfloat16* hp = p.split + static_cast<int64_t>(row) * p.ld_split + col0;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  if (col0 + 8 * j < p.split_half) {
+                    uint32_t hi[4], lo[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                      const float f0 = __uint_as_float(acc[8 * j + 2 * e]), f1 = __uint_as_float(acc[8 * j + 2 * e + 1]);
+                      const __nv_bfloat16 h0 = __float2bfloat16_rn(f0), h1 = __float2bfloat16_rn(f1);
+                      hi[e] = static_cast<uint32_t>(__bfloat16_as_ushort(h0)) |
+                              (static_cast<uint32_t>(__bfloat16_as_ushort(h1)) << 16);
+                      const __nv_bfloat162 l2 = __floats2bfloat162_rn(f0 - __bfloat162float(h0), f1 - __bfloat162float(h1));
+                      lo[e] = *reinterpret_cast<const uint32_t*>(&l2);
+                    }
+                    *reinterpret_cast<uint4*>(hp + 8 * j) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                    *reinterpret_cast<uint4*>(hp + p.split_half + 8 * j) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                  }
+                }
+              }
+            }
             if (lane == 0) tma_wait_group_read<R - 1>();   // the store that last used this slot has read it
             __syncwarp();
 #pragma unroll
@@ -182,7 +259,7 @@ forward_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&tempty[a]);
-        if (row < p.M) p.part[static_cast<int64_t>(n0 / BN) * p.part_ld + row] = make_float2(mx, sum);
+        if (EPI == F_SOFTMAX && row < p.M) p.part[static_cast<int64_t>(n0 / BN) * p.part_ld + row] = make_float2(mx, sum);
       }
       if (lane == 0) tma_wait_group<0>();
     }
@@ -270,18 +347,18 @@ __global__ void __launch_bounds__(256) pack_mlr_kernel(const float* __restrict__
 // FT [dim x 2*Kp] (samples contiguous): FT[c][i] = hi(F[i][c]), FT[c][Kp + i] = lo(F[i][c]) with
 // hi = bf16(f), lo = bf16(f - hi); samples n..Kp-1 are written as zeros.  64 x 64 tiles through shared memory.
 __global__ void __launch_bounds__(256) pack_split_t_kernel(const float* __restrict__ F, int64_t n, int64_t dim,
-                                                           __nv_bfloat16* __restrict__ FT, int64_t Kp) {
+                                                           int64_t ld, __nv_bfloat16* __restrict__ FT, int64_t Kp) {
   __shared__ float tile[64][65];
   const int64_t i0 = static_cast<int64_t>(blockIdx.y) * 64, c0 = static_cast<int64_t>(blockIdx.x) * 64;
   const int t = threadIdx.x;
-  const bool vec = (dim % 4) == 0;
+  const bool vec = (ld % 4) == 0;
 #pragma unroll
   for (int v = 0; v < 4; ++v) {
     const int idx = t + v * 256;            // 64 samples x 16 quads
     const int i = idx / 16, cq = (idx % 16) * 4;
     float f[4] = {0.f, 0.f, 0.f, 0.f};
     if (i0 + i < n) {
-      const float* src = F + (i0 + i) * dim + c0 + cq;
+      const float* src = F + (i0 + i) * ld + c0 + cq;
       if (vec && c0 + cq + 3 < dim) {
         const float4 q4 = *reinterpret_cast<const float4*>(src);
         f[0] = q4.x; f[1] = q4.y; f[2] = q4.z; f[3] = q4.w;
@@ -309,6 +386,27 @@ __global__ void __launch_bounds__(256) pack_split_t_kernel(const float* __restri
     __nv_bfloat16* dst = FT + (c0 + c) * 2 * Kp + i0 + ig;     // Kp is a multiple of 64: 16-byte aligned
     *reinterpret_cast<uint4*>(dst) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
     *reinterpret_cast<uint4*>(dst + Kp) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+  }
+}
+
+// fp32 [n x dim] (row pitch ld) -> the (hi | lo) bf16 operand [n x 2*dimp], no transpose: dst[r][c] = hi,
+// dst[r][dimp + c] = lo with hi = bf16(f), lo = bf16(f - hi).  Columns dim..dimp-1 are left as they are (zero since
+// set-up).  dim and ld are multiples of 4.
+__global__ void __launch_bounds__(256) pack_split_rows_kernel(const float* __restrict__ F, int64_t n, int64_t dim,
+                                                              int64_t ld, __nv_bfloat16* __restrict__ dst, int64_t dimp) {
+  const int64_t quads = dim / 4, total = n * quads;
+  const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+  for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total; i += stride) {
+    const int64_t r = i / quads, qd = i % quads;
+    const float4 v = *reinterpret_cast<const float4*>(F + r * ld + qd * 4);
+    const __nv_bfloat16 h0 = __float2bfloat16_rn(v.x), h1 = __float2bfloat16_rn(v.y), h2 = __float2bfloat16_rn(v.z),
+                        h3 = __float2bfloat16_rn(v.w);
+    __nv_bfloat16* d = dst + r * 2 * dimp + qd * 4;
+    *reinterpret_cast<uint2*>(d) =
+        make_uint2(static_cast<uint32_t>(__bfloat16_as_ushort(h0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(h1)) << 16),
+                   static_cast<uint32_t>(__bfloat16_as_ushort(h2)) | (static_cast<uint32_t>(__bfloat16_as_ushort(h3)) << 16));
+    *reinterpret_cast<uint2*>(d + dimp) = make_uint2(pack_bf16(v.x - __bfloat162float(h0), v.y - __bfloat162float(h1)),
+                                                     pack_bf16(v.z - __bfloat162float(h2), v.w - __bfloat162float(h3)));
   }
 }
 
@@ -404,18 +502,19 @@ __global__ void __launch_bounds__(256) mlr_emit_ut_kernel(const float* __restric
 // ---------------------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------------------
+template <int EPI>
 cudaError_t launch_forward(sfb_ctx* ctx, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c, TcParams p) {
   const TcState* st = static_cast<const TcState*>(ctx->tc);
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    cudaError_t e = cudaFuncSetAttribute(forward_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
   const int64_t tiles = static_cast<int64_t>(p.tilesM) * p.tilesN;
   if (tiles <= 0) return cudaSuccess;
   const int grid = static_cast<int>(tiles < st->sms ? tiles : st->sms);
-  forward_kernel<<<grid, kThreads, kSmem, ctx->stream>>>(a, b, c, p);
+  forward_kernel<EPI><<<grid, kThreads, kSmem, ctx->stream>>>(a, b, c, p);
   count_launch();
   return cudaGetLastError();
 }
@@ -437,11 +536,21 @@ void tc_extend_layout(const sfb_config& c, Layout& L, size_t& off) {
   L.Kp = round_up(static_cast<int64_t>(K), 64);
   L.colsb = round_up(c.cols, 64);
   if (c.model != SFB_MLR) {
-    // fp32 factors as the workers write them, and their split-bf16 transposes for the update product
+    // fp32 factors as the workers write them, their split-bf16 transposes for the update product, and the
+    // split-bf16 operands of the forward products
+    L.colsp = round_up(c.cols, 64);
+    L.rowsp = round_up(c.rows, 64);
+    L.ldu = round_up(c.rows, 4);                                        // TMA stores need a 16-byte row pitch
     L.V = take(K * static_cast<size_t>(c.cols) * 4);
-    L.U = take(K * static_cast<size_t>(c.rows) * 4);
+    L.U = take(K * static_cast<size_t>(L.ldu) * 4);
     L.UT = take(static_cast<size_t>(c.rows) * 2 * L.Kp * 2);
     L.VT = take(static_cast<size_t>(c.cols) * 2 * L.Kp * 2);
+    L.Ws = take(static_cast<size_t>(c.rows) * 2 * L.colsp * 2);         // W, rows x (hi | lo)
+    L.As = take(K * 2 * static_cast<size_t>(L.colsp) * 2);              // v (DML) or the codes a (SC)
+    if (c.model == SFB_SC) {
+      L.WTs = take(static_cast<size_t>(c.cols) * 2 * L.rowsp * 2);      // W^T, atoms x (hi | lo)
+      L.Rs = take(K * 2 * static_cast<size_t>(L.rowsp) * 2);            // residual r = W a - x
+    }
     return;
   }
   const size_t ldz = static_cast<size_t>(round_up(c.rows, 32));
@@ -475,7 +584,18 @@ int tc_init(sfb_ctx* ctx) {
     if (rc) return rc;
   }
   const sfb_config& c = ctx->cfg;
-  if (c.model != SFB_MLR) return SFB_OK;        // the forward products of DML and SC run on fp32 operands
+  if (c.model != SFB_MLR) {
+    // pad columns of the split operands are never written by the kernels: clear the buffers once
+    const Layout& L = ctx->lay;
+    const size_t K = static_cast<size_t>(ctx->K);
+    CKC(cudaMemsetAsync(ctx->at<char>(L.Ws), 0, static_cast<size_t>(c.rows) * 2 * L.colsp * 2, ctx->stream));
+    CKC(cudaMemsetAsync(ctx->at<char>(L.As), 0, K * 2 * L.colsp * 2, ctx->stream));
+    if (c.model == SFB_SC) {
+      CKC(cudaMemsetAsync(ctx->at<char>(L.WTs), 0, static_cast<size_t>(c.cols) * 2 * L.rowsp * 2, ctx->stream));
+      CKC(cudaMemsetAsync(ctx->at<char>(L.Rs), 0, K * 2 * L.rowsp * 2, ctx->stream));
+    }
+    return SFB_OK;
+  }
   // bf16 copy of W for the forward product; afterwards the update's epilogue keeps it current
   convert_rows_kernel<<<148 * 8, 256, 0, ctx->stream>>>(ctx->W, c.rows, c.cols, ctx->at<__nv_bfloat16>(ctx->lay.Wb),
                                                         ctx->lay.colsb);
@@ -489,7 +609,98 @@ void tc_destroy(sfb_ctx* ctx) {
   ctx->tc = nullptr;
 }
 
-int tc_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float* /*Y*/, const int32_t* labels) {
+namespace {
+
+inline unsigned grid1d(int64_t items, int per_block) {
+  int64_t g = (items + per_block - 1) / per_block;
+  return static_cast<unsigned>(std::max<int64_t>(1, std::min<int64_t>(g, 148 * 16)));
+}
+
+// One split-bf16 product  D[off..off+n) = A * B^T  with A = [*, 2*Cp] and B = [N x 2*Cp] (hi | lo) operands:
+// hi*hi + hi*lo + lo*hi over a contraction of Cp.
+template <int EPI>
+int split_product(sfb_ctx* ctx, int64_t off, int64_t n, __nv_bfloat16* A, __nv_bfloat16* B, int64_t N, int64_t Cp,
+                  float* C, int64_t ldc, TcParams p) {
+  const TcState* st = static_cast<const TcState*>(ctx->tc);
+  CUtensorMap ma, mb, mc;
+  if (!make_map(st, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, A, 2 * Cp, off + n, 2 * Cp * 2, BK, BM) ||
+      !make_map(st, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, B, 2 * Cp, N, 2 * Cp * 2, BK, BN) ||
+      !make_map(st, &mc, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, C, N, off + n, ldc * 4, kChunk, 32))
+    return SFB_ERR_CUDA;
+  p.M = static_cast<int32_t>(off + n); p.N = static_cast<int32_t>(N); p.Kc = static_cast<int32_t>(Cp);
+  p.m_off = static_cast<int32_t>(off);
+  p.tilesM = static_cast<int32_t>((n + BM - 1) / BM);
+  p.tilesN = static_cast<int32_t>((N + BN - 1) / BN);
+  p.nseg = 3; p.kseg = static_cast<int32_t>(Cp / BK);
+  p.a_off0 = 0; p.a_off1 = 0; p.a_off2 = static_cast<int32_t>(Cp);
+  p.b_off0 = 0; p.b_off1 = static_cast<int32_t>(Cp); p.b_off2 = 0;
+  p.status = ctx->at<uint32_t>(ctx->lay.status);
+  CKC(launch_forward<EPI>(ctx, ma, mb, mc, p));
+  ctx->stats.flops += 3.0 * 2.0 * n * N * Cp;
+  return SFB_OK;
+}
+
+// Sufficient factors of distance metric learning and sparse coding in bf16 mode: the same steps as the fp32
+// path (Section 2: z = W v with v = x - y; Figure 3: ISTA codes, u = W a - x), every product on the tensor cores
+// with (hi | lo) bf16 operands.
+int factors_split(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float* Y, const int32_t* labels) {
+  const sfb_config& c = ctx->cfg;
+  const Layout& L = ctx->lay;
+  const int64_t rows = c.rows, cols = c.cols;
+  cudaStream_t s = ctx->stream;
+  float* V = ctx->at<float>(L.V);
+  float* U = ctx->at<float>(L.U);
+  __nv_bfloat16* Ws = ctx->at<__nv_bfloat16>(L.Ws);
+  __nv_bfloat16* As = ctx->at<__nv_bfloat16>(L.As);
+  if (ctx->committed == 0) {
+    // first factors of the step: refresh the split copies of the W every worker sees (BSP)
+    pack_split_rows_kernel<<<grid1d(rows * cols / 4, 256), 256, 0, s>>>(ctx->W, rows, cols, cols, Ws, L.colsp);
+    count_launch();
+    if (c.model == SFB_SC) {
+      pack_split_t_kernel<<<dim3(static_cast<unsigned>((cols + 63) / 64), static_cast<unsigned>(L.rowsp / 64)), 256, 0, s>>>(
+          ctx->W, rows, cols, cols, ctx->at<__nv_bfloat16>(L.WTs), L.rowsp);
+      count_launch();
+    }
+    CKC(cudaGetLastError());
+  }
+  TcParams p{};
+  if (c.model == SFB_DML) {
+    CKC(pack_copy(s, V + off * cols, X, Y, n * cols));                                   // v = x - y
+    pack_split_rows_kernel<<<grid1d(n * cols / 4, 256), 256, 0, s>>>(V + off * cols, n, cols, cols,
+                                                                     As + off * 2 * L.colsp, L.colsp);
+    count_launch();
+    CKC(cudaGetLastError());
+    int rc = split_product<F_STORE>(ctx, off, n, As, Ws, rows, L.colsp, U, L.ldu, p);   // z_i = W v_i
+    if (rc) return rc;
+    CKC(dml_scale_rows(s, U + off * L.ldu, n, rows, L.ldu, labels, c.dml_margin));
+    return SFB_OK;
+  }
+  // sparse coding: ISTA from a = 0, then u = W a - x, v = a
+  __nv_bfloat16* WTs = ctx->at<__nv_bfloat16>(L.WTs);
+  __nv_bfloat16* Rs = ctx->at<__nv_bfloat16>(L.Rs);
+  CKC(cudaMemsetAsync(V + off * cols, 0, static_cast<size_t>(n) * cols * 4, s));
+  CKC(cudaMemsetAsync(As + off * 2 * L.colsp, 0, static_cast<size_t>(n) * 2 * L.colsp * 2, s));
+  for (int it = 0; it <= c.sc_ista_iters; ++it) {
+    p = TcParams{};
+    p.aux = X - off * rows; p.ldaux = rows;          // X holds this worker's samples: index it by the global row
+    p.split = Rs; p.ld_split = 2 * L.rowsp; p.split_half = static_cast<int32_t>(L.rowsp);
+    int rc = split_product<F_SUB>(ctx, off, n, As, Ws, rows, L.colsp, U, L.ldu, p);     // r = W a - x
+    if (rc) return rc;
+    if (it == c.sc_ista_iters) break;
+    p = TcParams{};
+    p.aux = V; p.ldaux = cols;
+    p.sc = ctx->at<Scalars>(L.scalars); p.lam = c.sc_lambda;
+    p.split = As; p.ld_split = 2 * L.colsp; p.split_half = static_cast<int32_t>(L.colsp);
+    rc = split_product<F_ISTA>(ctx, off, n, Rs, WTs, cols, L.rowsp, V, cols, p);        // a <- soft(a - W^T r / L)
+    if (rc) return rc;
+  }
+  return SFB_OK;
+}
+
+}  // namespace
+
+int tc_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float* Y, const int32_t* labels) {
+  if (ctx->cfg.model != SFB_MLR) return factors_split(ctx, off, n, X, Y, labels);
   const sfb_config& c = ctx->cfg;
   const TcState* st = static_cast<const TcState*>(ctx->tc);
   const Layout& L = ctx->lay;
@@ -523,7 +734,8 @@ int tc_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float
   p.tilesM = static_cast<int32_t>((n + BM - 1) / BM);
   p.tilesN = static_cast<int32_t>((rows + BN - 1) / BN);
   p.part = part; p.part_ld = K; p.status = status;
-  CKC(launch_forward(ctx, ma, mb, mc, p));
+  p.nseg = 1; p.kseg = (p.Kc + BK - 1) / BK;
+  CKC(launch_forward<F_SOFTMAX>(ctx, ma, mb, mc, p));
   ctx->stats.flops += 2.0 * n * rows * cols;
 
   mlr_lse_kernel<<<static_cast<unsigned>((n + 7) / 8), 256, 0, ctx->stream>>>(part, K, p.tilesN, Z, ldz, rows, labels, off,
@@ -544,10 +756,10 @@ int tc_gather(sfb_ctx* ctx) {
   const Layout& L = ctx->lay;
   const unsigned gy = static_cast<unsigned>(L.Kp / 64);
   pack_split_t_kernel<<<dim3(static_cast<unsigned>((c.rows + 63) / 64), gy), 256, 0, ctx->stream>>>(
-      ctx->at<float>(L.U), ctx->K, c.rows, ctx->at<__nv_bfloat16>(L.UT), L.Kp);
+      ctx->at<float>(L.U), ctx->K, c.rows, L.ldu, ctx->at<__nv_bfloat16>(L.UT), L.Kp);
   count_launch();
   pack_split_t_kernel<<<dim3(static_cast<unsigned>((c.cols + 63) / 64), gy), 256, 0, ctx->stream>>>(
-      ctx->at<float>(L.V), ctx->K, c.cols, ctx->at<__nv_bfloat16>(L.VT), L.Kp);
+      ctx->at<float>(L.V), ctx->K, c.cols, c.cols, ctx->at<__nv_bfloat16>(L.VT), L.Kp);
   count_launch();
   CKC(cudaGetLastError());
   return SFB_OK;
@@ -562,7 +774,7 @@ int tc_get_factors(sfb_ctx* ctx, const void** U, const void** V, int32_t* dtype,
     if (V) *V = ctx->at<float>(ctx->lay.V);
     if (dtype) *dtype = 0;
     if (layout) *layout = 0;
-    if (ldu) *ldu = ctx->cfg.rows;
+    if (ldu) *ldu = ctx->lay.ldu;
     if (ldv) *ldv = ctx->cfg.cols;
     return SFB_OK;
   }
