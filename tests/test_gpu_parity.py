@@ -114,18 +114,23 @@ def test_small_ragged_step_matches_oracle(name, prec):
 
 
 @pytest.mark.parametrize("prec", PRECS)
-def test_per_worker_calls_equal_the_fused_step(prec):
+@pytest.mark.parametrize("name", ["mlr", "dml", "sc"])
+def test_per_worker_calls_equal_the_fused_step(name, prec):
     """P calls of sfb_compute_factors (any order) + gather + apply == sfb_step: BSP, same W for all workers."""
-    wl = small("mlr")
+    wl = small(name)
     W0, inp = I.initial_W(wl), I.step_inputs(wl, 1)
-    Wa = gpu_step(wl, W0, inp, prec)[0]
-    Wb = gpu_step(wl, W0, inp, prec, per_worker=True)[0]
-    ref = oracle_step(wl, W0, inp)
-    assert rel_err(Wb, ref, W0) <= TOL[prec]
+    if name == "dml":
+        W0 = (W0 * np.float32(0.06)).astype(np.float32)
+    L = O.lipschitz_power_iteration(W0) if name == "sc" else 0.0
+    Wa = gpu_step(wl, W0, inp, prec, L)[0]
+    Wb = gpu_step(wl, W0, inp, prec, L, per_worker=True)[0]
+    ref = oracle_step(wl, W0, inp, L=L)
+    tol = step_tol(wl, prec, ref, W0)
+    assert rel_err(Wb, ref, W0) <= tol
     if prec == S.PREC_FP32:
         np.testing.assert_array_equal(Wa, Wb)
     else:
-        assert rel_err(Wb, Wa.astype(np.float64), W0) <= TOL[prec]
+        assert rel_err(Wb, Wa.astype(np.float64), W0) <= tol
 
 
 def test_worker_split_invariance_and_determinism():
