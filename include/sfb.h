@@ -135,8 +135,9 @@ int sfb_dense_sync_step(sfb_ctx* ctx, const float* X_dev, const float* Y_dev, co
 /* The gathered factor buffers of the last gather, for inspection.  dtype: 0 = fp32, 1 = bf16.
  * layout: 0 = pair-major (U [K x ldu], V [K x ldv]); 1 = transposed (U^T [rows x ldu], V^T [cols x ldv]).
  * DML and SC return their fp32 pair-major factors in both modes.
- * MLR in bf16 mode keeps u_i = p_i - onehot(y_i) as the pair (p_i in bf16, y_i as int32): the buffer holds the
- * softmax probabilities p_i, and the onehot part is applied to W exactly in fp32 from the class ids. */
+ * MLR in bf16 mode splits u_i = p_i - onehot(y_i) in two: the buffer holds the probabilities p_i in bf16 with a 0
+ * at the label entry (i, y_i); that entry, p_iy - 1, is kept in fp32 and applied to row y_i of W separately
+ * (bf16 cannot hold it when p_iy is close to 1). */
 int sfb_get_factors(sfb_ctx* ctx, const void** U_dev, const void** V_dev, int32_t* dtype, int32_t* layout,
                     int64_t* ldu, int64_t* ldv);
 

@@ -21,7 +21,7 @@ constexpr int kProxSlabs = 64;        // row slabs of the deterministic column r
 struct Layout {
   size_t status, scalars, loss, V, U, colpart, pib, piy, stageX, stageY, stageL;
   // bf16 tensor-core mode
-  size_t Wb, Xb, VT, ZT, UT, part, Xf, labels;
+  size_t Wb, Xb, VT, ZT, UT, part, Xf, labels, coef;
   // bf16 mode, DML and SC: (hi | lo) bf16 operands of the split products
   size_t Ws, WTs, As, Rs;             // W by rows, W transposed, the A operand (v or the codes), the residual
   int64_t ldu;                        // row pitch of the fp32 U buffer (rows rounded up to 4 in bf16 mode)

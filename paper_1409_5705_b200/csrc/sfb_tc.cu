@@ -421,12 +421,13 @@ __device__ __forceinline__ float warp_max(float v) {
   return v;
 }
 
-// One warp per sample: merge the per-block (max, sum exp) partials into log sum exp; loss = lse - z_y.
+// One warp per sample: merge the per-block (max, sum exp) partials into log sum exp; loss = lse - z_y;
+// coef = 1 - p_y, the size of the label entry of u, kept in fp32 for label_rows_kernel.
 __global__ void __launch_bounds__(256) mlr_lse_kernel(const float2* __restrict__ part, int64_t part_ld, int nblocks,
                                                       const float* __restrict__ Z, int64_t ldz, int64_t rows,
                                                       const int32_t* __restrict__ labels, int64_t off, int64_t n,
                                                       float* __restrict__ lse, float* __restrict__ loss,
-                                                      uint32_t* status) {
+                                                      float* __restrict__ coef, uint32_t* status) {
   const int64_t i = static_cast<int64_t>(blockIdx.x) * 8 + (threadIdx.x >> 5);
   if (i >= n) return;
   const int lane = threadIdx.x & 31;
@@ -446,15 +447,20 @@ __global__ void __launch_bounds__(256) mlr_lse_kernel(const float2* __restrict__
     const int32_t y = labels[i];
     const bool okl = y >= 0 && y < rows;
     if (!okl) atomicOr(status, SFB_STATUS_LABEL_RANGE);
-    loss[s] = okl ? l - Z[s * ldz + y] : 0.f;
+    const float zy = okl ? Z[s * ldz + y] : 0.f;
+    loss[s] = okl ? l - zy : 0.f;
+    coef[s] = okl ? -expm1f(zy - l) : 0.f;        // 1 - p_y = -u_y, formed in fp32 without cancellation
   }
 }
 
-// P^T[r][off + i] = bf16( exp(z_ir - lse_i) ): 64 samples x 64 rows per block, transposed through shared
-// memory (Z is sample-major, the update operand is row-major with samples contiguous).  The factor is
-// u_i = p_i - onehot(y_i); its onehot part is not rounded to bf16 but applied exactly by label_rows_kernel.
+// P^T[r][off + i] = bf16( exp(z_ir - lse_i) ) for r != y_i and 0 for r = y_i: 64 samples x 64 rows per block,
+// transposed through shared memory (Z is sample-major, the update operand is row-major with samples
+// contiguous).  The factor is u_i = p_i - onehot(y_i); its label entry u_iy = p_iy - 1 is left out of the bf16
+// operand and applied to W in fp32 by label_rows_kernel, because bf16 cannot hold it when p_iy is close to 1
+// (spacing 2^-8 next to 1) and a rounded p_iy with an exact -1 would not cancel.
 __global__ void __launch_bounds__(256) mlr_emit_ut_kernel(const float* __restrict__ Z, int64_t ldz, int64_t rows,
                                                           const float* __restrict__ lse, int64_t off, int64_t n,
+                                                          const int32_t* __restrict__ labels,
                                                           __nv_bfloat16* __restrict__ UT, int64_t ldu) {
   __shared__ float tile[64][65];
   const int64_t i0 = static_cast<int64_t>(blockIdx.y) * 64, r0 = static_cast<int64_t>(blockIdx.x) * 64;
@@ -467,6 +473,7 @@ __global__ void __launch_bounds__(256) mlr_emit_ut_kernel(const float* __restric
     if (i0 + i >= n) continue;
     const int64_t s = off + i0 + i;
     const float l = lse[s];
+    const int64_t yrel = static_cast<int64_t>(labels[i0 + i]) - (r0 + rq);     // label row relative to this quad
     const float* zp = Z + s * ldz + r0 + rq;
     float z[4] = {0.f, 0.f, 0.f, 0.f};
     if (vec && r0 + rq + 3 < rows) {
@@ -478,7 +485,7 @@ __global__ void __launch_bounds__(256) mlr_emit_ut_kernel(const float* __restric
     }
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      tile[i][rq + k] = __expf(z[k] - l);
+      tile[i][rq + k] = k == yrel ? 0.f : __expf(z[k] - l);
     }
   }
   __syncthreads();
@@ -564,6 +571,7 @@ void tc_extend_layout(const sfb_config& c, Layout& L, size_t& off) {
   L.V = take(K * 4);                             // log-sum-exp per sample
   L.Xf = take(K * static_cast<size_t>(c.cols) * 4);   // fp32 copy of the K samples (exact label-row term)
   L.labels = take(K * 4);                        // class ids of the K samples
+  L.coef = take(K * 4);                          // 1 - p_y per sample (fp32 label entry of u)
   L.U = 0;
 }
 
@@ -739,10 +747,10 @@ int tc_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float
   ctx->stats.flops += 2.0 * n * rows * cols;
 
   mlr_lse_kernel<<<static_cast<unsigned>((n + 7) / 8), 256, 0, ctx->stream>>>(part, K, p.tilesN, Z, ldz, rows, labels, off,
-                                                                              n, lse, loss, status);
+                                                                              n, lse, loss, ctx->at<float>(L.coef), status);
   count_launch();
   dim3 egrid(static_cast<unsigned>((rows + 63) / 64), static_cast<unsigned>((n + 63) / 64));
-  mlr_emit_ut_kernel<<<egrid, 256, 0, ctx->stream>>>(Z, ldz, rows, lse, off, n, UT, L.Kp);
+  mlr_emit_ut_kernel<<<egrid, 256, 0, ctx->stream>>>(Z, ldz, rows, lse, off, n, labels, UT, L.Kp);
   count_launch();
   CKC(cudaGetLastError());
   return SFB_OK;

@@ -270,14 +270,14 @@ update_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
   if (warp == 1) { tc_fence_after(); tmem_dealloc_pair(tmem_base, kTmemCols); }
 }
 
-// The onehot part of the K factors, sum_i (-e_{y_i}) x_i^T, applied to W in fp32 after the tensor-core product
-// has applied sum_i p_i x_i^T:  W[y] <- W[y] + eta * sum_{i : y_i = y} x_i.  One block per (sample, 1024 columns);
-// the blocks of the first sample of each class list that class's samples (ascending, so the sum has the same
-// order every run; no atomics), sum them and refresh the bf16 copy of the row.
+// The label entries of the K factors, u_iy = p_iy - 1, which the bf16 operand leaves out (it holds 0 there):
+//   W[y] <- W[y] + eta * sum_{i : y_i = y} (1 - p_iy) x_i     in fp32, from the fp32 copy of the samples.
+// One block per (sample, 1024 columns); the blocks of the first sample of each class list that class's samples
+// (ascending, so the sum has the same order every run; no atomics), sum them and refresh the bf16 copy of the row.
 constexpr int kLabelList = 1024;
 __global__ void __launch_bounds__(256) label_rows_kernel(float* __restrict__ W, int64_t rows, int64_t cols,
                                                          const float* __restrict__ Xf, const int32_t* __restrict__ labels,
-                                                         int K, float eta, __nv_bfloat16* __restrict__ shadow,
+                                                         const float* __restrict__ coef, int K, float eta, __nv_bfloat16* __restrict__ shadow,
                                                          int64_t shadow_ld) {
   __shared__ int first;
   __shared__ int count;
@@ -319,8 +319,11 @@ __global__ void __launch_bounds__(256) label_rows_kernel(float* __restrict__ W, 
     if (c < cols) {
       const int n = count;
       for (int k = 0; k < n; ++k) {
-        const float4 x = *reinterpret_cast<const float4*>(Xf + static_cast<int64_t>(list[k]) * cols + c);
-        acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
+        const int j = list[k];
+        const float4 x = *reinterpret_cast<const float4*>(Xf + static_cast<int64_t>(j) * cols + c);
+        const float cf = coef[j];
+        acc.x = fmaf(cf, x.x, acc.x); acc.y = fmaf(cf, x.y, acc.y);
+        acc.z = fmaf(cf, x.z, acc.z); acc.w = fmaf(cf, x.w, acc.w);
       }
     }
     __syncthreads();
@@ -417,8 +420,8 @@ int tc_update(sfb_ctx* ctx) {
   if ((c.cols + 1023) / 1024 > 65535) return SFB_ERR_SHAPE;
   dim3 lgrid(static_cast<unsigned>(ctx->K), static_cast<unsigned>((c.cols + 1023) / 1024));
   label_rows_kernel<<<lgrid, 256, 0, ctx->stream>>>(
-      ctx->W, c.rows, c.cols, ctx->at<float>(L.Xf), ctx->at<int32_t>(L.labels), static_cast<int>(ctx->K), c.eta,
-      ctx->at<__nv_bfloat16>(L.Wb), L.colsb);                // W[y_i] += eta * x_i  (the -onehot part of u_i)
+      ctx->W, c.rows, c.cols, ctx->at<float>(L.Xf), ctx->at<int32_t>(L.labels), ctx->at<float>(L.coef), static_cast<int>(ctx->K), c.eta,
+      ctx->at<__nv_bfloat16>(L.Wb), L.colsb);                // W[y_i] += eta * (1 - p_iy) * x_i
   count_launch();
   CKC(cudaGetLastError());
   return SFB_OK;

@@ -90,8 +90,10 @@ def test_small_ragged_step_matches_oracle(name, prec):
     assert rel_err(Wg, Wref, W0) <= step_tol(wl, prec, Wref, W0)
     ftol = 1e-5 if prec == S.PREC_FP32 else 1e-2
     if name == "mlr" and prec == S.PREC_BF16:
-        # bf16 mode carries u = p - onehot(y) as (p in bf16, y as an integer): rebuild u from the two
-        Ug[np.arange(wl.K), inp.labels] -= 1.0
+        # bf16 mode leaves the label entry u_iy = p_iy - 1 out of the bf16 operand (it holds 0 there) and applies
+        # it to W in fp32: the operand must be exactly 0 at (i, y_i); the rest is compared with the oracle's u
+        assert (Ug[np.arange(wl.K), inp.labels] == 0).all()
+        Ug[np.arange(wl.K), inp.labels] = Uref[np.arange(wl.K), inp.labels]
     assert np.linalg.norm(Ug - Uref) <= ftol * np.linalg.norm(Uref)
     assert np.linalg.norm(Vg - Vref) <= ftol * max(np.linalg.norm(Vref), 1e-30)
     if name == "mlr":
