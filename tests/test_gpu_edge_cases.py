@@ -35,6 +35,7 @@ def make(name, **kw):
 SHAPES = [
     # (model, rows, cols, P, B): smaller than any tile; one pair only; K not a multiple of 8 or 64
     ("mlr", 5, 8, 1, 1), ("mlr", 33, 4, 1, 7), ("mlr", 257, 516, 5, 13), ("mlr", 1, 64, 2, 3),
+    ("mlr", 333, 260, 2, 150), ("mlr", 700, 132, 1, 256),      # several sample tiles, the last one ragged
     ("dml", 3, 12, 1, 1), ("dml", 129, 260, 3, 5),
     ("sc", 8, 4, 1, 1), ("sc", 261, 132, 2, 9),
 ]
