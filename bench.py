@@ -201,7 +201,7 @@ def ncu_traffic_per_launch(wl, prec):
 
 
 def workload_config(wl, dtype):
-    return {"workload": wl.name, "model": ["mlr", "dml", "sc"][wl.model], "rows": wl.rows, "cols": wl.cols,
+    return {"workload": wl.name, "family": ["mlr", "dml", "sc"][wl.model], "rows": wl.rows, "cols": wl.cols,
             "workers_P": wl.workers, "batch_B": wl.batch, "K": wl.K, "eta": wl.eta, "operands": dtype,
             "master_W": "f32", "l2": "inputs_larger_than_l2" if wl.rows * wl.cols * 4 > 2 * 126e6
             else "l2_flushed_between_steps"}
