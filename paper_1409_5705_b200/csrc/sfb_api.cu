@@ -263,10 +263,6 @@ extern "C" int sfb_apply_update(sfb_ctx* ctx) {
   ctx->stats.flops += 2.0 * c.rows * c.cols * ctx->K;
   rc = apply_prox(ctx);
   if (rc) return rc;
-  if (c.precision == SFB_PREC_BF16) {
-    rc = tc_after_update(ctx);
-    if (rc) return rc;
-  }
   CK(cudaEventRecord(ctx->ev[3], ctx->stream));
   ctx->committed = 0;
   ctx->gathered = false;

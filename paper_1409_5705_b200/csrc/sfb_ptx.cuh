@@ -1,6 +1,6 @@
 // Thin inline-PTX wrappers for the sm_100a features the tensor-core kernels use: mbarrier, TMA
 // (cp.async.bulk.tensor), tcgen05 (TMEM allocation, MMA issue, commit, TMEM loads) and the proxy fences.
-// Every wait is bounded: it returns false after a fixed number of polls instead of spinning forever.
+// Every wait is bounded: it returns false after a fixed number of SM cycles instead of spinning forever.
 #pragma once
 
 #include <cuda.h>
@@ -12,18 +12,6 @@ namespace ptx {
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-
-__device__ __forceinline__ bool elect_one() {
-  uint32_t pred = 0;
-  asm volatile(
-      "{\n\t"
-      ".reg .pred P;\n\t"
-      "elect.sync _|P, 0xffffffff;\n\t"
-      "selp.u32 %0, 1, 0, P;\n\t"
-      "}\n"
-      : "=r"(pred));
-  return pred != 0;
 }
 
 // ---- mbarrier -------------------------------------------------------------------------------------------
@@ -92,15 +80,10 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, const void* s
                ::"l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(src)), "r"(x), "r"(y)
                : "memory");
 }
-// L2 eviction-priority policies for TMA traffic: operands that every tile re-reads stay, streamed tiles go first.
+// L2 eviction-priority policy for TMA traffic: operands that every tile re-reads stay.
 __device__ __forceinline__ uint64_t policy_evict_last() {
   uint64_t pol;
   asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
-  return pol;
-}
-__device__ __forceinline__ uint64_t policy_evict_first() {
-  uint64_t pol;
-  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
   return pol;
 }
 __device__ __forceinline__ void tma_load_2d_hint(void* dst, const CUtensorMap* m, int32_t x, int32_t y, uint64_t* bar,

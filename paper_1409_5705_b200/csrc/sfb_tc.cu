@@ -773,8 +773,6 @@ int tc_gather(sfb_ctx* ctx) {
   return SFB_OK;
 }
 
-int tc_after_update(sfb_ctx*) { return SFB_OK; }
-
 int tc_get_factors(sfb_ctx* ctx, const void** U, const void** V, int32_t* dtype, int32_t* layout, int64_t* ldu,
                    int64_t* ldv) {
   if (ctx->cfg.model != SFB_MLR) {   // the workers' fp32 factors, pair-major

@@ -14,7 +14,6 @@ void tc_destroy(sfb_ctx* ctx);
 int tc_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float* Y, const int32_t* labels);
 int tc_gather(sfb_ctx* ctx);
 int tc_update(sfb_ctx* ctx);
-int tc_after_update(sfb_ctx* ctx);
 int tc_get_factors(sfb_ctx* ctx, const void** U, const void** V, int32_t* dtype, int32_t* layout, int64_t* ldu,
                    int64_t* ldv);
 
