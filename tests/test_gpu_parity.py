@@ -117,6 +117,32 @@ def test_small_ragged_step_matches_oracle(name, prec):
 
 @pytest.mark.parametrize("prec", PRECS)
 @pytest.mark.parametrize("name", ["mlr", "dml", "sc"])
+def test_three_steps_teacher_forced_on_ragged_shapes(name, prec):
+    """Several steps on one context: whatever the library keeps between steps (the bf16 copy of W and its label
+    rows, the split copies of W rebuilt at the start of a step) must follow W.  Each step is compared with one
+    oracle step from the GPU's own W_t."""
+    wl = small(name)
+    W0 = I.initial_W(wl)
+    if name == "dml":
+        W0 = (W0 * np.float32(0.06)).astype(np.float32)
+    W = to_dev(W0, torch)
+    L0 = O.lipschitz_power_iteration(W0) if name == "sc" else 0.0
+    ctx = S.Context(config_for(wl, prec, L0 * 1.05), W)       # any step 1/L with L >= ||W||^2 is a valid ISTA step
+    true_dict = I.sc_true_dictionary(wl) if name == "sc" else None
+    for t in range(3):
+        inp = I.step_inputs(wl, t, true_dict)
+        Wt = W.cpu().numpy()
+        if name == "dml" and O.dml_hinge_distance(Wt, inp.X, inp.Y, inp.labels) < 4e-3:
+            continue                                           # a pair on the kink: two answers are correct
+        ctx.sfb_step(to_dev(inp.X, torch), to_dev(inp.Y, torch), to_dev(inp.labels, torch))
+        ref = oracle_step(wl, Wt, inp, L=float(np.float32(L0 * 1.05)) if name == "sc" else None)
+        assert rel_err(W.cpu().numpy(), ref, Wt) <= step_tol(wl, prec, ref, Wt), f"step {t}"
+    assert ctx.sfb_get_status() == 0
+    ctx.close()
+
+
+@pytest.mark.parametrize("prec", PRECS)
+@pytest.mark.parametrize("name", ["mlr", "dml", "sc"])
 def test_per_worker_calls_equal_the_fused_step(name, prec):
     """P calls of sfb_compute_factors (any order) + gather + apply == sfb_step: BSP, same W for all workers."""
     wl = small(name)
