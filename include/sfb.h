@@ -103,7 +103,9 @@ int sfb_init(const sfb_config* cfg, float* W_dev, void* workspace_dev, size_t wo
  *   DML: Y_dev = pair partner, labels_dev = 1 similar / 0 dissimilar;
  *        v = x - y, u = 2 W v (similar), -2 W v if ||W v||^2 < margin else 0       (Section 2, DML)
  *   SC : v = a = ISTA code of x, u = W a - x                                        (Figure 3)
- * Factors are written at the worker's row offset p*B of the gathered buffers. */
+ * Factors are written at the worker's row offset p*B of the gathered buffers.  All P workers of a step see the
+ * same W (bulk-synchronous consistency, Section 4.1): copies of W that the library derives (bf16 operands) are
+ * refreshed by the first call of a step. */
 int sfb_compute_factors(sfb_ctx* ctx, int32_t worker, const float* X_dev, const float* Y_dev,
                         const int32_t* labels_dev);
 
@@ -128,7 +130,8 @@ int sfb_step_host(sfb_ctx* ctx, const float* X_host, const float* Y_host, const 
 
 /* Full-matrix-synchronisation comparison path (Section 3 "SFB vs client-server", Section 5): every worker
  * materialises its dense update U_p^T V_p in scratch, the P matrices are summed, and W <- W - eta * sum.
- * scratch_dev: at least 2*rows*cols*4 bytes.  Same result as sfb_step up to summation order. */
+ * scratch_dev: at least 2*rows*cols*4 bytes.  Same result as sfb_step up to summation order.  Built for
+ * SFB_PREC_FP32 contexts only (a comparison path, not a product path); SFB_ERR_UNSUPPORTED otherwise. */
 int sfb_dense_sync_step(sfb_ctx* ctx, const float* X_dev, const float* Y_dev, const int32_t* labels_dev,
                         float* scratch_dev, size_t scratch_bytes);
 
