@@ -382,7 +382,7 @@ def main():
     roof["achieved_incl_bf16_copy_of_W"] = (upd_bytes + shadow_bytes) / (ms_u * 1e-3) / 1e9
 
     cpu = None
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and world == 1:       # the oracle is timed beside the single-GPU run only
         v, dt, sample = time_oracle(wl, 1, 0, 15.0)
         cpu = {"value": v, "unit": UNIT, "cores": cores_used(), "kind": "oracle", "sample": sample,
                "sample_seconds": dt}
