@@ -240,3 +240,23 @@ def test_host_buffer_step_matches_device_step():
     assert status == 0 and abs(loss - O.mlr_loss(W0, inp.X, inp.labels).mean()) < 1e-4
     np.testing.assert_array_equal(W.cpu().numpy(), Wa)
     ctx.close()
+
+
+@pytest.mark.parametrize("prec", PRECS)
+@pytest.mark.parametrize("name", ["dml", "sc"])
+def test_host_buffer_step_for_pairs_and_codes(name, prec):
+    """sfb_step_host stages X (and the pair partner and the flags) itself: same W as the device-resident step."""
+    wl = small(name)
+    W0 = I.initial_W(wl)
+    if name == "dml":
+        W0 = (W0 * np.float32(0.06)).astype(np.float32)
+    inp = I.step_inputs(wl, 5, I.sc_true_dictionary(wl) if name == "sc" else None)
+    L = O.lipschitz_power_iteration(W0) if name == "sc" else 0.0
+    Wa = gpu_step(wl, W0, inp, prec, L)[0]
+    W = to_dev(W0, torch)
+    ctx = S.Context(config_for(wl, prec, L), W)
+    pin = lambda a: None if a is None else torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    loss, status = ctx.sfb_step_host(pin(inp.X), pin(inp.Y), pin(inp.labels))
+    assert status == 0 and loss == 0.0
+    np.testing.assert_array_equal(W.cpu().numpy(), Wa)
+    ctx.close()
