@@ -1,5 +1,5 @@
 """Helpers of the GPU parity tests: run one step through the C ABI, run the oracle on the same inputs,
-and form the spec error ratio  ||W_gpu - W_ref||_F / ||W_ref - W_0||_F."""
+and form the error ratio  ||W_gpu - W_ref||_F / ||W_ref - W_0||_F  (error of the stored W over the size of the update)."""
 from __future__ import annotations
 
 import numpy as np
