@@ -11,6 +11,7 @@
 #include <cuda_bf16.h>
 
 #include <algorithm>
+#include <cstdint>
 #include <new>
 
 #include "sfb_ptx.cuh"
@@ -44,6 +45,7 @@ struct TcParams {
   int32_t M, N, Kc;            // extents of the product: samples, output columns, contraction
   int32_t m_off;               // first sample handled by this launch (per-worker slices)
   int32_t tilesM, tilesN;
+  int32_t bn;                  // columns per tile: a multiple of 32, at most BN (chosen so that the tiles fill the SMs)
   // The contraction runs over nseg segments of kseg k-blocks; segment s reads A from column a_off<s> and B from
   // column b_off<s> of their tensors: one segment is the plain product, three segments over [hi | lo] operand
   // halves form the split-bf16 product hi*hi + hi*lo + lo*hi.  (Scalars: an indexed array would send the whole
@@ -67,7 +69,7 @@ struct TcParams {
 __device__ __forceinline__ void tile_coords(const TcParams& p, int tile, int& m0, int& n0) {
   const int tm = tile % p.tilesM, tn = tile / p.tilesM;
   m0 = p.m_off + tm * BM;
-  n0 = tn * BN;
+  n0 = tn * p.bn;
 }
 
 __device__ __forceinline__ float soft_threshold(float w, float t) {
@@ -125,7 +127,7 @@ forward_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int kl = 0; kl < p.kseg; ++kl, ++it) {
             const uint32_t s = it % S, ph = (it / S) & 1;
             if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
-            mbar_expect_tx(&full[s], kBytesA + kBytesB);
+            mbar_expect_tx(&full[s], kBytesA + p.bn * BK * 2);
             tma_load_2d_hint(sA + s * kBytesA, &tmA, xa0 + kl * BK, m0, &full[s], pol_keep);
             tma_load_2d(sB + s * kBytesB, &tmB, xb0 + kl * BK, n0, &full[s]);
           }
@@ -135,7 +137,7 @@ forward_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
-      const uint32_t idesc = umma_idesc_bf16(BM, BN);
+      const uint32_t idesc = umma_idesc_bf16(BM, p.bn);
       uint32_t it = 0, tl = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++tl) {
@@ -176,7 +178,7 @@ forward_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tc_fence_after();
         const int row = m0 + q * 32 + lane;
         float mx = -INFINITY, sum = 0.f;
-        for (int c = 0; c < BN / kChunk; ++c) {
+        for (int c = 0; c < p.bn / kChunk; ++c) {
           uint8_t* sl = ring + (gs % R) * kSlotBytes;
           uint32_t acc[32];
           tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + a * BN + c * kChunk, acc);
@@ -259,7 +261,7 @@ forward_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&tempty[a]);
-        if (EPI == F_SOFTMAX && row < p.M) p.part[static_cast<int64_t>(n0 / BN) * p.part_ld + row] = make_float2(mx, sum);
+        if (EPI == F_SOFTMAX && row < p.M) p.part[static_cast<int64_t>(n0 / p.bn) * p.part_ld + row] = make_float2(mx, sum);
       }
       if (lane == 0) tma_wait_group<0>();
     }
@@ -624,21 +626,39 @@ inline unsigned grid1d(int64_t items, int per_block) {
   return static_cast<unsigned>(std::max<int64_t>(1, std::min<int64_t>(g, 148 * 16)));
 }
 
+// Tile width (a multiple of 32, at most BN) for a product with tilesM row blocks and N columns on `sms` SMs.  The
+// persistent kernel runs ceil(tiles / sms) rounds of tiles; measured, a tile costs about max(width, 128) + 16
+// column-equivalents (below 128 columns a k-block is bound by the latency of its operand loads, not by the MMA).
+// Narrower tiles fill the SMs of small products, where 256-wide ones leave many idle or need a nearly empty
+// second round; ties go to the wider tile.
+inline int pick_tile_width(int sms, int64_t tilesM, int64_t N) {
+  int best = BN;
+  int64_t best_cost = INT64_MAX;
+  for (int bn = BN; bn >= 128; bn -= 32) {
+    const int64_t tiles = tilesM * ((N + bn - 1) / bn);
+    const int64_t cost = ((tiles + sms - 1) / sms) * (bn + 16);
+    if (cost < best_cost) { best_cost = cost; best = bn; }
+  }
+  return best;
+}
+
 // One split-bf16 product  D[off..off+n) = A * B^T  with A = [*, 2*Cp] and B = [N x 2*Cp] (hi | lo) operands:
 // hi*hi + hi*lo + lo*hi over a contraction of Cp.
 template <int EPI>
 int split_product(sfb_ctx* ctx, int64_t off, int64_t n, __nv_bfloat16* A, __nv_bfloat16* B, int64_t N, int64_t Cp,
                   float* C, int64_t ldc, TcParams p) {
   const TcState* st = static_cast<const TcState*>(ctx->tc);
+  const int bn = pick_tile_width(st->sms, (n + BM - 1) / BM, N);
   CUtensorMap ma, mb, mc;
   if (!make_map(st, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, A, 2 * Cp, off + n, 2 * Cp * 2, BK, BM) ||
-      !make_map(st, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, B, 2 * Cp, N, 2 * Cp * 2, BK, BN) ||
+      !make_map(st, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, B, 2 * Cp, N, 2 * Cp * 2, BK, bn) ||
       !make_map(st, &mc, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, C, N, off + n, ldc * 4, kChunk, 32))
     return SFB_ERR_CUDA;
   p.M = static_cast<int32_t>(off + n); p.N = static_cast<int32_t>(N); p.Kc = static_cast<int32_t>(Cp);
   p.m_off = static_cast<int32_t>(off);
   p.tilesM = static_cast<int32_t>((n + BM - 1) / BM);
-  p.tilesN = static_cast<int32_t>((N + BN - 1) / BN);
+  p.bn = bn;
+  p.tilesN = static_cast<int32_t>((N + bn - 1) / bn);
   p.nseg = 3; p.kseg = static_cast<int32_t>(Cp / BK);
   p.a_off0 = 0; p.a_off1 = 0; p.a_off2 = static_cast<int32_t>(Cp);
   p.b_off0 = 0; p.b_off1 = static_cast<int32_t>(Cp); p.b_off2 = 0;
@@ -740,6 +760,7 @@ int tc_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float
   p.M = static_cast<int32_t>(off + n); p.N = static_cast<int32_t>(rows); p.Kc = static_cast<int32_t>(cols);
   p.m_off = static_cast<int32_t>(off);
   p.tilesM = static_cast<int32_t>((n + BM - 1) / BM);
+  p.bn = BN;
   p.tilesN = static_cast<int32_t>((rows + BN - 1) / BN);
   p.part = part; p.part_ld = K; p.status = status;
   p.nseg = 1; p.kseg = (p.Kc + BK - 1) / BK;
