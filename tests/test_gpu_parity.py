@@ -260,3 +260,31 @@ def test_host_buffer_step_for_pairs_and_codes(name, prec):
     assert status == 0 and loss == 0.0
     np.testing.assert_array_equal(W.cpu().numpy(), Wa)
     ctx.close()
+
+
+def test_two_contexts_on_two_streams_step_concurrently():
+    """One context per stream: two independent problems stepped from two streams at once (their kernels all want
+    the whole tensor memory and most of the shared memory of an SM, so they take turns) both match the oracle."""
+    wl = small("mlr")
+    ctxs = []
+    for k in range(2):
+        W0, inp = I.initial_W(wl), I.step_inputs(wl, 10 + k)
+        W0 = (W0 * np.float32(1.0 + 0.5 * k)).astype(np.float32)
+        stream = torch.cuda.Stream()
+        W = to_dev(W0, torch)
+        X, lab = to_dev(inp.X, torch), to_dev(inp.labels, torch)
+        torch.cuda.synchronize()
+        ctx = S.Context(config_for(wl, S.PREC_BF16), W, stream=stream)
+        ctxs.append((ctx, W, W0, inp, X, lab))
+    for ctx, W, W0, inp, X, lab in ctxs:                 # interleave the launches of the two streams
+        ctx.sfb_compute_factors(-1, X, None, lab)
+    for ctx, *_ in ctxs:
+        ctx.sfb_gather_factors()
+    for ctx, *_ in ctxs:
+        ctx.sfb_apply_update()
+    torch.cuda.synchronize()
+    for ctx, W, W0, inp, X, lab in ctxs:
+        assert ctx.sfb_get_status() == 0
+        ref = oracle_step(wl, W0, inp)
+        assert rel_err(W.cpu().numpy(), ref, W0) <= TOL[S.PREC_BF16]
+        ctx.close()
