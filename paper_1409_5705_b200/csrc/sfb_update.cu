@@ -64,10 +64,17 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// Tiles are numbered with the column block fastest: the pairs that run at the same time share a block of U^T
-// (512 KB), and V^T (all of it, marked evict_last) stays in L2.
+// Tile order: row blocks are taken in groups of kGroup; within a group the tiles are numbered row block fastest,
+// then column block.  The pairs that run at the same time therefore work on kGroup blocks of U^T (512 KB each) and
+// on about 74 / kGroup blocks of V^T: every operand line has a handful of readers at a time instead of one block of
+// U^T having forty (measured: groups of 8 are 4-5 % faster than column-block-fastest order, groups of 37 or more
+// slower again).  All of V^T (marked evict_last) and the group's blocks of U^T stay in L2.
+constexpr int kGroup = 8;
 __device__ __forceinline__ void tile_origin(const UpdParams& p, int tile, int& m0, int& n0) {
-  const int tn = tile % p.tilesN, tm = tile / p.tilesN;
+  const int per_group = kGroup * p.tilesN;
+  const int grp = tile / per_group, within = tile - grp * per_group;
+  const int gsz = min(kGroup, p.tilesM - grp * kGroup);       // the last group may be smaller
+  const int tm = grp * kGroup + within % gsz, tn = within / gsz;
   m0 = tm * (2 * UM);
   n0 = tn * UN;
 }
