@@ -190,7 +190,7 @@ def run_reference(args, wl, rank):
 # DRAM bytes per launch of the update kernel from the ncu capture summarised in profiles/ (a slab of 16384 rows of
 # the paper-scale MLR shape; traffic is proportional to the rows, see that file).  None when the kernel or the
 # workload is not the captured one.
-NCU_UPDATE_TRAFFIC = {"rows": 16384, "cols": 10000, "K": 1024, "bytes": 712201216 + 932222464}
+NCU_UPDATE_TRAFFIC = {"rows": 16384, "cols": 10000, "K": 1024, "bytes": 764645888 + 933098496}
 
 
 def ncu_traffic_per_launch(wl, prec):
