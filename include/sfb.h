@@ -157,6 +157,15 @@ int sfb_last_cuda_error(sfb_ctx* ctx);
 
 int sfb_destroy(sfb_ctx* ctx);
 
+/* Self-test of the failure-detection path (no counterpart in the paper).  Every wait inside the tensor-core kernels
+ * is bounded: after a cycle limit it gives up, the kernel sets SFB_STATUS_TIMEOUT in the status word, releases what
+ * it holds and returns, so a pipeline fault surfaces as a status bit and the context stays usable.  This call
+ * enqueues, on the context's stream, a one-block kernel that runs that same wait on a barrier nothing ever arrives
+ * at, with a limit of max_cycles SM clock cycles (1 .. 2e9; about 1e6 = well under a millisecond).  It holds no copy
+ * in flight and no tensor memory.  Afterwards sfb_get_status reports SFB_STATUS_TIMEOUT (and clears it); later steps
+ * on the context are unaffected.  The limits of the product kernels are not changed by this call. */
+int sfb_selftest_wait_timeout(sfb_ctx* ctx, int64_t max_cycles);
+
 /* Largest column count sfb_prox_columns_noalloc accepts. */
 #define SFB_NOALLOC_MAX_COLS 16384
 
@@ -176,7 +185,11 @@ int sfb_destroy(sfb_ctx* ctx);
  *    W_dev (updated in place, 16-byte aligned, cols a multiple of 4) and the stream the work is enqueued on.
  *  - cols > SFB_NOALLOC_MAX_COLS is refused with SFB_ERR_STATIC_LIMIT and nothing is launched.
  *  - The first call on each device looks up the array's device address (once per device, with that device
- *    current).  Make that first call outside any stream capture.
+ *    current).  The CUDA runtime may load this library's device code on that device at that moment, the 8 MB array
+ *    included: a one-off, driver-side set-up cost that is not a cudaMalloc but can synchronise the device.  Make
+ *    that first call at start-up, outside any stream capture and outside latency-critical sections.
+ *  - W_dev must be device memory of the CURRENT device (the array address is per device); anything else is refused
+ *    with SFB_ERR_ARG.
  *  - All calls on one device share the one array.  Nothing in it has to start at zero -- each call overwrites
  *    every entry it later reads -- but two calls whose kernels overlap on the GPU (different streams, no
  *    ordering between them) race on it and both results are then undefined.  Order them on one stream or with

@@ -17,7 +17,8 @@ STATUS_LABEL_RANGE, STATUS_TIMEOUT = 0x1, 0x2
 
 EXPORTS = ("sfb_workspace_bytes", "sfb_init", "sfb_compute_factors", "sfb_gather_factors", "sfb_apply_update",
            "sfb_step", "sfb_step_host", "sfb_dense_sync_step", "sfb_get_factors", "sfb_get_stats",
-           "sfb_get_status", "sfb_strerror", "sfb_last_cuda_error", "sfb_destroy", "sfb_prox_columns_noalloc")
+           "sfb_get_status", "sfb_strerror", "sfb_last_cuda_error", "sfb_destroy", "sfb_prox_columns_noalloc",
+           "sfb_selftest_wait_timeout")
 NOALLOC_MAX_COLS = 16384
 
 
@@ -74,6 +75,7 @@ def lib() -> ctypes.CDLL:
         L.sfb_last_cuda_error.argtypes = [vp]
         L.sfb_destroy.argtypes = [vp]
         L.sfb_prox_columns_noalloc.argtypes = [vp, i64, i64, vp]
+        L.sfb_selftest_wait_timeout.argtypes = [vp, i64]
         for name in EXPORTS:
             if name != "sfb_strerror":
                 getattr(L, name).restype = ctypes.c_int
@@ -192,6 +194,9 @@ class Context:
         self._ck(lib().sfb_get_status(self._h, ctypes.byref(st)), "sfb_get_status")
         return st.value
 
+    def sfb_selftest_wait_timeout(self, max_cycles):
+        self._ck(lib().sfb_selftest_wait_timeout(self._h, max_cycles), "sfb_selftest_wait_timeout")
+
     def close(self):
         if self._h:
             lib().sfb_destroy(self._h)
@@ -211,7 +216,8 @@ def sfb_prox_columns_noalloc(W, stream=None):
     import torch
     assert W.is_cuda and W.dtype == torch.float32 and W.is_contiguous() and W.dim() == 2
     st = stream if stream is not None else torch.cuda.current_stream(W.device)
-    rc = lib().sfb_prox_columns_noalloc(W.data_ptr(), W.shape[0], W.shape[1], st.cuda_stream)
+    with torch.cuda.device(W.device):          # the built-in scratch array is per device: W's device must be current
+        rc = lib().sfb_prox_columns_noalloc(W.data_ptr(), W.shape[0], W.shape[1], st.cuda_stream)
     if rc:
         raise SfbError(rc, "sfb_prox_columns_noalloc")
 

@@ -7,7 +7,20 @@
 
 namespace sfb {
 
-int64_t g_kernel_launches = 0;
+std::atomic<int64_t> g_kernel_launches{0};
+
+int sm_count() {
+  constexpr int kMaxDevices = 64;
+  static std::atomic<int> cache[kMaxDevices];          // zero-initialised: 0 = not looked up yet
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 148;
+  int n = cache[dev].load(std::memory_order_relaxed);
+  if (n == 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cache[dev].store(n, std::memory_order_relaxed);
+  }
+  return n;
+}
 
 static size_t up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
@@ -373,7 +386,7 @@ extern "C" int sfb_get_stats(sfb_ctx* ctx, sfb_stats* out) {
     ctx->stats.last_loss = h.loss_mean;
     ctx->stats.sc_lipschitz = h.L;
   }
-  ctx->stats.kernel_launches = g_kernel_launches;
+  ctx->stats.kernel_launches = g_kernel_launches.load(std::memory_order_relaxed);
   *out = ctx->stats;
   return SFB_OK;
 }

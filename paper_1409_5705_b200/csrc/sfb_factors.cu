@@ -278,7 +278,7 @@ __global__ void set_L_kernel(Scalars* sc, float L) { sc->L = L; sc->invL = 1.f /
 inline unsigned grid_for(int64_t n, int per_block) {
   int64_t g = (n + per_block - 1) / per_block;
   if (g < 1) g = 1;
-  const int64_t cap = 148 * 16;
+  const int64_t cap = static_cast<int64_t>(sm_count()) * 16;
   return static_cast<unsigned>(g > cap ? cap : g);
 }
 
@@ -412,6 +412,14 @@ extern "C" int sfb_prox_columns_noalloc(float* W_dev, int64_t rows, int64_t cols
   if ((reinterpret_cast<uintptr_t>(W_dev) & 15u) != 0) return SFB_ERR_ALIGN;
   if (cols % 4 != 0 || rows > (1LL << 30)) return SFB_ERR_SHAPE;
   if (cols > kNoAllocMaxCols) return SFB_ERR_STATIC_LIMIT;
+  // The scratch array looked up below belongs to the current device: W must live there too.
+  {
+    int dev = -1;
+    cudaPointerAttributes attr{};
+    if (cudaGetDevice(&dev) != cudaSuccess) return SFB_ERR_CUDA;
+    if (cudaPointerGetAttributes(&attr, W_dev) != cudaSuccess) { cudaGetLastError(); return SFB_ERR_ARG; }
+    if (attr.type != cudaMemoryTypeDevice || attr.device != dev) return SFB_ERR_ARG;
+  }
   double* part = nullptr;
   if (noalloc_scratch(&part) != cudaSuccess) return SFB_ERR_CUDA;
   // Every partial that the second kernel reads is written by the first one in this call, so nothing has to start

@@ -3,14 +3,19 @@
 
 #include <cuda_runtime.h>
 #include <stddef.h>
+
+#include <atomic>
 #include <stdint.h>
 
 #include "sfb.h"
 
 namespace sfb {
 
-extern int64_t g_kernel_launches;     // kernels launched by this library in this process
-inline void count_launch(int n = 1) { g_kernel_launches += n; }
+extern std::atomic<int64_t> g_kernel_launches;     // kernels launched by this library in this process
+inline void count_launch(int n = 1) { g_kernel_launches.fetch_add(n, std::memory_order_relaxed); }
+
+// Multiprocessors of the current device (looked up once per device ordinal).
+int sm_count();
 
 // ---------------------------------------------------------------------------------------------------------
 // Workspace carve-up.  Every offset is a multiple of 1024 bytes so that any sub-buffer can be a TMA base.

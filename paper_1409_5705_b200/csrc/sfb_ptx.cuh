@@ -44,14 +44,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // role of the CTA.  The clock is the SM's own cycle counter, which costs a few cycles to read.
 constexpr uint32_t kMaxPolls = 1u << 26;
 constexpr long long kMaxWaitCycles = 4000000000ll;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort,
+                                          long long max_cycles = kMaxWaitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t i = 0; i < kMaxPolls; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 255u) == 255u) {
       if (*abort) return false;
-      if (clock64() - t0 > kMaxWaitCycles) break;
+      if (clock64() - t0 > max_cycles) break;
     }
   }
   *abort = 1;

@@ -514,18 +514,22 @@ __global__ void __launch_bounds__(256) mlr_emit_ut_kernel(const float* __restric
 template <int EPI>
 cudaError_t launch_forward(sfb_ctx* ctx, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c, TcParams p) {
   const TcState* st = static_cast<const TcState*>(ctx->tc);
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(forward_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
   const int64_t tiles = static_cast<int64_t>(p.tilesM) * p.tilesN;
   if (tiles <= 0) return cudaSuccess;
   const int grid = static_cast<int>(tiles < st->sms ? tiles : st->sms);
   forward_kernel<EPI><<<grid, kThreads, kSmem, ctx->stream>>>(a, b, c, p);
   count_launch();
   return cudaGetLastError();
+}
+
+// The shared-memory opt-in is a per-device attribute of each kernel: set for every instantiation when a context is
+// created (with its device current), not once per process.
+cudaError_t prepare_forward_kernels() {
+  cudaError_t e = cudaFuncSetAttribute(forward_kernel<F_SOFTMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(forward_kernel<F_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(forward_kernel<F_SUB>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(forward_kernel<F_ISTA>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+  return e;
 }
 
 }  // namespace
@@ -589,6 +593,7 @@ int tc_init(sfb_ctx* ctx) {
   int dev = 0;
   CKC(cudaGetDevice(&dev));
   CKC(cudaDeviceGetAttribute(&st->sms, cudaDevAttrMultiProcessorCount, dev));
+  CKC(prepare_forward_kernels());
   {
     const int rc = tc_update_init(ctx, st);
     if (rc) return rc;
@@ -607,7 +612,7 @@ int tc_init(sfb_ctx* ctx) {
     return SFB_OK;
   }
   // bf16 copy of W for the forward product; afterwards the update's epilogue keeps it current
-  convert_rows_kernel<<<148 * 8, 256, 0, ctx->stream>>>(ctx->W, c.rows, c.cols, ctx->at<__nv_bfloat16>(ctx->lay.Wb),
+  convert_rows_kernel<<<st->sms * 8, 256, 0, ctx->stream>>>(ctx->W, c.rows, c.cols, ctx->at<__nv_bfloat16>(ctx->lay.Wb),
                                                         ctx->lay.colsb);
   count_launch();
   CKC(cudaGetLastError());
@@ -623,7 +628,7 @@ namespace {
 
 inline unsigned grid1d(int64_t items, int per_block) {
   int64_t g = (items + per_block - 1) / per_block;
-  return static_cast<unsigned>(std::max<int64_t>(1, std::min<int64_t>(g, 148 * 16)));
+  return static_cast<unsigned>(std::max<int64_t>(1, std::min<int64_t>(g, static_cast<int64_t>(sm_count()) * 16)));
 }
 
 // Tile width (a multiple of 32, at most BN) for a product with tilesM row blocks and N columns on `sms` SMs.  The
