@@ -36,9 +36,10 @@ enum sfb_model { SFB_MLR = 0, SFB_DML = 1, SFB_SC = 2 };
 
 /* Operand precision of the matrix products.  The master copy of W is fp32 in both modes.
  * SFB_PREC_BF16: tensor-core products on bf16 operands with fp32 accumulation.  MLR: forward and update
- *                products on single bf16 operands.  DML, SC: the factors are computed on fp32 operands (u is a
- *                residual that cancels); the update product runs on the tensor cores with every factor value
- *                carried as a (hi, lo) pair of bf16, three bf16 products per term.
+ *                products on single bf16 operands (the label entry of u is kept in fp32).  DML, SC: u is a residual
+ *                that cancels, so every product -- the forward W v, the products of the ISTA coder and the update --
+ *                runs on the tensor cores with each value carried as a (hi, lo) pair of bf16, three bf16 products
+ *                per term (about 2^-16 relative error per product).
  * SFB_PREC_FP32: fp32 operands, fp32 FMA accumulation. */
 enum sfb_precision { SFB_PREC_BF16 = 0, SFB_PREC_FP32 = 1 };
 
@@ -127,6 +128,32 @@ int sfb_step(sfb_ctx* ctx, const float* X_dev, const float* Y_dev, const int32_t
  * waits for the stream.  loss_out and status_out may be NULL. */
 int sfb_step_host(sfb_ctx* ctx, const float* X_host, const float* Y_host, const int32_t* labels_host,
                   float* loss_out, uint32_t* status_out);
+
+/* ---- The parameter matrix partitioned by rows over several contexts (multiclass logistic regression) -------------
+ * Section 3 assumes every worker holds a full copy of W and notes (footnote to the set-up of SFB) that a W too large
+ * for that can be partitioned across machines.  On GPUs the partition also removes the redundant work of the replicas:
+ * each context (one per GPU) owns rows [row_offset, row_offset + rows) of a matrix with global_rows classes, computes
+ * the logits of ALL K samples against its own rows, and updates only those rows.  The softmax couples the shards
+ * through one small exchange per step, which the caller performs (an all-gather of K*16 bytes per shard):
+ *
+ *   sfb_set_row_shard       once after sfb_init (rows of the config = this shard's row count; class ids stay global)
+ *   sfb_forward_partials    logits of the K samples against this shard's rows and, per sample i, the shard's softmax
+ *                           partial  partials_dev[i] = { m_i, s_i, zy_i, has_i }  (4 floats):  m_i = max_j z_ij and
+ *                           s_i = sum_j exp(z_ij - m_i) over the shard's rows j;  zy_i = z_{i,y_i} and has_i = 1 if
+ *                           the shard owns class y_i, else 0 and 0.   X_dev [K x cols], labels_dev [K] (global ids).
+ *   (caller)                gathers the partials of all shards into partials_all_dev [shards][K][4], shard order
+ *   sfb_finish_factors      log-partition lse_i = M + log sum_g s_gi exp(m_gi - M), M = max_g m_gi;  this shard's part
+ *                           of the factor, u_ij = exp(z_ij - lse_i) - [j = y_i] (Section 2.1), v_i = x_i;  the loss
+ *                           lse_i - z_{i,y_i}, identical on every shard.  A class id no shard owns sets
+ *                           SFB_STATUS_LABEL_RANGE.  Afterwards every worker counts as committed:
+ *   sfb_gather_factors, sfb_apply_update   as for an unsharded context, on this shard's rows.
+ *
+ * With one shard (row_offset 0, global_rows = rows) the three calls compute what sfb_compute_factors(-1) computes.
+ * Errors: SFB_ERR_UNSUPPORTED for other models, SFB_ERR_STATE for calls out of order, SFB_ERR_SHAPE for a row range
+ * outside [0, global_rows). */
+int sfb_set_row_shard(sfb_ctx* ctx, int64_t row_offset, int64_t global_rows);
+int sfb_forward_partials(sfb_ctx* ctx, const float* X_dev, const int32_t* labels_dev, float* partials_dev);
+int sfb_finish_factors(sfb_ctx* ctx, const float* partials_all_dev, int32_t shards);
 
 /* Full-matrix-synchronisation comparison path (Section 3 "SFB vs client-server", Section 5): every worker
  * materialises its dense update U_p^T V_p in scratch, the P matrices are summed, and W <- W - eta * sum.

@@ -18,7 +18,7 @@ STATUS_LABEL_RANGE, STATUS_TIMEOUT = 0x1, 0x2
 EXPORTS = ("sfb_workspace_bytes", "sfb_init", "sfb_compute_factors", "sfb_gather_factors", "sfb_apply_update",
            "sfb_step", "sfb_step_host", "sfb_dense_sync_step", "sfb_get_factors", "sfb_get_stats",
            "sfb_get_status", "sfb_strerror", "sfb_last_cuda_error", "sfb_destroy", "sfb_prox_columns_noalloc",
-           "sfb_selftest_wait_timeout")
+           "sfb_selftest_wait_timeout", "sfb_set_row_shard", "sfb_forward_partials", "sfb_finish_factors")
 NOALLOC_MAX_COLS = 16384
 
 
@@ -76,6 +76,9 @@ def lib() -> ctypes.CDLL:
         L.sfb_destroy.argtypes = [vp]
         L.sfb_prox_columns_noalloc.argtypes = [vp, i64, i64, vp]
         L.sfb_selftest_wait_timeout.argtypes = [vp, i64]
+        L.sfb_set_row_shard.argtypes = [vp, i64, i64]
+        L.sfb_forward_partials.argtypes = [vp, vp, vp, vp]
+        L.sfb_finish_factors.argtypes = [vp, vp, i32]
         for name in EXPORTS:
             if name != "sfb_strerror":
                 getattr(L, name).restype = ctypes.c_int
@@ -193,6 +196,17 @@ class Context:
         st = ctypes.c_uint32(0)
         self._ck(lib().sfb_get_status(self._h, ctypes.byref(st)), "sfb_get_status")
         return st.value
+
+    def sfb_set_row_shard(self, row_offset, global_rows):
+        self._ck(lib().sfb_set_row_shard(self._h, row_offset, global_rows), "sfb_set_row_shard")
+
+    def sfb_forward_partials(self, X, labels, partials):
+        """partials: fp32 CUDA tensor [K, 4] that receives this shard's (max, sum exp, label logit, owner flag)."""
+        self._ck(lib().sfb_forward_partials(self._h, _ptr(X), _ptr(labels), _ptr(partials)), "sfb_forward_partials")
+
+    def sfb_finish_factors(self, partials_all, shards):
+        """partials_all: fp32 CUDA tensor [shards, K, 4], the partials of every shard in shard order."""
+        self._ck(lib().sfb_finish_factors(self._h, _ptr(partials_all), shards), "sfb_finish_factors")
 
     def sfb_selftest_wait_timeout(self, max_cycles):
         self._ck(lib().sfb_selftest_wait_timeout(self._h, max_cycles), "sfb_selftest_wait_timeout")

@@ -117,6 +117,9 @@ extern "C" int sfb_init(const sfb_config* cfg, float* W_dev, void* workspace_dev
   ctx->in_dim = cfg->model == SFB_SC ? cfg->rows : cfg->cols;
   ctx->committed = 0;
   ctx->gathered = false;
+  ctx->row_offset = 0;
+  ctx->global_rows = cfg->rows;
+  ctx->partials_ready = false;
   ctx->last_cuda = 0;
   ctx->stats = sfb_stats{};
   ctx->tc = nullptr;
@@ -230,6 +233,72 @@ extern "C" int sfb_compute_factors(sfb_ctx* ctx, int32_t worker, const float* X_
   if (rc) return rc;
   const uint64_t all = c.workers == 64 ? ~0ull : ((1ull << c.workers) - 1);
   ctx->committed |= worker < 0 ? all : (1ull << worker);
+  ctx->gathered = false;
+  return SFB_OK;
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Row-sharded MLR: the parameter matrix partitioned by rows over several contexts (one per GPU)
+// ---------------------------------------------------------------------------------------------------------
+extern "C" int sfb_set_row_shard(sfb_ctx* ctx, int64_t row_offset, int64_t global_rows) {
+  if (!ctx) return SFB_ERR_ARG;
+  if (ctx->cfg.model != SFB_MLR) return SFB_ERR_UNSUPPORTED;
+  if (row_offset < 0 || global_rows < row_offset + ctx->cfg.rows || global_rows > (1LL << 31) - 1) return SFB_ERR_SHAPE;
+  if (ctx->committed != 0 || ctx->partials_ready) return SFB_ERR_STATE;
+  ctx->row_offset = row_offset;
+  ctx->global_rows = global_rows;
+  return SFB_OK;
+}
+
+extern "C" int sfb_forward_partials(sfb_ctx* ctx, const float* X_dev, const int32_t* labels_dev, float* partials_dev) {
+  int rc = check_inputs(ctx, X_dev, nullptr, labels_dev);
+  if (rc) return rc;
+  if (ctx->cfg.model != SFB_MLR) return SFB_ERR_UNSUPPORTED;
+  if (!partials_dev) return SFB_ERR_ARG;
+  if (!al16(partials_dev)) return SFB_ERR_ALIGN;
+  const sfb_config& c = ctx->cfg;
+  ctx->committed = 0;
+  ctx->gathered = false;
+  CK(cudaEventRecord(ctx->ev[0], ctx->stream));
+  if (c.precision == SFB_PREC_BF16) {
+    rc = tc_forward_partials(ctx, X_dev, labels_dev, partials_dev);
+    if (rc) return rc;
+  } else {
+    const int64_t K = ctx->K;
+    float* V = ctx->at<float>(ctx->lay.V);
+    float* U = ctx->at<float>(ctx->lay.U);
+    CK(pack_copy(ctx->stream, V, X_dev, nullptr, K * c.cols));                                    // v = x
+    EpiArgs e{};
+    e.C = U; e.ldc = c.rows;
+    CK(sgemm(ctx->stream, true, true, EPI_STORE, K, c.rows, c.cols, V, c.cols, ctx->W, c.cols, e));   // z_i = W_shard x_i
+    ctx->stats.flops += 2.0 * K * c.rows * c.cols;
+    // the class ids are kept for the finish (the caller's buffer may change before it)
+    CK(cudaMemcpyAsync(ctx->at<int32_t>(ctx->lay.stageL), labels_dev, static_cast<size_t>(K) * 4, cudaMemcpyDeviceToDevice,
+                       ctx->stream));
+    CK(mlr_shard_partials(ctx->stream, U, K, c.rows, c.rows, ctx->at<int32_t>(ctx->lay.stageL), ctx->row_offset,
+                          partials_dev));
+  }
+  ctx->partials_ready = true;
+  return SFB_OK;
+}
+
+extern "C" int sfb_finish_factors(sfb_ctx* ctx, const float* partials_all_dev, int32_t shards) {
+  if (!ctx || !partials_all_dev) return SFB_ERR_ARG;
+  if (ctx->cfg.model != SFB_MLR) return SFB_ERR_UNSUPPORTED;
+  if (shards < 1 || shards > 4096) return SFB_ERR_ARG;
+  if (!al16(partials_all_dev)) return SFB_ERR_ALIGN;
+  if (!ctx->partials_ready) return SFB_ERR_STATE;
+  const sfb_config& c = ctx->cfg;
+  if (c.precision == SFB_PREC_BF16) {
+    const int rc = tc_finish_factors(ctx, partials_all_dev, shards);
+    if (rc) return rc;
+  } else {
+    CK(mlr_shard_finish(ctx->stream, ctx->at<float>(ctx->lay.U), ctx->K, c.rows, c.rows, ctx->at<int32_t>(ctx->lay.stageL),
+                        ctx->row_offset, partials_all_dev, shards, ctx->at<float>(ctx->lay.loss),
+                        ctx->at<uint32_t>(ctx->lay.status)));
+  }
+  ctx->partials_ready = false;
+  ctx->committed = c.workers == 64 ? ~0ull : ((1ull << c.workers) - 1);
   ctx->gathered = false;
   return SFB_OK;
 }

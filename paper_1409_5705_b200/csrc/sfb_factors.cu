@@ -104,6 +104,75 @@ __global__ void __launch_bounds__(NTHREADS) mlr_softmax_kernel(float* __restrict
   }
 }
 
+// Row-sharded form of the same factor (the parameter matrix partitioned by rows; every shard holds all K samples'
+// logits against its own rows only).  First half, one block per sample: the shard's softmax partial
+//   part[i] = (m_i, s_i, zy_i, has_i):  m_i = max_j z_ij,  s_i = sum_j exp(z_ij - m_i)  over the shard's rows j,
+//   zy_i = z_{i,y_i} and has_i = 1 when class y_i is one of the shard's rows, else 0 and 0.
+// labels are global class ids; the shard holds rows [row_off, row_off + rows).
+template <int NTHREADS>
+__global__ void __launch_bounds__(NTHREADS) mlr_shard_partials_kernel(const float* __restrict__ Z, int64_t rows, int64_t ldz,
+                                                                      const int32_t* __restrict__ labels, int64_t row_off,
+                                                                      float4* __restrict__ part) {
+  __shared__ float sh[32];
+  const float* z = Z + static_cast<int64_t>(blockIdx.x) * ldz;
+  float m = -INFINITY;
+  for (int64_t j = threadIdx.x; j < rows; j += NTHREADS) m = fmaxf(m, z[j]);
+  m = block_max<NTHREADS>(m, sh);
+  float s = 0.f;
+  for (int64_t j = threadIdx.x; j < rows; j += NTHREADS) s += expf(z[j] - m);
+  s = block_sum<NTHREADS>(s, sh);
+  if (threadIdx.x == 0) {
+    const int64_t yl = static_cast<int64_t>(labels[blockIdx.x]) - row_off;
+    const bool mine = yl >= 0 && yl < rows;
+    part[blockIdx.x] = make_float4(m, s, mine ? z[yl] : 0.f, mine ? 1.f : 0.f);
+  }
+}
+
+// Merge of the shards' partials of one sample, in shard order:  lse = M + log sum_g s_g exp(m_g - M),  M = max_g m_g;
+// zy = sum_g zy_g (only the owning shard contributes).  parts is [shards][K].
+__device__ __forceinline__ void merge_shard_partials(const float4* __restrict__ parts, int shards, int64_t K, int64_t i,
+                                                     float& lse, float& zy, float& has) {
+  float M = -INFINITY;
+  for (int g = 0; g < shards; ++g) M = fmaxf(M, parts[static_cast<int64_t>(g) * K + i].x);
+  float S = 0.f;
+  zy = 0.f; has = 0.f;
+  for (int g = 0; g < shards; ++g) {
+    const float4 v = parts[static_cast<int64_t>(g) * K + i];
+    S += v.y * expf(v.x - M);
+    zy += v.z;
+    has += v.w;
+  }
+  lse = M + logf(S);
+}
+
+// Second half, one block per sample: with the global log-partition, u_ij = exp(z_ij - lse_i) - [j is y_i's row] in
+// place over the shard's rows; loss_i = lse_i - z_{i,y_i} (the same on every shard).  A class id that no shard owns
+// sets the status bit and subtracts nothing.
+template <int NTHREADS>
+__global__ void __launch_bounds__(NTHREADS) mlr_shard_finish_kernel(float* __restrict__ Z, int64_t rows, int64_t ldz,
+                                                                    const int32_t* __restrict__ labels, int64_t row_off,
+                                                                    const float4* __restrict__ parts, int shards, int64_t K,
+                                                                    float* __restrict__ loss, uint32_t* status) {
+  __shared__ float sh_lse;
+  float* z = Z + static_cast<int64_t>(blockIdx.x) * ldz;
+  if (threadIdx.x == 0) {
+    float lse, zy, has;
+    merge_shard_partials(parts, shards, K, blockIdx.x, lse, zy, has);
+    const bool ok = has > 0.5f;
+    if (!ok) atomicOr(status, SFB_STATUS_LABEL_RANGE);
+    loss[blockIdx.x] = ok ? lse - zy : 0.f;
+    sh_lse = lse;
+  }
+  __syncthreads();
+  const float lse = sh_lse;
+  const int64_t yl = static_cast<int64_t>(labels[blockIdx.x]) - row_off;
+  for (int64_t j = threadIdx.x; j < rows; j += NTHREADS) {
+    float u = expf(z[j] - lse);
+    if (j == yl) u -= 1.f;
+    z[j] = u;
+  }
+}
+
 // One block per pair: q = ||z||^2; similar: u = 2z; dissimilar: u = -2z if q < margin else 0 (Section 2, DML).
 template <int NTHREADS>
 __global__ void __launch_bounds__(NTHREADS) dml_scale_kernel(float* __restrict__ Z, int64_t rows, int64_t ld,
@@ -311,6 +380,24 @@ cudaError_t mlr_softmax_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t ro
                              float* loss, uint32_t* status) {
   if (nsamp <= 0) return cudaSuccess;
   mlr_softmax_kernel<512><<<static_cast<unsigned>(nsamp), 512, 0, s>>>(Z, rows, labels, loss, status);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t mlr_shard_partials(cudaStream_t s, const float* Z, int64_t nsamp, int64_t rows, int64_t ldz,
+                               const int32_t* labels, int64_t row_off, float* part) {
+  if (nsamp <= 0) return cudaSuccess;
+  mlr_shard_partials_kernel<512><<<static_cast<unsigned>(nsamp), 512, 0, s>>>(Z, rows, ldz, labels, row_off,
+                                                                           reinterpret_cast<float4*>(part));
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t mlr_shard_finish(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows, int64_t ldz, const int32_t* labels,
+                             int64_t row_off, const float* parts, int shards, float* loss, uint32_t* status) {
+  if (nsamp <= 0) return cudaSuccess;
+  mlr_shard_finish_kernel<512><<<static_cast<unsigned>(nsamp), 512, 0, s>>>(
+      Z, rows, ldz, labels, row_off, reinterpret_cast<const float4*>(parts), shards, nsamp, loss, status);
   count_launch();
   return cudaGetLastError();
 }

@@ -55,6 +55,9 @@ struct sfb_ctx {
   cudaStream_t stream;
   int64_t K;
   int64_t in_dim;
+  int64_t row_offset;                 // row-sharded MLR: this context's W holds rows [row_offset, row_offset + rows)
+  int64_t global_rows;                //   of a matrix with global_rows rows (class ids are global); 0, rows when unsharded
+  bool partials_ready;                // sfb_forward_partials has run since the last update
   uint64_t committed;                 // bit p set: worker p has written its factors since the last update
   bool gathered;
   int last_cuda;
@@ -93,6 +96,12 @@ cudaError_t pack_copy(cudaStream_t s, float* dst, const float* x, const float* y
 cudaError_t fill_zero(cudaStream_t s, float* dst, int64_t n);
 cudaError_t mlr_softmax_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows, const int32_t* labels,
                              float* loss_per_sample, uint32_t* status);
+// Row-sharded MLR: per-sample softmax partials (max, sum exp, label logit, owner flag) of a shard, and the finish with
+// the partials of all shards ([shards][nsamp] float4).
+cudaError_t mlr_shard_partials(cudaStream_t s, const float* Z, int64_t nsamp, int64_t rows, int64_t ldz,
+                               const int32_t* labels, int64_t row_off, float* part);
+cudaError_t mlr_shard_finish(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows, int64_t ldz, const int32_t* labels,
+                             int64_t row_off, const float* parts, int shards, float* loss, uint32_t* status);
 cudaError_t dml_scale_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows, int64_t ld,
                            const int32_t* similar, float margin);
 cudaError_t mean_of(cudaStream_t s, const float* v, int64_t n, float* out);

@@ -455,6 +455,61 @@ __global__ void __launch_bounds__(256) mlr_lse_kernel(const float2* __restrict__
   }
 }
 
+// Row-sharded form, first half: one warp per sample merges the forward's per-block (max, sum exp) partials over the
+// shard's rows into the shard's partial (m_i, s_i, zy_i, has_i); zy_i = z_{i,y_i} and has_i = 1 when the shard owns
+// class y_i (labels are global ids; the shard holds rows [row_off, row_off + rows)).
+__global__ void __launch_bounds__(256) mlr_shard_partials_tc_kernel(const float2* __restrict__ part, int64_t part_ld, int nblocks,
+                                                                    const float* __restrict__ Z, int64_t ldz, int64_t rows,
+                                                                    const int32_t* __restrict__ labels, int64_t row_off,
+                                                                    int64_t n, float4* __restrict__ out) {
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * 8 + (threadIdx.x >> 5);
+  if (i >= n) return;
+  const int lane = threadIdx.x & 31;
+  float m = -INFINITY;
+  for (int b = lane; b < nblocks; b += 32) m = fmaxf(m, part[static_cast<int64_t>(b) * part_ld + i].x);
+  m = warp_max(m);
+  float sum = 0.f;
+  for (int b = lane; b < nblocks; b += 32) {
+    const float2 v = part[static_cast<int64_t>(b) * part_ld + i];
+    sum += v.y * __expf(v.x - m);
+  }
+  sum = warp_sum(sum);
+  if (lane == 0) {
+    const int64_t yl = static_cast<int64_t>(labels[i]) - row_off;
+    const bool mine = yl >= 0 && yl < rows;
+    out[i] = make_float4(m, sum, mine ? Z[i * ldz + yl] : 0.f, mine ? 1.f : 0.f);
+  }
+}
+
+// Second half, one thread per sample: merge the partials of all shards ([shards][n], shard order) into the global
+// log-partition; loss = lse - z_y; coef = 1 - p_y for the samples whose class this shard owns (0 otherwise); the class
+// ids are rewritten as row indices of this shard (-1: another shard's row).  A class no shard owns sets the status bit.
+__global__ void __launch_bounds__(256) mlr_shard_finish_tc_kernel(const float4* __restrict__ parts, int shards, int64_t n,
+                                                                  int64_t rows, int64_t row_off, int32_t* __restrict__ labels,
+                                                                  float* __restrict__ lse, float* __restrict__ loss,
+                                                                  float* __restrict__ coef, uint32_t* status) {
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
+  if (i >= n) return;
+  float M = -INFINITY;
+  for (int g = 0; g < shards; ++g) M = fmaxf(M, parts[static_cast<int64_t>(g) * n + i].x);
+  float S = 0.f, zy = 0.f, has = 0.f;
+  for (int g = 0; g < shards; ++g) {
+    const float4 v = parts[static_cast<int64_t>(g) * n + i];
+    S += v.y * expf(v.x - M);
+    zy += v.z;
+    has += v.w;
+  }
+  const float l = M + logf(S);
+  const bool ok = has > 0.5f;
+  if (!ok) atomicOr(status, SFB_STATUS_LABEL_RANGE);
+  const int64_t yl = static_cast<int64_t>(labels[i]) - row_off;
+  const bool mine = ok && yl >= 0 && yl < rows;
+  lse[i] = l;
+  loss[i] = ok ? l - zy : 0.f;
+  coef[i] = mine ? -expm1f(zy - l) : 0.f;
+  labels[i] = mine ? static_cast<int32_t>(yl) : -1;
+}
+
 // P^T[r][off + i] = bf16( exp(z_ir - lse_i) ) for r != y_i and 0 for r = y_i: 64 samples x 64 rows per block,
 // transposed through shared memory (Z is sample-major, the update operand is row-major with samples
 // contiguous).  The factor is u_i = p_i - onehot(y_i); its label entry u_iy = p_iy - 1 is left out of the bf16
@@ -732,34 +787,25 @@ int factors_split(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const fl
 
 }  // namespace
 
-int tc_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float* Y, const int32_t* labels) {
-  if (ctx->cfg.model != SFB_MLR) return factors_split(ctx, off, n, X, Y, labels);
+// Pack of n samples at pair offset off and their logits against the rows of this context's W:
+// Z[off .. off+n) = X W^T with the per-(sample, 256-row block) softmax partials.
+static int mlr_forward(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const int32_t* labels, int* tiles_n) {
   const sfb_config& c = ctx->cfg;
   const TcState* st = static_cast<const TcState*>(ctx->tc);
   const Layout& L = ctx->lay;
   const int64_t rows = c.rows, cols = c.cols, K = ctx->K;
   const int64_t ldz = round_up(rows, 32);
   __nv_bfloat16* Xb = ctx->at<__nv_bfloat16>(L.Xb);
-  __nv_bfloat16* VT = ctx->at<__nv_bfloat16>(L.VT);
-  __nv_bfloat16* Wb = ctx->at<__nv_bfloat16>(L.Wb);
-  __nv_bfloat16* UT = ctx->at<__nv_bfloat16>(L.UT);
-  float* Z = ctx->at<float>(L.ZT);
-  float2* part = ctx->at<float2>(L.part);
-  float* lse = ctx->at<float>(L.V);
-  float* loss = ctx->at<float>(L.loss);
-  uint32_t* status = ctx->at<uint32_t>(L.status);
-
   dim3 pgrid(static_cast<unsigned>((cols + 63) / 64), static_cast<unsigned>((n + 63) / 64));
-  pack_mlr_kernel<<<pgrid, 256, 0, ctx->stream>>>(X, n, cols, Xb, L.colsb, VT, L.Kp, off, ctx->at<float>(L.Xf), labels,
-                                                  ctx->at<int32_t>(L.labels));
+  pack_mlr_kernel<<<pgrid, 256, 0, ctx->stream>>>(X, n, cols, Xb, L.colsb, ctx->at<__nv_bfloat16>(L.VT), L.Kp, off,
+                                                  ctx->at<float>(L.Xf), labels, ctx->at<int32_t>(L.labels));
   count_launch();
   CKC(cudaGetLastError());
-
-  // Z[off .. off+n) = X W^T : samples on the lanes (A), rows of W on the accumulator columns (B)
+  // samples on the lanes (A), rows of W on the accumulator columns (B)
   CUtensorMap ma, mb, mc;
   if (!make_map(st, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, Xb, cols, off + n, L.colsb * 2, BK, BM) ||
-      !make_map(st, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, Wb, cols, rows, L.colsb * 2, BK, BN) ||
-      !make_map(st, &mc, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, Z, rows, off + n, ldz * 4, kChunk, 32))
+      !make_map(st, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, ctx->at<__nv_bfloat16>(L.Wb), cols, rows, L.colsb * 2, BK, BN) ||
+      !make_map(st, &mc, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, ctx->at<float>(L.ZT), rows, off + n, ldz * 4, kChunk, 32))
     return SFB_ERR_CUDA;
   TcParams p{};
   p.M = static_cast<int32_t>(off + n); p.N = static_cast<int32_t>(rows); p.Kc = static_cast<int32_t>(cols);
@@ -767,16 +813,61 @@ int tc_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float
   p.tilesM = static_cast<int32_t>((n + BM - 1) / BM);
   p.bn = BN;
   p.tilesN = static_cast<int32_t>((rows + BN - 1) / BN);
-  p.part = part; p.part_ld = K; p.status = status;
+  p.part = ctx->at<float2>(L.part); p.part_ld = K; p.status = ctx->at<uint32_t>(L.status);
   p.nseg = 1; p.kseg = (p.Kc + BK - 1) / BK;
   CKC(launch_forward<F_SOFTMAX>(ctx, ma, mb, mc, p));
   ctx->stats.flops += 2.0 * n * rows * cols;
+  *tiles_n = p.tilesN;
+  return SFB_OK;
+}
 
-  mlr_lse_kernel<<<static_cast<unsigned>((n + 7) / 8), 256, 0, ctx->stream>>>(part, K, p.tilesN, Z, ldz, rows, labels, off,
-                                                                              n, lse, loss, ctx->at<float>(L.coef), status);
+int tc_forward_partials(sfb_ctx* ctx, const float* X, const int32_t* labels, float* part_out) {
+  const sfb_config& c = ctx->cfg;
+  const Layout& L = ctx->lay;
+  int tiles_n = 0;
+  const int rc = mlr_forward(ctx, 0, ctx->K, X, labels, &tiles_n);
+  if (rc) return rc;
+  mlr_shard_partials_tc_kernel<<<static_cast<unsigned>((ctx->K + 7) / 8), 256, 0, ctx->stream>>>(
+      ctx->at<float2>(L.part), ctx->K, tiles_n, ctx->at<float>(L.ZT), round_up(c.rows, 32), c.rows,
+      ctx->at<int32_t>(L.labels), ctx->row_offset, ctx->K, reinterpret_cast<float4*>(part_out));
+  count_launch();
+  CKC(cudaGetLastError());
+  return SFB_OK;
+}
+
+int tc_finish_factors(sfb_ctx* ctx, const float* parts, int shards) {
+  const sfb_config& c = ctx->cfg;
+  const Layout& L = ctx->lay;
+  const int64_t K = ctx->K;
+  mlr_shard_finish_tc_kernel<<<static_cast<unsigned>((K + 255) / 256), 256, 0, ctx->stream>>>(
+      reinterpret_cast<const float4*>(parts), shards, K, c.rows, ctx->row_offset, ctx->at<int32_t>(L.labels),
+      ctx->at<float>(L.V), ctx->at<float>(L.loss), ctx->at<float>(L.coef), ctx->at<uint32_t>(L.status));
+  count_launch();
+  dim3 egrid(static_cast<unsigned>((c.rows + 63) / 64), static_cast<unsigned>((K + 63) / 64));
+  mlr_emit_ut_kernel<<<egrid, 256, 0, ctx->stream>>>(ctx->at<float>(L.ZT), round_up(c.rows, 32), c.rows, ctx->at<float>(L.V), 0, K,
+                                                     ctx->at<int32_t>(L.labels), ctx->at<__nv_bfloat16>(L.UT), L.Kp);
+  count_launch();
+  CKC(cudaGetLastError());
+  return SFB_OK;
+}
+
+int tc_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float* Y, const int32_t* labels) {
+  if (ctx->cfg.model != SFB_MLR) return factors_split(ctx, off, n, X, Y, labels);
+  const sfb_config& c = ctx->cfg;
+  const Layout& L = ctx->lay;
+  const int64_t rows = c.rows, K = ctx->K;
+  const int64_t ldz = round_up(rows, 32);
+  float* Z = ctx->at<float>(L.ZT);
+  float* lse = ctx->at<float>(L.V);
+  int tiles_n = 0;
+  const int rc = mlr_forward(ctx, off, n, X, labels, &tiles_n);
+  if (rc) return rc;
+  mlr_lse_kernel<<<static_cast<unsigned>((n + 7) / 8), 256, 0, ctx->stream>>>(
+      ctx->at<float2>(L.part), K, tiles_n, Z, ldz, rows, labels, off, n, lse, ctx->at<float>(L.loss), ctx->at<float>(L.coef),
+      ctx->at<uint32_t>(L.status));
   count_launch();
   dim3 egrid(static_cast<unsigned>((rows + 63) / 64), static_cast<unsigned>((n + 63) / 64));
-  mlr_emit_ut_kernel<<<egrid, 256, 0, ctx->stream>>>(Z, ldz, rows, lse, off, n, labels, UT, L.Kp);
+  mlr_emit_ut_kernel<<<egrid, 256, 0, ctx->stream>>>(Z, ldz, rows, lse, off, n, labels, ctx->at<__nv_bfloat16>(L.UT), L.Kp);
   count_launch();
   CKC(cudaGetLastError());
   return SFB_OK;

@@ -12,6 +12,10 @@ void tc_extend_layout(const sfb_config& c, Layout& L, size_t& off);
 int tc_init(sfb_ctx* ctx);
 void tc_destroy(sfb_ctx* ctx);
 int tc_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float* Y, const int32_t* labels);
+// Row-sharded MLR: logits and softmax partials of all K samples against this context's rows; then the factors from
+// the partials of all shards.
+int tc_forward_partials(sfb_ctx* ctx, const float* X, const int32_t* labels, float* part_out);
+int tc_finish_factors(sfb_ctx* ctx, const float* parts, int shards);
 int tc_gather(sfb_ctx* ctx);
 int tc_update(sfb_ctx* ctx);
 int tc_get_factors(sfb_ctx* ctx, const void** U, const void** V, int32_t* dtype, int32_t* layout, int64_t* ldu,

@@ -1,0 +1,82 @@
+"""Row-sharded multiclass logistic regression over several GPUs: host-side sequencing only.
+
+Each rank owns a contiguous block of the rows (classes) of W and a block of the K samples of a step (its logical
+workers).  One step is
+
+    all-gather of the ranks' samples and class ids          K*cols*4 + K*4 bytes received in total per rank
+    sfb_forward_partials on the local rows                  (library kernels)
+    all-gather of the per-sample softmax partials           shards*K*16 bytes
+    sfb_finish_factors, sfb_gather_factors, sfb_apply_update on the local rows   (library kernels)
+
+so W, U and the update never leave their GPU.  The collectives run through ``torch.distributed`` on whatever backend
+the process group has (NCCL on GPUs); no arithmetic happens here.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+
+def row_shard_bounds(rows: int, shards: int, g: int) -> tuple[int, int]:
+    """Rows [r0, r1) of shard g when ``rows`` rows are dealt to ``shards`` shards as evenly as possible (the first
+    ``rows % shards`` shards get one row more)."""
+    if not (0 <= g < shards) or shards < 1 or rows < shards:
+        raise ValueError(f"bad shard {g} of {shards} for {rows} rows")
+    base, rem = divmod(rows, shards)
+    r0 = g * base + min(g, rem)
+    return r0, r0 + base + (1 if g < rem else 0)
+
+
+@dataclass
+class ExchangeBytes:
+    """Bytes this rank received in the collectives of one step."""
+    samples: int = 0
+    partials: int = 0
+
+    @property
+    def total(self) -> int:
+        return self.samples + self.partials
+
+
+def exchange_model_bytes(P: int, B: int, rows: int, cols: int, shards: int) -> dict:
+    """Values moved per step by the schemes of the paper's cost table (Section 5), in bytes of fp32, for P workers with
+    B samples each, beside what the row-sharded step moves: the paper's peer-to-peer broadcast of sufficient factors,
+    P*(P-1)*B*(rows+cols); full-matrix synchronisation, P*rows*cols (every worker's update matrix); row sharding,
+    per rank the other ranks' samples plus everyone's partials."""
+    K = P * B
+    return {
+        "sfb_p2p": 4 * P * (P - 1) * B * (rows + cols),
+        "full_matrix_sync": 4 * P * rows * cols,
+        "row_sharded_per_rank": (shards - 1) * (K // shards) * (cols * 4 + 4) + (shards - 1) * K * 16,
+    }
+
+
+def sharded_step(ctx, X_local, labels_local, partials, partials_all, X_all, labels_all, group=None, dist=None):
+    """One row-sharded step on this rank.
+
+    ctx            a context over this rank's rows, already told its shard with ``sfb_set_row_shard``
+    X_local        [K/shards, cols] this rank's samples; labels_local [K/shards] their (global) class ids
+    partials       [K, 4] scratch for this rank's partials;  partials_all  [shards, K, 4]
+    X_all          [K, cols] and labels_all [K]: receive the gathered samples (rank-major = worker-major order)
+    dist           the ``torch.distributed`` module (or a stand-in with the same two calls); None: single shard
+    Returns the ExchangeBytes of the step.
+    """
+    moved = ExchangeBytes()
+    if dist is None:
+        X_all.copy_(X_local)
+        labels_all.copy_(labels_local)
+    else:
+        dist.all_gather_into_tensor(X_all, X_local, group=group)
+        dist.all_gather_into_tensor(labels_all, labels_local, group=group)
+        moved.samples = (X_all.numel() - X_local.numel()) * X_all.element_size() + \
+                        (labels_all.numel() - labels_local.numel()) * labels_all.element_size()
+    ctx.sfb_forward_partials(X_all, labels_all, partials)
+    if dist is None:
+        partials_all.view(-1).copy_(partials.view(-1))
+    else:
+        dist.all_gather_into_tensor(partials_all.view(-1, partials.shape[-1]), partials, group=group)   # shard-major rows
+        moved.partials = (partials_all.numel() - partials.numel()) * partials_all.element_size()
+    shards = partials_all.shape[0]
+    ctx.sfb_finish_factors(partials_all, shards)
+    ctx.sfb_gather_factors()
+    ctx.sfb_apply_update()
+    return moved
