@@ -4,6 +4,8 @@ roofline fraction, an end-to-end (host buffers) figure and the CPU oracle timed 
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--precision bf16|fp32] [--workload mlr_large]
     python bench.py --impl reference ...      # times the fp64 CPU oracle on a bounded sample instead
+    python bench.py --phase update ...        # adds a loop of the fused update alone (>= 2 s, back to back)
+    torchrun ... bench.py --gpus N --shard rows   # W partitioned by rows over the N ranks (one exchange per step)
 
 A step is one pass of the whole hot path over one minibatch of K = P*B synthetic samples: pack, forward
 product, softmax-minus-onehot, gather, fused rank-K update of W.  Prints ONE JSON line on rank 0.
@@ -72,6 +74,39 @@ def oracle_sample_setup(wl, budget_s):
     per_row = (time.perf_counter() - t0) / probe_rows             # seconds per row of W on this machine
     rows = int(max(probe_rows, min(wl.rows, budget_s / per_row)))
     return make(rows), rows
+
+
+def host_mem_available_gb():
+    try:
+        for line in open("/proc/meminfo"):
+            if line.startswith("MemAvailable:"):
+                return int(line.split()[1]) / 1e6
+    except OSError:
+        pass
+    return 0.0
+
+
+def time_oracle_mlr_full_forward(wl, W_host, sample_rows=8192):
+    """Paper-scale MLR on the host cores with the oracle's own routines for shapes too large to hold W in fp64:
+    the log-partition of all K samples over ALL rows of W (the whole forward product, visited block by block),
+    then the update of a contiguous sample of rows from that log-partition, its time scaled to all rows.  The
+    sampled-row routine forms the logits of its rows again, so the scaled figure is an upper bound on the time of
+    a step that keeps them."""
+    from oracle import sfb_oracle as O
+    inp = I.step_inputs(wl, 0)
+    t0 = time.perf_counter()
+    lse = O.mlr_log_partition(W_host, inp.X)
+    t_fwd = time.perf_counter() - t0
+    n = int(min(sample_rows, wl.rows))
+    ids = np.arange(n)
+    t0 = time.perf_counter()
+    O.mlr_updated_rows(W_host[:n], ids, inp.X, inp.labels, lse, wl.eta)
+    t_upd = time.perf_counter() - t0
+    full = t_fwd + t_upd * wl.rows / n
+    sample = (f"oracle on the full problem: log-partition of all K={wl.K} samples over all {wl.rows} rows "
+              f"({t_fwd:.1f} s), then the updated rows of a sample of {n} rows ({t_upd:.2f} s, scaled by "
+              f"{wl.rows}/{n}; that routine recomputes its rows' logits)")
+    return wl.K / full, t_fwd + t_upd, sample
 
 
 def cores_used():
@@ -187,10 +222,12 @@ def run_reference(args, wl, rank):
     print(json.dumps(line), flush=True)
 
 
-# DRAM bytes per launch of the update kernel from the ncu capture summarised in profiles/ (a slab of 16384 rows of
-# the paper-scale MLR shape; traffic is proportional to the rows, see that file).  None when the kernel or the
-# workload is not the captured one.
-NCU_UPDATE_TRAFFIC = {"rows": 16384, "cols": 10000, "K": 1024, "bytes": 764645888 + 933098496}
+# DRAM bytes per launch of the update kernel from the ncu capture summarised in
+# profiles/ncu_update_pair_kernel_mlr_rows16384.md (a slab of 16384 rows of the paper-scale MLR shape; traffic is
+# proportional to the rows, see that file).  "kernel_unchanged_since" names the commit of csrc/sfb_update.cu the
+# counters were taken at: when the kernel is edited this entry has to be re-captured or set to None.
+NCU_UPDATE_TRAFFIC = {"rows": 16384, "cols": 10000, "K": 1024, "bytes": 764645888 + 933098496,
+                      "kernel_unchanged_since": "cf145f9"}
 
 
 def ncu_traffic_per_launch(wl, prec):
@@ -207,6 +244,181 @@ def workload_config(wl, dtype):
             else "l2_flushed_between_steps"}
 
 
+NOMINAL_BF16_TFLOPS = 2250.0        # dense bf16, vendor figure (context only)
+NOMINAL_HBM_GBS = 7700.0
+
+
+def update_roofline(wl, prec_bf16, ms_u, peaks, clocks, sustained=True):
+    """Roofline entry of the fused update W += -eta U^T V (one launch per step).  Algorithmic bytes per launch: W read
+    and written once in fp32 plus U and V read once (what the method has to move).  The bf16 copy of W that this design
+    writes alongside (the operand of the next forward product) is real traffic of the kernel and is reported beside
+    it, not counted as algorithmic."""
+    K = wl.K
+    esz = 2 if prec_bf16 else 4
+    if prec_bf16 and wl.model != I.MLR:
+        esz = 4                                                               # (hi, lo) pairs of bf16
+    upd_flops = 2.0 * wl.rows * wl.cols * K
+    upd_bytes = 8.0 * wl.rows * wl.cols + K * (wl.rows + wl.cols) * esz
+    shadow_bytes = 2.0 * wl.rows * wl.cols if (prec_bf16 and wl.model == I.MLR) else 0.0
+    tf_peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
+    if prec_bf16:
+        t_flop = upd_flops / (tf_peak * 1e12)
+        t_mem = upd_bytes / (peaks["hbm_gbs"] * 1e9)
+        if t_mem >= t_flop:
+            roof = {"bound": "hbm", "achieved": upd_bytes / (ms_u * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s"}
+        else:
+            roof = {"bound": "tensor", "achieved": upd_flops / (ms_u * 1e-3) / 1e12, "peak": tf_peak,
+                    "unit": "TFLOP/s"}
+        roof["roof_ms"] = max(t_flop, t_mem) * 1e3
+    else:
+        # fp32 FMA pipe: SMs x 128 lanes x 2 flop x max SM clock
+        peak = 148 * 128 * 2 * ((clocks or {}).get("sm_max_mhz") or 1965.0) * 1e6 / 1e12
+        roof = {"bound": "alu", "achieved": upd_flops / (ms_u * 1e-3) / 1e12, "peak": peak, "unit": "TFLOP/s"}
+        roof["roof_ms"] = upd_flops / (peak * 1e12) * 1e3
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = ncu_traffic_per_launch(wl, 0 if prec_bf16 else 1)
+    roof["traffic_captured_at"] = NCU_UPDATE_TRAFFIC["kernel_unchanged_since"] if roof["traffic"] else None
+    roof["kernel"] = "update_pair_kernel + label_rows_kernel (sfb_apply_update)" if prec_bf16 \
+        else "sgemm_kernel EPI_RMW (sfb_apply_update)"
+    roof["ms"] = ms_u
+    roof["peaks"] = "of " + peaks["source"] + (" (sustained tensor figure: timed inside a long step)" if sustained
+                                               else " (burst tensor figure: timed alone)")
+    roof["update_tflops"] = upd_flops / (ms_u * 1e-3) / 1e12
+    roof["frac_of_measured_sustained"] = roof["update_tflops"] / peaks["bf16_tflops_sustained"]
+    roof["frac_of_measured_burst"] = roof["update_tflops"] / peaks["bf16_tflops"]
+    roof["frac_of_nominal_peak"] = max(roof["update_tflops"] / NOMINAL_BF16_TFLOPS,
+                                       upd_bytes / (ms_u * 1e-3) / 1e9 / NOMINAL_HBM_GBS) if prec_bf16 else None
+    roof["algorithmic_bytes"] = upd_bytes
+    roof["algorithmic_flops"] = upd_flops
+    roof["achieved_incl_bf16_copy_of_W"] = (upd_bytes + shadow_bytes) / (ms_u * 1e-3) / 1e9
+    return roof
+
+
+def forward_and_step_rooflines(wl, ms_f, ms_step, upd_roof_ms, peaks):
+    """Rooflines of the factor phase (bf16 MLR: forward product + softmax finish) and of the whole step, against the
+    measured sustained tensor figure and the measured copy bandwidth."""
+    K = wl.K
+    fl = 2.0 * wl.rows * wl.cols * K
+    t_fwd = max(fl / (peaks["bf16_tflops_sustained"] * 1e12),
+                (2.0 * wl.rows * wl.cols + 4.0 * K * wl.rows) / (peaks["hbm_gbs"] * 1e9))        # bf16 W in, logits out
+    t_fin = (4.0 * K * wl.rows + 2.0 * K * wl.rows) / (peaks["hbm_gbs"] * 1e9)                    # logits in, bf16 U out
+    fwd = {"bound": "tensor", "roof_ms": (t_fwd + t_fin) * 1e3, "ms": ms_f, "frac": (t_fwd + t_fin) * 1e3 / ms_f,
+           "achieved": fl / (ms_f * 1e-3) / 1e12, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+           "kernel": "pack + forward_kernel + softmax finish (sfb_compute_factors)"}
+    roof_ms = (t_fwd + t_fin) * 1e3 + upd_roof_ms
+    step = {"roof_ms": roof_ms, "ms": ms_step, "frac": roof_ms / ms_step}
+    return fwd, step
+
+
+def draw_W(torch, wl, dev, seed, rows=None):
+    """W ~ the workload's init distribution, drawn on the device (13 GB of host generation would dominate the run)."""
+    rows = wl.rows if rows is None else rows
+    g = torch.Generator(device=dev)
+    g.manual_seed(seed)
+    W = torch.empty((rows, wl.cols), dtype=torch.float32, device=dev)
+    std = {"normal": wl.w_std, "dml": 1.0 / math.sqrt(wl.cols), "zeros": 0.0, "unit_columns": 1.0}[wl.w_init]
+    for r0 in range(0, rows, 65536):
+        blk = W[r0:r0 + 65536]
+        if std == 0.0:
+            blk.zero_()
+        else:
+            blk.normal_(0.0, std, generator=g)
+    return W
+
+
+# ----------------------------------------------------------------------------------------------------------
+# W partitioned by rows over the ranks (strong scaling: one problem, N GPUs)
+# ----------------------------------------------------------------------------------------------------------
+def run_sharded(args, wl, rank, world, local):
+    import torch
+    import torch.distributed as dist
+    import paper_1409_5705_b200 as S
+    from paper_1409_5705_b200.sharded import exchange_model_bytes, row_shard_bounds, sharded_step
+
+    if wl.model != I.MLR:
+        raise SystemExit("--shard rows is built for the MLR workloads")
+    if wl.K % world != 0:
+        raise SystemExit(f"K = {wl.K} samples do not split over {world} ranks")
+    if world > 1:
+        # NCCL's own log (communicator set-up: ranks, transports) goes to a file, not into the JSON line's stream
+        os.environ.setdefault("NCCL_DEBUG", "INFO")
+        os.environ.setdefault("NCCL_DEBUG_FILE", os.path.join(tempfile.gettempdir(), "sfb_nccl.%h.%p.log"))
+    S.build()
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl")
+    dev = torch.device("cuda", local)
+    prec = S.PREC_BF16 if args.precision == "bf16" else S.PREC_FP32
+    peaks = load_peaks()
+    r0, r1 = row_shard_bounds(wl.rows, world, rank)
+    W = draw_W(torch, wl, dev, 1234 + rank, rows=r1 - r0)
+    K, n = wl.K, wl.K // world
+    nb = 4
+    batches = [I.step_inputs(wl, t) for t in range(nb)]                 # every rank draws the step, keeps its workers
+    dX = [torch.from_numpy(b.X[rank * n:(rank + 1) * n]).to(dev) for b in batches]
+    dL = [torch.from_numpy(b.labels[rank * n:(rank + 1) * n]).to(dev) for b in batches]
+    cfg = S.make_config(wl.model, r1 - r0, wl.cols, wl.workers, wl.batch, wl.eta, prec)
+    ctx = S.Context(cfg, W)
+    ctx.sfb_set_row_shard(r0, wl.rows)
+    partials = torch.zeros((K, 4), dtype=torch.float32, device=dev)
+    partials_all = torch.zeros((world, K, 4), dtype=torch.float32, device=dev)
+    X_all = torch.zeros((K, wl.cols), dtype=torch.float32, device=dev)
+    y_all = torch.zeros((K,), dtype=torch.int32, device=dev)
+    d = dist if world > 1 else None
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler, sfile = clocks_sampler(local) if rank == 0 else (None, None)
+    moved = None
+    for i in range(args.warmup):
+        moved = sharded_step(ctx, dX[i % nb], dL[i % nb], partials, partials_all, X_all, y_all, dist=d)
+    launches0 = ctx.sfb_get_stats().kernel_launches
+    barrier()
+    wall0 = time.time()
+    t_start = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    for i in range(args.steps):
+        sharded_step(ctx, dX[i % nb], dL[i % nb], partials, partials_all, X_all, y_all, dist=d)
+    t_end.record()
+    barrier()
+    clocks = clocks_summary(sampler, sfile, wall0, time.time()) if rank == 0 else None
+    total_ms = t_start.elapsed_time(t_end)
+    st = ctx.sfb_get_stats()
+    launches = st.kernel_launches - launches0
+    status = ctx.sfb_get_status()
+    ms_u = st.ms_update
+    total_ms, ms_u = max_over_ranks([total_ms, ms_u], dev, world)
+    if rank == 0:
+        value = K * args.steps / (total_ms * 1e-3)                          # one problem: K samples per step in all
+        shard = I.scaled(wl, wl.name, rows=r1 - r0)
+        roof = update_roofline(shard, prec == S.PREC_BF16, ms_u, peaks, clocks)
+        roof["traffic"] = None
+        roof["traffic_captured_at"] = None
+        model = exchange_model_bytes(wl.workers, wl.batch, wl.rows, wl.cols, world)
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+                "scaling": "strong", "vs_baseline": None, "dtype": "bf16" if prec == S.PREC_BF16 else "f32",
+                "data": "synthetic",
+                "config": dict(workload_config(wl, "bf16" if prec == S.PREC_BF16 else "f32"),
+                               parallelism=f"rows{world}", rows_per_rank=r1 - r0),
+                "roofline": roof, "cpu_baseline": None, "e2e": None, "gpu_launches": int(launches), "clocks": clocks,
+                "exchange": {"measured_bytes_received_per_rank": moved.total if moved else 0,
+                             "samples": moved.samples if moved else 0, "partials": moved.partials if moved else 0,
+                             "model_row_sharded_per_rank": model["row_sharded_per_rank"] if world > 1 else 0,
+                             "paper_sfb_p2p_total": model["sfb_p2p"],
+                             "paper_full_matrix_sync_total": model["full_matrix_sync"]},
+                "status_word": status}
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -218,6 +430,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--rows", type=int, default=0,
                     help="run a slab of the workload with this many rows of W (small cases for profiler captures)")
+    ap.add_argument("--phase", default="", choices=["", "update"],
+                    help="update: after the timed steps, loop the fused update alone for --phase-seconds")
+    ap.add_argument("--phase-seconds", type=float, default=2.0)
+    ap.add_argument("--shard", default="", choices=["", "rows"],
+                    help="rows: partition W by rows over the ranks instead of running replicas")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     wl = I.WORKLOADS[args.workload]
@@ -229,6 +446,9 @@ def main():
 
     if args.impl == "reference":
         run_reference(args, wl, rank)
+        return
+    if args.shard == "rows":
+        run_sharded(args, wl, rank, world, local)
         return
 
     import torch
@@ -245,22 +465,19 @@ def main():
     prec = S.PREC_BF16 if args.precision == "bf16" else S.PREC_FP32
     peaks = load_peaks()
 
-    # ---- synthetic state: W ~ the workload's init distribution, drawn on the device; minibatches from the
-    # seeded input module (each rank its own step indices)
-    g = torch.Generator(device=dev)
-    g.manual_seed(1234 + rank)
-    W = torch.empty((wl.rows, wl.cols), dtype=torch.float32, device=dev)
-    std = {"normal": wl.w_std, "dml": 1.0 / math.sqrt(wl.cols), "zeros": 0.0, "unit_columns": 1.0}[wl.w_init]
-    for r0 in range(0, wl.rows, 65536):
-        blk = W[r0:r0 + 65536]
-        if std == 0.0:
-            blk.zero_()
-        else:
-            blk.normal_(0.0, std, generator=g)
+    # ---- synthetic state: W drawn on the device; minibatches from the seeded input module (each rank its own
+    # step indices)
+    W = draw_W(torch, wl, dev, 1234 + rank)
     L = 0.0
     if wl.w_init == "unit_columns":
         W /= W.norm(dim=0, keepdim=True)
         L = float(torch.linalg.matrix_norm(W, 2) ** 2)
+    # host copy of the initial W for the oracle timed beside the paper-scale run (taken before any step)
+    W_host = None
+    full_forward_oracle = (not args.no_cpu_baseline and world == 1 and wl.model == I.MLR
+                           and wl.rows * wl.cols * 4 > 4e9 and host_mem_available_gb() > wl.rows * wl.cols * 4 / 1e9 + 16)
+    if full_forward_oracle:
+        W_host = W.cpu().numpy()
     nb = 4
     true_dict = I.sc_true_dictionary(wl) if wl.model == I.SC else None
     batches = [I.step_inputs(wl, rank * 1000 + t, true_dict) for t in range(nb)]
@@ -323,6 +540,28 @@ def main():
     ms_g = sum(e[1].elapsed_time(e[2]) for e in evs) / args.steps
     ms_u = sum(e[2].elapsed_time(e[3]) for e in evs) / args.steps
 
+    # ---- the fused update alone, back to back (same factors applied again and again): separates the kernel from the
+    # rest of the step; ms x median SM MHz is the clock-independent figure
+    update_loop = None
+    if args.phase == "update" and rank == 0:
+        sampler2, sfile2 = clocks_sampler(local)
+        for _ in range(3):
+            ctx.sfb_replay_update()
+        torch.cuda.synchronize()
+        reps = max(10, int(args.phase_seconds * 1e3 / max(ms_u, 1e-3)))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        w0 = time.time()
+        e0.record()
+        for _ in range(reps):
+            ctx.sfb_replay_update()
+        e1.record()
+        torch.cuda.synchronize()
+        ck = clocks_summary(sampler2, sfile2, w0, time.time())
+        ms_loop = e0.elapsed_time(e1) / reps
+        update_loop = {"launches": reps, "ms": ms_loop, "seconds": ms_loop * reps * 1e-3, "clocks": ck,
+                       "ms_x_sm_mhz": ms_loop * ck["sm_mhz"] if ck.get("sm_mhz") else None,
+                       "roofline": update_roofline(wl, prec == S.PREC_BF16, ms_loop, peaks, ck)}
+
     # ---- end to end: host minibatch -> sfb_step_host -> loss back on the host, every step
     for i in range(3):
         ctx.sfb_step_host(hX[i % nb], hY[i % nb], hL[i % nb])
@@ -346,53 +585,32 @@ def main():
     e2e_value = aggregate_value(world, K, e2e_steps, e2e_ms)
     h2d = K * wl.in_dim * 4 + (K * wl.cols * 4 if wl.model == I.DML else 0) + (K * 4 if wl.model != I.SC else 0)
 
-    # ---- roofline of the dominant kernel: the fused update  W += -eta U^T V  (one launch per step).
-    # Algorithmic bytes per launch: W read and written once in fp32 plus U and V read once (what the method
-    # itself has to move).  The bf16 copy of W that this design writes alongside (the operand of the next forward
-    # product) is real traffic of the kernel and is reported beside it, not counted as algorithmic.
-    esz = 2 if prec == S.PREC_BF16 else 4
-    if prec == S.PREC_BF16 and wl.model != I.MLR:
-        esz = 4                                                               # (hi, lo) pairs of bf16
-    upd_flops = 2.0 * wl.rows * wl.cols * K
-    upd_bytes = 8.0 * wl.rows * wl.cols + K * (wl.rows + wl.cols) * esz
-    shadow_bytes = 2.0 * wl.rows * wl.cols if (prec == S.PREC_BF16 and wl.model == I.MLR) else 0.0
-    if prec == S.PREC_BF16:
-        t_flop = upd_flops / (peaks["bf16_tflops_sustained"] * 1e12)
-        t_mem = upd_bytes / (peaks["hbm_gbs"] * 1e9)
-        if t_mem >= t_flop:
-            roof = {"bound": "hbm", "achieved": upd_bytes / (ms_u * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
-                    "unit": "GB/s"}
-        else:
-            roof = {"bound": "tensor", "achieved": upd_flops / (ms_u * 1e-3) / 1e12,
-                    "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s"}
-    else:
-        # fp32 FMA pipe: 148 SMs x 128 lanes x 2 flop x max SM clock
-        peak = 148 * 128 * 2 * ((clocks or {}).get("sm_max_mhz") or 1965.0) * 1e6 / 1e12
-        roof = {"bound": "alu", "achieved": upd_flops / (ms_u * 1e-3) / 1e12, "peak": peak, "unit": "TFLOP/s"}
-    roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["traffic"] = ncu_traffic_per_launch(wl, prec)
-    roof["kernel"] = "update_pair_kernel + label_rows_kernel (sfb_apply_update)" if prec == S.PREC_BF16 \
-        else "sgemm_kernel EPI_RMW (sfb_apply_update)"
-    roof["ms"] = ms_u
-    roof["peaks"] = "of " + peaks["source"]
-    roof["update_tflops"] = upd_flops / (ms_u * 1e-3) / 1e12
-    roof["tensor_frac_of_sustained"] = roof["update_tflops"] / peaks["bf16_tflops_sustained"]
-    roof["algorithmic_bytes"] = upd_bytes
-    roof["algorithmic_flops"] = upd_flops
-    roof["achieved_incl_bf16_copy_of_W"] = (upd_bytes + shadow_bytes) / (ms_u * 1e-3) / 1e9
+    # ---- roofline of the dominant kernel (the fused update), timed inside the long step: sustained tensor figure
+    roof = update_roofline(wl, prec == S.PREC_BF16, ms_u, peaks, clocks)
+    roof_fwd, roof_step = (None, None)
+    if prec == S.PREC_BF16 and wl.model == I.MLR:
+        roof_fwd, roof_step = forward_and_step_rooflines(wl, ms_f, total_ms / args.steps, roof["roof_ms"], peaks)
 
     cpu = None
     if not args.no_cpu_baseline and world == 1:       # the oracle is timed beside the single-GPU run only
-        v, dt, sample = time_oracle(wl, 1, 0, 15.0)
+        if W_host is not None:
+            v, dt, sample = time_oracle_mlr_full_forward(wl, W_host)
+        else:
+            v, dt, sample = time_oracle(wl, 1, 0, 15.0)
+            sample += " (row-slab extrapolation: the host has no room for the full matrix, or the workload is small)" \
+                if wl.rows * wl.cols * 4 > 4e9 else ""
         cpu = {"value": v, "unit": UNIT, "cores": cores_used(), "kind": "oracle", "sample": sample,
                "sample_seconds": dt}
 
+    esz = 2 if prec == S.PREC_BF16 else 4
+    if prec == S.PREC_BF16 and wl.model != I.MLR:
+        esz = 4
     one_copy = K * (wl.rows + wl.cols) * esz
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if prec == S.PREC_BF16 else "f32",
             "data": "synthetic", "config": workload_config(wl, "bf16" if prec == S.PREC_BF16 else "f32"),
-            "roofline": roof, "cpu_baseline": cpu,
+            "roofline": roof, "roofline_forward": roof_fwd, "roofline_step": roof_step, "cpu_baseline": cpu,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 8,
                     "ms_per_step": e2e_ms / e2e_steps, "last_loss": loss},
             "gpu_launches": int(launches), "clocks": clocks,
@@ -402,6 +620,8 @@ def main():
                       "dense_sync": wl.workers * wl.rows * wl.cols * 4,
                       "dense_over_sf": wl.workers * wl.rows * wl.cols * 4 / one_copy},
             "status_word": status}
+    if update_loop is not None:
+        line["update_loop"] = update_loop
     print(json.dumps(line), flush=True)
     ctx.close()
     if world > 1:

@@ -119,6 +119,12 @@ int sfb_gather_factors(sfb_ctx* ctx);
  * sc_prox = 1).  Section 2.1 (proximal SGD) and Figure 1. */
 int sfb_apply_update(sfb_ctx* ctx);
 
+/* Measurement hook (the paper has no counterpart): applies the factors gathered by the last completed step once
+ * more, W <- prox(W - eta * U^T V) with the same U and V, so that the reconstruct-and-apply pass can be timed on its
+ * own, back to back.  It moves W a second time by the same update: for benchmarks, not for training.  Counts flops
+ * but no step.  SFB_ERR_STATE before the first completed step or while a step is under way. */
+int sfb_replay_update(sfb_ctx* ctx);
+
 /* compute_factors(all workers) + gather + apply_update for K samples resident on the device. */
 int sfb_step(sfb_ctx* ctx, const float* X_dev, const float* Y_dev, const int32_t* labels_dev);
 

@@ -18,7 +18,8 @@ STATUS_LABEL_RANGE, STATUS_TIMEOUT = 0x1, 0x2
 EXPORTS = ("sfb_workspace_bytes", "sfb_init", "sfb_compute_factors", "sfb_gather_factors", "sfb_apply_update",
            "sfb_step", "sfb_step_host", "sfb_dense_sync_step", "sfb_get_factors", "sfb_get_stats",
            "sfb_get_status", "sfb_strerror", "sfb_last_cuda_error", "sfb_destroy", "sfb_prox_columns_noalloc",
-           "sfb_selftest_wait_timeout", "sfb_set_row_shard", "sfb_forward_partials", "sfb_finish_factors")
+           "sfb_selftest_wait_timeout", "sfb_set_row_shard", "sfb_forward_partials", "sfb_finish_factors",
+           "sfb_replay_update")
 NOALLOC_MAX_COLS = 16384
 
 
@@ -79,6 +80,7 @@ def lib() -> ctypes.CDLL:
         L.sfb_set_row_shard.argtypes = [vp, i64, i64]
         L.sfb_forward_partials.argtypes = [vp, vp, vp, vp]
         L.sfb_finish_factors.argtypes = [vp, vp, i32]
+        L.sfb_replay_update.argtypes = [vp]
         for name in EXPORTS:
             if name != "sfb_strerror":
                 getattr(L, name).restype = ctypes.c_int
@@ -146,6 +148,9 @@ class Context:
 
     def sfb_apply_update(self):
         self._ck(lib().sfb_apply_update(self._h), "sfb_apply_update")
+
+    def sfb_replay_update(self):
+        self._ck(lib().sfb_replay_update(self._h), "sfb_replay_update")
 
     def sfb_step(self, X, Y=None, labels=None):
         self._ck(lib().sfb_step(self._h, _ptr(X), _ptr(Y), _ptr(labels)), "sfb_step")

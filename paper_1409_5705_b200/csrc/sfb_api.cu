@@ -353,6 +353,20 @@ extern "C" int sfb_apply_update(sfb_ctx* ctx) {
   return SFB_OK;
 }
 
+extern "C" int sfb_replay_update(sfb_ctx* ctx) {
+  if (!ctx) return SFB_ERR_ARG;
+  if (ctx->stats.steps < 1 || ctx->committed != 0 || ctx->partials_ready) return SFB_ERR_STATE;
+  const sfb_config& c = ctx->cfg;
+  CK(cudaEventRecord(ctx->ev[2], ctx->stream));
+  int rc = c.precision == SFB_PREC_FP32 ? update_fp32(ctx) : tc_update(ctx);
+  if (rc) return rc;
+  ctx->stats.flops += 2.0 * c.rows * c.cols * ctx->K;
+  rc = apply_prox(ctx);
+  if (rc) return rc;
+  CK(cudaEventRecord(ctx->ev[3], ctx->stream));
+  return SFB_OK;
+}
+
 extern "C" int sfb_step(sfb_ctx* ctx, const float* X_dev, const float* Y_dev, const int32_t* labels_dev) {
   if (!ctx) return SFB_ERR_ARG;
   ctx->committed = 0;
