@@ -34,16 +34,23 @@ def rel_err(W_gpu, W_ref64, W0):
     return float(np.linalg.norm(W_gpu.astype(np.float64) - ref32) / den)
 
 
-def entries_ok(W_gpu, W_ref64, W0, tol):
-    """Entry-wise check for rows whose update is only a few fp32 ulps of W (rows of classes absent from the
-    batch): every stored entry must lie within half an fp32 spacing of the oracle's value, plus 8*tol times
-    the rms entry of the update on those rows.  A missing or misplaced update (tens of ulps) fails it."""
+def entries_excess(W_gpu, W_ref64, W0, stores=1):
+    """Largest entry-wise error beyond what storing W in fp32 `stores` times allows (half an fp32 spacing per store),
+    in units of the rms entry of the update."""
     ref32 = np.abs(W_ref64).astype(np.float32)
-    half_ulp = 0.5 * np.spacing(ref32).astype(np.float64)
+    half_ulp = 0.5 * stores * np.spacing(ref32).astype(np.float64)
     upd = W_ref64 - W0.astype(np.float64)
     rms = float(np.sqrt((upd * upd).mean()))
     excess = np.abs(W_gpu.astype(np.float64) - W_ref64) - half_ulp
-    return float(excess.max()) <= 8 * tol * rms
+    return float(excess.max()) / rms
+
+
+def entries_ok(W_gpu, W_ref64, W0, tol, stores=1):
+    """Entry-wise check, for what a norm over the whole matrix can hide (rows whose update is only a few fp32 ulps
+    of W, a ragged last tile): every stored entry must lie within half an fp32 spacing per store of the oracle's
+    value, plus 8*tol times the rms entry of the update on those rows.  A missing or misplaced update (tens of
+    ulps) fails it."""
+    return entries_excess(W_gpu, W_ref64, W0, stores) <= 8 * tol
 
 
 def storage_floor(W_ref64, W0):
@@ -54,6 +61,8 @@ def storage_floor(W_ref64, W0):
     return float(np.linalg.norm(ref32 - W_ref64) / np.linalg.norm(W_ref64 - W0.astype(np.float64)))
 
 
-def step_tol(wl, prec, W_ref64, W0):
-    extra = 2.0 * storage_floor(W_ref64, W0) if wl.model == I.SC else 0.0
+def step_tol(wl, prec, W_ref64, W0, prox=True):
+    """Tolerance of one step: the stated bound, plus for sparse coding the storage floor once per extra store of W
+    (with the prox the step stores W twice: twice the floor; without it once: one floor)."""
+    extra = (2.0 if prox else 1.0) * storage_floor(W_ref64, W0) if wl.model == I.SC else 0.0
     return TOL[prec] + extra
