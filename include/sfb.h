@@ -105,8 +105,12 @@ int sfb_init(const sfb_config* cfg, float* W_dev, void* workspace_dev, size_t wo
  *        v = x - y, u = 2 W v (similar), -2 W v if ||W v||^2 < margin else 0       (Section 2, DML)
  *   SC : v = a = ISTA code of x, u = W a - x                                        (Figure 3)
  * Factors are written at the worker's row offset p*B of the gathered buffers.  All P workers of a step see the
- * same W (bulk-synchronous consistency, Section 4.1): copies of W that the library derives (bf16 operands) are
- * refreshed by the first call of a step. */
+ * same W (bulk-synchronous consistency, Section 4.1).
+ * Copies of W that the library derives: in bf16 mode the forward product reads a bf16 operand copy of W.  DML and SC
+ * rebuild theirs from W in the first factors call of every step.  MLR builds it once in sfb_init and afterwards the
+ * update pass rewrites it together with W (W makes one trip through the SM per step), so it tracks every change the
+ * LIBRARY makes to W -- but not writes the caller makes to W_dev between steps (loading weights, rescaling, a prox of
+ * its own): after such a write call sfb_refresh_operands, or the next forward product runs on the stale copy. */
 int sfb_compute_factors(sfb_ctx* ctx, int32_t worker, const float* X_dev, const float* Y_dev,
                         const int32_t* labels_dev);
 
@@ -118,6 +122,11 @@ int sfb_gather_factors(sfb_ctx* ctx);
 /* Reconstruct and apply:  W <- W - eta * U^T V  in one pass over W, then the proximal operator (SC, when
  * sc_prox = 1).  Section 2.1 (proximal SGD) and Figure 1. */
 int sfb_apply_update(sfb_ctx* ctx);
+
+/* Re-derives the library's operand copies of W from the caller's W_dev (enqueued on the stream): to be called after
+ * the caller itself has written W_dev between two steps.  MLR in bf16 mode: one conversion pass over W (reads 4,
+ * writes 2 bytes per entry); a no-op for the other models and for fp32 mode.  SFB_ERR_STATE in the middle of a step. */
+int sfb_refresh_operands(sfb_ctx* ctx);
 
 /* Measurement hook (the paper has no counterpart): applies the factors gathered by the last completed step once
  * more, W <- prox(W - eta * U^T V) with the same U and V, so that the reconstruct-and-apply pass can be timed on its

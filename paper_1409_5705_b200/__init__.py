@@ -19,7 +19,7 @@ EXPORTS = ("sfb_workspace_bytes", "sfb_init", "sfb_compute_factors", "sfb_gather
            "sfb_step", "sfb_step_host", "sfb_dense_sync_step", "sfb_get_factors", "sfb_get_stats",
            "sfb_get_status", "sfb_strerror", "sfb_last_cuda_error", "sfb_destroy", "sfb_prox_columns_noalloc",
            "sfb_selftest_wait_timeout", "sfb_set_row_shard", "sfb_forward_partials", "sfb_finish_factors",
-           "sfb_replay_update")
+           "sfb_replay_update", "sfb_refresh_operands")
 NOALLOC_MAX_COLS = 16384
 
 
@@ -81,6 +81,7 @@ def lib() -> ctypes.CDLL:
         L.sfb_forward_partials.argtypes = [vp, vp, vp, vp]
         L.sfb_finish_factors.argtypes = [vp, vp, i32]
         L.sfb_replay_update.argtypes = [vp]
+        L.sfb_refresh_operands.argtypes = [vp]
         for name in EXPORTS:
             if name != "sfb_strerror":
                 getattr(L, name).restype = ctypes.c_int
@@ -149,8 +150,11 @@ class Context:
     def sfb_apply_update(self):
         self._ck(lib().sfb_apply_update(self._h), "sfb_apply_update")
 
+    def sfb_refresh_operands(self):
+        self._ck(lib().sfb_refresh_operands(self._h), "sfb_refresh_operands")
+
     def sfb_replay_update(self):
-        self._ck(lib().sfb_replay_update(self._h), "sfb_replay_update")
+        self._ck(lib().sfb_replay_update(self._h), "sfb_replay_update", "sfb_refresh_operands")
 
     def sfb_step(self, X, Y=None, labels=None):
         self._ck(lib().sfb_step(self._h, _ptr(X), _ptr(Y), _ptr(labels)), "sfb_step")

@@ -353,6 +353,13 @@ extern "C" int sfb_apply_update(sfb_ctx* ctx) {
   return SFB_OK;
 }
 
+extern "C" int sfb_refresh_operands(sfb_ctx* ctx) {
+  if (!ctx) return SFB_ERR_ARG;
+  if (ctx->committed != 0 || ctx->partials_ready) return SFB_ERR_STATE;      // not in the middle of a step
+  if (ctx->cfg.precision != SFB_PREC_BF16) return SFB_OK;                     // fp32 mode reads W itself
+  return tc_refresh_operands(ctx);
+}
+
 extern "C" int sfb_replay_update(sfb_ctx* ctx) {
   if (!ctx) return SFB_ERR_ARG;
   if (ctx->stats.steps < 1 || ctx->committed != 0 || ctx->partials_ready) return SFB_ERR_STATE;

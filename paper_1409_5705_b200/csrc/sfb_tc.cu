@@ -667,8 +667,15 @@ int tc_init(sfb_ctx* ctx) {
     return SFB_OK;
   }
   // bf16 copy of W for the forward product; afterwards the update's epilogue keeps it current
+  return tc_refresh_operands(ctx);
+}
+
+int tc_refresh_operands(sfb_ctx* ctx) {
+  const sfb_config& c = ctx->cfg;
+  if (c.model != SFB_MLR) return SFB_OK;          // the split copies of W are rebuilt by the first factors call of a step
+  const TcState* st = static_cast<const TcState*>(ctx->tc);
   convert_rows_kernel<<<st->sms * 8, 256, 0, ctx->stream>>>(ctx->W, c.rows, c.cols, ctx->at<__nv_bfloat16>(ctx->lay.Wb),
-                                                        ctx->lay.colsb);
+                                                            ctx->lay.colsb);
   count_launch();
   CKC(cudaGetLastError());
   return SFB_OK;

@@ -11,6 +11,8 @@ namespace sfb {
 void tc_extend_layout(const sfb_config& c, Layout& L, size_t& off);
 int tc_init(sfb_ctx* ctx);
 void tc_destroy(sfb_ctx* ctx);
+// Rebuilds the bf16 operand copy of W from the caller's fp32 W (MLR; the other models rebuild theirs every step).
+int tc_refresh_operands(sfb_ctx* ctx);
 int tc_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float* Y, const int32_t* labels);
 // Row-sharded MLR: logits and softmax partials of all K samples against this context's rows; then the factors from
 // the partials of all shards.

@@ -82,3 +82,75 @@ def test_a_planted_mistake_is_caught_by_some_pin(name, monkeypatch):
     attr, fn = MUTATIONS[name]
     monkeypatch.setattr(O, attr, fn)
     assert _caught(), f"no pin noticed: {name}"
+
+
+# ----------------------------------------------------------------------------------------------------------
+# The same for the SDCA oracle: mistakes planted in oracle/sdca_oracle.py must fail a pin of test_sdca_pins.py
+# ----------------------------------------------------------------------------------------------------------
+from oracle import sdca_oracle as D   # noqa: E402
+import test_sdca_pins as TS           # noqa: E402
+
+SDCA_PINS = [TS.test_coordinate_minimiser_is_the_constrained_minimum, TS.test_two_classes_reduce_to_one_scalar_equation,
+             TS.test_without_the_quadratic_term_the_minimiser_is_the_softmax,
+             TS.test_weak_duality_for_any_feasible_dual_state,
+             TS.test_dual_objective_never_increases_and_W_tracks_the_dual_state,
+             TS.test_single_sample_step_is_the_exact_coordinate_minimum_of_the_dual,
+             TS.test_sweeps_close_the_gap_and_reach_the_primal_optimum,
+             TS.test_hand_worked_case_two_classes_one_sample]
+DORIG = {n: getattr(D, n) for n in ("coordinate_minimiser", "sdca_factors", "sdca_step", "w_from_dual", "l2mlr_dual")}
+
+
+def _sdca_caught():
+    for pin in SDCA_PINS:
+        try:
+            pin()
+        except Exception:
+            return True
+    return False
+
+
+def _factors_sign(W, X, y, Q_rows, lam, N):
+    U, V = DORIG["sdca_factors"](W, X, y, Q_rows, lam, N)
+    return -U, V
+
+
+def _factors_kappa_without_norm(W, X, y, Q_rows, lam, N):
+    X = np.asarray(X, dtype=np.float64)
+    Z = X @ np.asarray(W, dtype=np.float64).T
+    U = np.stack([DORIG["coordinate_minimiser"](Z[i], Q_rows[i], 1.0 / (lam * N)) - Q_rows[i] for i in range(len(X))])
+    return U, X.copy()
+
+
+def _step_without_one_over_N(W, X, y, ids, Q, lam, gamma, workers=1):
+    W1, Q1, U, V = DORIG["sdca_step"](W, X, y, ids, Q, lam, gamma, workers)
+    return np.asarray(W, dtype=np.float64) - (gamma / lam) * (U.T @ V), Q1, U, V
+
+
+def _step_dual_not_damped(W, X, y, ids, Q, lam, gamma, workers=1):
+    W1, Q1, U, V = DORIG["sdca_step"](W, X, y, ids, Q, lam, gamma, workers)
+    Q2 = np.asarray(Q, dtype=np.float64).copy()
+    Q2[np.asarray(ids)] += U                                  # gamma forgotten on the dual side only
+    return W1, Q2, U, V
+
+
+SDCA_MUTATIONS = {
+    "sdca: du with the wrong sign": ("sdca_factors", _factors_sign),
+    "sdca: kappa without ||a||^2": ("sdca_factors", _factors_kappa_without_norm),
+    "sdca: quadratic term ignored (plain softmax)": ("coordinate_minimiser", lambda z, q_old, kappa, iters=200: DORIG["coordinate_minimiser"](z, q_old, 0.0)),
+    "sdca: q_old dropped from the right-hand side": ("coordinate_minimiser", lambda z, q_old, kappa, iters=200: DORIG["coordinate_minimiser"](z, np.zeros_like(q_old), kappa)),
+    "sdca: Z updated without 1/N": ("sdca_step", _step_without_one_over_N),
+    "sdca: dual state moved by the undamped change": ("sdca_step", _step_dual_not_damped),
+    "sdca: W = Z (1/lam dropped)": ("w_from_dual", lambda Q, A, y, lam: lam * DORIG["w_from_dual"](Q, A, y, lam)),
+    "sdca: conjugate with the wrong sign": ("l2mlr_dual", lambda Q, A, y, lam: DORIG["l2mlr_dual"](Q, A, y, lam) - 2 * float(np.where(np.asarray(Q) > 0, Q * np.log(np.where(np.asarray(Q) > 0, Q, 1.0)), 0.0).sum()) / len(y)),
+}
+
+
+def test_unmutated_sdca_oracle_passes_every_pin():
+    assert not _sdca_caught()
+
+
+@pytest.mark.parametrize("name", sorted(SDCA_MUTATIONS))
+def test_a_planted_sdca_mistake_is_caught_by_some_pin(name, monkeypatch):
+    attr, fn = SDCA_MUTATIONS[name]
+    monkeypatch.setattr(D, attr, fn)
+    assert _sdca_caught(), f"no pin noticed: {name}"
