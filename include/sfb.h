@@ -32,7 +32,9 @@ extern "C" {
 
 typedef struct sfb_ctx sfb_ctx;
 
-enum sfb_model { SFB_MLR = 0, SFB_DML = 1, SFB_SC = 2 };
+/* SFB_L2MLR: multiclass logistic regression with the regulariser lam/2 ||W||_F^2, learnt by stochastic dual coordinate
+ * ascent (Section 2.1 "Stochastic DCA"; the fourth model of Section 6).  See sfb_sdca_compute_factors. */
+enum sfb_model { SFB_MLR = 0, SFB_DML = 1, SFB_SC = 2, SFB_L2MLR = 3 };
 
 /* Operand precision of the matrix products.  The master copy of W is fp32 in both modes.
  * SFB_PREC_BF16: tensor-core products on bf16 operands with fp32 accumulation.  MLR: forward and update
@@ -61,6 +63,7 @@ enum sfb_error {
 /* Bits of the device status word. */
 #define SFB_STATUS_LABEL_RANGE 0x1u
 #define SFB_STATUS_TIMEOUT     0x2u
+#define SFB_STATUS_SAMPLE_RANGE 0x4u   /* SDCA: a sample id outside [0, sdca_n) was skipped */
 
 typedef struct sfb_config {
   int32_t model;          /* enum sfb_model                                                            */
@@ -75,6 +78,8 @@ typedef struct sfb_config {
   float   sc_lipschitz;   /* step is 1/L; <= 0: the library estimates L = ||W||_2^2 by 50 power
                              iterations at the start of every step                                     */
   int32_t sc_prox;        /* 0 none | 1 rescale columns of norm > 1 to norm 1 (Figure 3)               */
+  float   sdca_lambda;    /* SFB_L2MLR: weight lam of the regulariser h(W) = lam/2 ||W||_F^2 (> 0)    */
+  int64_t sdca_n;         /* SFB_L2MLR: N, the number of training samples (rows of the dual state)     */
   void*   stream;         /* cudaStream_t                                                              */
 } sfb_config;
 
@@ -113,6 +118,34 @@ int sfb_init(const sfb_config* cfg, float* W_dev, void* workspace_dev, size_t wo
  * its own): after such a write call sfb_refresh_operands, or the next forward product runs on the stale copy. */
 int sfb_compute_factors(sfb_ctx* ctx, int32_t worker, const float* X_dev, const float* Y_dev,
                         const int32_t* labels_dev);
+
+/* ---- l2-regularised MLR by stochastic dual coordinate ascent (model SFB_L2MLR) ------------------------------------
+ * Section 2.1 "Stochastic DCA": with the dual matrix U = [u_1 .. u_N], Z = 1/N U A^T and W = grad h^*(Z) = Z / lam, a
+ * step picks samples i, finds the change du_i that minimises the dual (D) over u_i with the other dual vectors fixed,
+ * and applies  u_i <- u_i - du_i,  Z <- Z - 1/N du_i a_i^T,  W <- grad h^*(Z).  The sufficient factors of the step are
+ * (du_i, a_i) (Section 3: "the above procedure is instead used to broadcast SFs for the auxiliary matrix Z").
+ *
+ * Dual state: the caller owns Q_dev [sdca_n x rows] fp32 with rows q_i = e_{y_i} - u_i, points of the probability
+ * simplex (for the multiclass logistic loss f_i^*(-u_i) = sum_j q_ij log q_ij); q_i = e_{y_i} (u_i = 0) with W = 0 is
+ * the usual start.  The caller keeps W_dev = 1/(lam N) sum_i (e_{y_i} - q_i) a_i^T consistent with it at set-up; the
+ * steps keep it so.
+ *
+ * sfb_sdca_compute_factors: for every sample of the worker (or of all workers, worker = -1), against the same W:
+ *     z = W a_i,  kappa = ||a_i||^2 / (lam N),  q_new = argmin over the simplex of
+ *         sum_j q_j log q_j - q.(z + kappa q_old) + kappa/2 ||q||^2
+ *     (stationarity: log q_j + kappa q_j = z_j + kappa q_old_j - nu, sum_j q_j = 1; solved by a safeguarded Newton
+ *     iteration on nu with a Newton solve per class), du_i = q_new - q_old, and, averaging the K changes of a
+ *     mini-batch with the weight eta of the config (Section 3, "Mini-batch proximal SGD/SDCA": 1/K sum u_i v_i^T, so
+ *     eta = 1/K; eta = 1 with K = 1 is the single-sample step),   q_i <- q_old + eta * du_i   in Q_dev.
+ *     sample_ids_dev [B or K] int32: the rows of Q_dev of the samples, distinct within a step; an id outside
+ *     [0, sdca_n) sets SFB_STATUS_SAMPLE_RANGE and contributes nothing.  labels_dev: class ids.
+ * sfb_gather_factors, then sfb_apply_update:   W <- W - eta/(lam N) * sum_i du_i a_i^T   (the fused update pass).
+ * sfb_sdca_step = the three calls for all K samples.  sfb_compute_factors / sfb_step on such a context and these
+ * calls on any other return SFB_ERR_UNSUPPORTED; SFB_ERR_STATE before sfb_sdca_set_dual. */
+int sfb_sdca_set_dual(sfb_ctx* ctx, float* Q_dev, int64_t n_samples);
+int sfb_sdca_compute_factors(sfb_ctx* ctx, int32_t worker, const float* X_dev, const int32_t* labels_dev,
+                             const int32_t* sample_ids_dev);
+int sfb_sdca_step(sfb_ctx* ctx, const float* X_dev, const int32_t* labels_dev, const int32_t* sample_ids_dev);
 
 /* The broadcast of Section 3 as an on-device gather: after it, U [K x rows] and V [K x cols] of all P workers
  * sit in one buffer in the operand layout of the update.  Fails with SFB_ERR_STATE unless every worker has

@@ -11,15 +11,16 @@ import os
 
 from .build import LIB, build
 
-MLR, DML, SC = 0, 1, 2
+MLR, DML, SC, L2MLR = 0, 1, 2, 3
 PREC_BF16, PREC_FP32 = 0, 1
-STATUS_LABEL_RANGE, STATUS_TIMEOUT = 0x1, 0x2
+STATUS_LABEL_RANGE, STATUS_TIMEOUT, STATUS_SAMPLE_RANGE = 0x1, 0x2, 0x4
 
 EXPORTS = ("sfb_workspace_bytes", "sfb_init", "sfb_compute_factors", "sfb_gather_factors", "sfb_apply_update",
            "sfb_step", "sfb_step_host", "sfb_dense_sync_step", "sfb_get_factors", "sfb_get_stats",
            "sfb_get_status", "sfb_strerror", "sfb_last_cuda_error", "sfb_destroy", "sfb_prox_columns_noalloc",
            "sfb_selftest_wait_timeout", "sfb_set_row_shard", "sfb_forward_partials", "sfb_finish_factors",
-           "sfb_replay_update", "sfb_refresh_operands")
+           "sfb_replay_update", "sfb_refresh_operands", "sfb_sdca_set_dual", "sfb_sdca_compute_factors",
+           "sfb_sdca_step")
 NOALLOC_MAX_COLS = 16384
 
 
@@ -28,7 +29,7 @@ class sfb_config(ctypes.Structure):
                 ("cols", ctypes.c_int64), ("workers", ctypes.c_int32), ("batch", ctypes.c_int32),
                 ("eta", ctypes.c_float), ("dml_margin", ctypes.c_float), ("sc_lambda", ctypes.c_float),
                 ("sc_ista_iters", ctypes.c_int32), ("sc_lipschitz", ctypes.c_float), ("sc_prox", ctypes.c_int32),
-                ("stream", ctypes.c_void_p)]
+                ("sdca_lambda", ctypes.c_float), ("sdca_n", ctypes.c_int64), ("stream", ctypes.c_void_p)]
 
 
 class sfb_stats(ctypes.Structure):
@@ -82,6 +83,9 @@ def lib() -> ctypes.CDLL:
         L.sfb_finish_factors.argtypes = [vp, vp, i32]
         L.sfb_replay_update.argtypes = [vp]
         L.sfb_refresh_operands.argtypes = [vp]
+        L.sfb_sdca_set_dual.argtypes = [vp, vp, i64]
+        L.sfb_sdca_compute_factors.argtypes = [vp, i32, vp, vp, vp]
+        L.sfb_sdca_step.argtypes = [vp, vp, vp, vp]
         for name in EXPORTS:
             if name != "sfb_strerror":
                 getattr(L, name).restype = ctypes.c_int
@@ -94,9 +98,9 @@ def strerror(code: int) -> str:
 
 
 def make_config(model, rows, cols, workers, batch, eta, precision=PREC_FP32, dml_margin=1.0, sc_lambda=0.1,
-                sc_ista_iters=20, sc_lipschitz=0.0, sc_prox=0, stream=0) -> sfb_config:
+                sc_ista_iters=20, sc_lipschitz=0.0, sc_prox=0, stream=0, sdca_lambda=0.0, sdca_n=0) -> sfb_config:
     return sfb_config(model, precision, rows, cols, workers, batch, eta, dml_margin, sc_lambda, sc_ista_iters,
-                      sc_lipschitz, sc_prox, stream)
+                      sc_lipschitz, sc_prox, sdca_lambda, sdca_n, stream)
 
 
 def sfb_workspace_bytes(cfg: sfb_config) -> int:
@@ -150,11 +154,24 @@ class Context:
     def sfb_apply_update(self):
         self._ck(lib().sfb_apply_update(self._h), "sfb_apply_update")
 
+    def sfb_sdca_set_dual(self, Q):
+        """Q: fp32 CUDA tensor [sdca_n, rows], the dual state (kept alive by the caller; updated in place)."""
+        self._dual = Q
+        self._ck(lib().sfb_sdca_set_dual(self._h, _ptr(Q), Q.shape[0]), "sfb_sdca_set_dual")
+
+    def sfb_sdca_compute_factors(self, worker, X, labels, sample_ids):
+        self._ck(lib().sfb_sdca_compute_factors(self._h, worker, _ptr(X), _ptr(labels), _ptr(sample_ids)),
+                 "sfb_sdca_compute_factors")
+
+    def sfb_sdca_step(self, X, labels, sample_ids):
+        self._ck(lib().sfb_sdca_step(self._h, _ptr(X), _ptr(labels), _ptr(sample_ids)), "sfb_sdca_step")
+
     def sfb_refresh_operands(self):
         self._ck(lib().sfb_refresh_operands(self._h), "sfb_refresh_operands")
 
     def sfb_replay_update(self):
-        self._ck(lib().sfb_replay_update(self._h), "sfb_replay_update", "sfb_refresh_operands")
+        self._ck(lib().sfb_replay_update(self._h), "sfb_replay_update", "sfb_refresh_operands", "sfb_sdca_set_dual", "sfb_sdca_compute_factors",
+           "sfb_sdca_step")
 
     def sfb_step(self, X, Y=None, labels=None):
         self._ck(lib().sfb_step(self._h, _ptr(X), _ptr(Y), _ptr(labels)), "sfb_step")

@@ -24,7 +24,9 @@ int sm_count() {
 
 static size_t up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
-Layout make_layout(const sfb_config& c) {
+Layout make_layout(const sfb_config& cfg) {
+  sfb_config c = cfg;
+  if (c.model == SFB_L2MLR) c.model = SFB_MLR;        // same buffers: the factors differ, the products do not
   Layout L{};
   const size_t K = static_cast<size_t>(c.workers) * c.batch;
   const size_t rows = c.rows, cols = c.cols;
@@ -70,7 +72,8 @@ static bool al16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) 
 
 static int check_config(const sfb_config* c) {
   if (!c) return SFB_ERR_ARG;
-  if (c->model < SFB_MLR || c->model > SFB_SC) return SFB_ERR_ARG;
+  if (c->model < SFB_MLR || c->model > SFB_L2MLR) return SFB_ERR_ARG;
+  if (c->model == SFB_L2MLR && (!(c->sdca_lambda > 0.f) || c->sdca_n < 1)) return SFB_ERR_ARG;
   if (c->precision != SFB_PREC_BF16 && c->precision != SFB_PREC_FP32) return SFB_ERR_ARG;
   if (c->rows <= 0 || c->cols <= 0 || c->workers <= 0 || c->batch <= 0) return SFB_ERR_ARG;
   if (c->workers > 64) return SFB_ERR_SHAPE;
@@ -109,6 +112,13 @@ extern "C" int sfb_init(const sfb_config* cfg, float* W_dev, void* workspace_dev
   sfb_ctx* ctx = new (std::nothrow) sfb_ctx();
   if (!ctx) return SFB_ERR_ARG;
   ctx->cfg = *cfg;
+  ctx->sdca = cfg->model == SFB_L2MLR;
+  if (ctx->sdca) ctx->cfg.model = SFB_MLR;            // the products, buffers and the update are those of MLR
+  ctx->dualQ = nullptr;
+  ctx->dual_n = 0;
+  ctx->step = ctx->sdca ? static_cast<float>(static_cast<double>(cfg->eta) / (static_cast<double>(cfg->sdca_lambda) *
+                                                                            static_cast<double>(cfg->sdca_n)))
+                        : cfg->eta;
   ctx->lay = lay;
   ctx->W = W_dev;
   ctx->ws = static_cast<char*>(workspace_dev);
@@ -195,7 +205,7 @@ static int factors_fp32(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, co
 static int update_fp32(sfb_ctx* ctx) {
   const sfb_config& c = ctx->cfg;
   EpiArgs e{};
-  e.C = ctx->W; e.ldc = c.cols; e.alpha = -c.eta;
+  e.C = ctx->W; e.ldc = c.cols; e.alpha = -ctx->step;
   CK(sgemm(ctx->stream, false, false, EPI_RMW, c.rows, c.cols, ctx->K, ctx->at<float>(ctx->lay.U), c.rows,
            ctx->at<float>(ctx->lay.V), c.cols, e));
   return SFB_OK;
@@ -215,6 +225,7 @@ extern "C" int sfb_compute_factors(sfb_ctx* ctx, int32_t worker, const float* X_
   int rc = check_inputs(ctx, X_dev, Y_dev, labels_dev);
   if (rc) return rc;
   const sfb_config& c = ctx->cfg;
+  if (ctx->sdca) return SFB_ERR_UNSUPPORTED;          // the dual step needs the samples' ids: sfb_sdca_compute_factors
   if (worker < -1 || worker >= c.workers) return SFB_ERR_SHAPE;
   const int64_t off = worker < 0 ? 0 : static_cast<int64_t>(worker) * c.batch;
   const int64_t n = worker < 0 ? ctx->K : c.batch;
@@ -242,7 +253,7 @@ extern "C" int sfb_compute_factors(sfb_ctx* ctx, int32_t worker, const float* X_
 // ---------------------------------------------------------------------------------------------------------
 extern "C" int sfb_set_row_shard(sfb_ctx* ctx, int64_t row_offset, int64_t global_rows) {
   if (!ctx) return SFB_ERR_ARG;
-  if (ctx->cfg.model != SFB_MLR) return SFB_ERR_UNSUPPORTED;
+  if (ctx->cfg.model != SFB_MLR || ctx->sdca) return SFB_ERR_UNSUPPORTED;
   if (row_offset < 0 || global_rows < row_offset + ctx->cfg.rows || global_rows > (1LL << 31) - 1) return SFB_ERR_SHAPE;
   if (ctx->committed != 0 || ctx->partials_ready) return SFB_ERR_STATE;
   ctx->row_offset = row_offset;
@@ -253,7 +264,7 @@ extern "C" int sfb_set_row_shard(sfb_ctx* ctx, int64_t row_offset, int64_t globa
 extern "C" int sfb_forward_partials(sfb_ctx* ctx, const float* X_dev, const int32_t* labels_dev, float* partials_dev) {
   int rc = check_inputs(ctx, X_dev, nullptr, labels_dev);
   if (rc) return rc;
-  if (ctx->cfg.model != SFB_MLR) return SFB_ERR_UNSUPPORTED;
+  if (ctx->cfg.model != SFB_MLR || ctx->sdca) return SFB_ERR_UNSUPPORTED;
   if (!partials_dev) return SFB_ERR_ARG;
   if (!al16(partials_dev)) return SFB_ERR_ALIGN;
   const sfb_config& c = ctx->cfg;
@@ -353,6 +364,63 @@ extern "C" int sfb_apply_update(sfb_ctx* ctx) {
   return SFB_OK;
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// l2-regularised MLR by stochastic dual coordinate ascent
+// ---------------------------------------------------------------------------------------------------------
+extern "C" int sfb_sdca_set_dual(sfb_ctx* ctx, float* Q_dev, int64_t n_samples) {
+  if (!ctx || !Q_dev) return SFB_ERR_ARG;
+  if (!ctx->sdca) return SFB_ERR_UNSUPPORTED;
+  if (n_samples != ctx->cfg.sdca_n) return SFB_ERR_SHAPE;
+  if (!al16(Q_dev)) return SFB_ERR_ALIGN;
+  ctx->dualQ = Q_dev;
+  ctx->dual_n = n_samples;
+  return SFB_OK;
+}
+
+extern "C" int sfb_sdca_compute_factors(sfb_ctx* ctx, int32_t worker, const float* X_dev, const int32_t* labels_dev,
+                                        const int32_t* sample_ids_dev) {
+  if (!ctx || !X_dev || !labels_dev || !sample_ids_dev) return SFB_ERR_ARG;
+  if (!ctx->sdca) return SFB_ERR_UNSUPPORTED;
+  if (!ctx->dualQ) return SFB_ERR_STATE;
+  if (!al16(X_dev)) return SFB_ERR_ALIGN;
+  const sfb_config& c = ctx->cfg;
+  if (worker < -1 || worker >= c.workers) return SFB_ERR_SHAPE;
+  const int64_t off = worker < 0 ? 0 : static_cast<int64_t>(worker) * c.batch;
+  const int64_t n = worker < 0 ? ctx->K : c.batch;
+  if (ctx->committed == 0) CK(cudaEventRecord(ctx->ev[0], ctx->stream));
+  const float inv_lam_n = static_cast<float>(1.0 / (static_cast<double>(c.sdca_lambda) * static_cast<double>(c.sdca_n)));
+  uint32_t* status = ctx->at<uint32_t>(ctx->lay.status);
+  float* loss = ctx->at<float>(ctx->lay.loss) + off;
+  if (c.precision == SFB_PREC_FP32) {
+    float* V = ctx->at<float>(ctx->lay.V) + off * c.cols;
+    float* U = ctx->at<float>(ctx->lay.U) + off * c.rows;
+    CK(pack_copy(ctx->stream, V, X_dev, nullptr, n * c.cols));                                        // v = a_i
+    EpiArgs e{};
+    e.C = U; e.ldc = c.rows;
+    CK(sgemm(ctx->stream, true, true, EPI_STORE, n, c.rows, c.cols, V, c.cols, ctx->W, c.cols, e));   // z_i = W a_i
+    ctx->stats.flops += 2.0 * n * c.rows * c.cols;
+    CK(sdca_dual_rows(ctx->stream, U, n, c.rows, c.rows, X_dev, c.cols, labels_dev, sample_ids_dev, ctx->dualQ, ctx->dual_n,
+                      inv_lam_n, c.eta, nullptr, loss, status));                                      // u_i = du_i
+  } else {
+    const int rc = tc_sdca_factors(ctx, off, n, X_dev, labels_dev, sample_ids_dev, inv_lam_n);
+    if (rc) return rc;
+  }
+  const uint64_t all = c.workers == 64 ? ~0ull : ((1ull << c.workers) - 1);
+  ctx->committed |= worker < 0 ? all : (1ull << worker);
+  ctx->gathered = false;
+  return SFB_OK;
+}
+
+extern "C" int sfb_sdca_step(sfb_ctx* ctx, const float* X_dev, const int32_t* labels_dev, const int32_t* sample_ids_dev) {
+  if (!ctx) return SFB_ERR_ARG;
+  ctx->committed = 0;
+  int rc = sfb_sdca_compute_factors(ctx, -1, X_dev, labels_dev, sample_ids_dev);
+  if (rc) return rc;
+  rc = sfb_gather_factors(ctx);
+  if (rc) return rc;
+  return sfb_apply_update(ctx);
+}
+
 extern "C" int sfb_refresh_operands(sfb_ctx* ctx) {
   if (!ctx) return SFB_ERR_ARG;
   if (ctx->committed != 0 || ctx->partials_ready) return SFB_ERR_STATE;      // not in the middle of a step
@@ -387,6 +455,7 @@ extern "C" int sfb_step(sfb_ctx* ctx, const float* X_dev, const float* Y_dev, co
 extern "C" int sfb_step_host(sfb_ctx* ctx, const float* X_host, const float* Y_host, const int32_t* labels_host,
                              float* loss_out, uint32_t* status_out) {
   if (!ctx || !X_host) return SFB_ERR_ARG;
+  if (ctx->sdca) return SFB_ERR_UNSUPPORTED;
   const sfb_config& c = ctx->cfg;
   if (c.model == SFB_DML && (!Y_host || !labels_host)) return SFB_ERR_ARG;
   if (c.model == SFB_MLR && !labels_host) return SFB_ERR_ARG;

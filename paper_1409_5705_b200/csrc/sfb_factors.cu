@@ -173,6 +173,103 @@ __global__ void __launch_bounds__(NTHREADS) mlr_shard_finish_kernel(float* __res
   }
 }
 
+// SDCA for l2-regularised multiclass logistic regression (Section 2.1, "Stochastic DCA").  One block per sample:
+// the new dual row q minimises  sum_j q_j log q_j - q.(z + kappa q_old) + kappa/2 ||q||^2  over the simplex, kappa =
+// ||x||^2 / (lam N).  Stationarity: log q_j + kappa q_j = t_j - nu with t = z + kappa q_old, and nu such that the q_j sum
+// to 1; nu lies in [lse(t) - kappa, lse(t)].
+// q_j(nu): Newton on y = log q for  y + kappa e^y = c  (increasing and convex in y, so the iteration is monotone from
+// the right of the root, where it starts).
+__device__ __forceinline__ float sdca_coordinate(float c, float kappa) {
+  if (kappa <= 0.f) return expf(c);
+  float y = c;                                       // y + kappa e^y - c = kappa e^c >= 0 here: right of the root
+  if (c > 0.f) y = fminf(c, logf((c + 1.f) / kappa));
+#pragma unroll 1
+  for (int it = 0; it < 24; ++it) {
+    const float e = kappa * expf(y);
+    const float d = (y + e - c) / (1.f + e);
+    y -= d;
+    if (fabsf(d) <= 1e-7f * fmaxf(1.f, fabsf(y))) break;
+  }
+  return expf(y);
+}
+
+template <int NTHREADS>
+__global__ void __launch_bounds__(NTHREADS) sdca_dual_kernel(float* __restrict__ Z, int64_t rows, int64_t ldz,
+                                                             const float* __restrict__ X, int64_t cols,
+                                                             const int32_t* __restrict__ labels,
+                                                             const int32_t* __restrict__ ids, float* __restrict__ Q,
+                                                             int64_t n_samples, float inv_lam_n, float gamma,
+                                                             float* __restrict__ coef, float* __restrict__ loss,
+                                                             uint32_t* status) {
+  __shared__ float sh[32];
+  const int64_t i = blockIdx.x;
+  float* z = Z + i * ldz;
+  const int64_t id = ids[i];
+  const int32_t y = labels[i];
+  const bool ok = id >= 0 && id < n_samples && y >= 0 && y < rows;
+  if (!ok) {                                         // uniform over the block: skip the sample, contribute nothing
+    if (threadIdx.x == 0) {
+      atomicOr(status, (id >= 0 && id < n_samples) ? SFB_STATUS_LABEL_RANGE : SFB_STATUS_SAMPLE_RANGE);
+      if (coef) coef[i] = 0.f;
+      loss[i] = 0.f;
+    }
+    for (int64_t j = threadIdx.x; j < rows; j += NTHREADS) z[j] = 0.f;
+    return;
+  }
+  float* q = Q + id * rows;
+  const float* x = X + i * cols;
+  float ss = 0.f;
+  for (int64_t d = threadIdx.x; d < cols; d += NTHREADS) ss = fmaf(x[d], x[d], ss);
+  const float kappa = block_sum<NTHREADS>(ss, sh) * inv_lam_n;
+  // lse(t) and, for the read-out, lse(z)
+  float m = -INFINITY, mz = -INFINITY;
+  for (int64_t j = threadIdx.x; j < rows; j += NTHREADS) {
+    m = fmaxf(m, fmaf(kappa, q[j], z[j]));
+    mz = fmaxf(mz, z[j]);
+  }
+  m = block_max<NTHREADS>(m, sh);
+  mz = block_max<NTHREADS>(mz, sh);
+  float s = 0.f, sz = 0.f;
+  for (int64_t j = threadIdx.x; j < rows; j += NTHREADS) {
+    s += expf(fmaf(kappa, q[j], z[j]) - m);
+    sz += expf(z[j] - mz);
+  }
+  s = block_sum<NTHREADS>(s, sh);
+  sz = block_sum<NTHREADS>(sz, sh);
+  const float lse = m + logf(s);
+  if (threadIdx.x == 0) loss[i] = (mz + logf(sz)) - z[y];        // the sample's logistic loss at the W of this step
+  // safeguarded Newton on nu: G(nu) = sum_j q_j(nu) is decreasing and convex, G(lse - kappa) >= 1 >= G(lse)
+  float lo = lse - kappa, hi = lse, nu = lse;
+#pragma unroll 1
+  for (int it = 0; it < 12; ++it) {
+    float G = 0.f, Dv = 0.f;
+    for (int64_t j = threadIdx.x; j < rows; j += NTHREADS) {
+      const float qj = sdca_coordinate(fmaf(kappa, q[j], z[j]) - nu, kappa);
+      G += qj;
+      Dv += qj / fmaf(kappa, qj, 1.f);
+    }
+    G = block_sum<NTHREADS>(G, sh);
+    Dv = block_sum<NTHREADS>(Dv, sh);
+    const float g = G - 1.f;
+    if (fabsf(g) <= 2e-7f) break;                    // uniform over the block: every thread holds the same sums
+    if (g > 0.f) lo = fmaxf(lo, nu); else hi = fminf(hi, nu);
+    float next = nu + g / Dv;
+    if (!(next > lo && next < hi)) next = 0.5f * (lo + hi);
+    nu = next;
+  }
+  float S = 0.f;
+  for (int64_t j = threadIdx.x; j < rows; j += NTHREADS) S += sdca_coordinate(fmaf(kappa, q[j], z[j]) - nu, kappa);
+  S = block_sum<NTHREADS>(S, sh);
+  const float invS = 1.f / S;
+  for (int64_t j = threadIdx.x; j < rows; j += NTHREADS) {
+    const float qo = q[j];
+    const float du = sdca_coordinate(fmaf(kappa, qo, z[j]) - nu, kappa) * invS - qo;      // du = q_new - q_old
+    z[j] = du;
+    q[j] = fmaf(gamma, du, qo);
+    if (coef && j == y) coef[i] = -du;
+  }
+}
+
 // One block per pair: q = ||z||^2; similar: u = 2z; dissimilar: u = -2z if q < margin else 0 (Section 2, DML).
 template <int NTHREADS>
 __global__ void __launch_bounds__(NTHREADS) dml_scale_kernel(float* __restrict__ Z, int64_t rows, int64_t ld,
@@ -398,6 +495,16 @@ cudaError_t mlr_shard_finish(cudaStream_t s, float* Z, int64_t nsamp, int64_t ro
   if (nsamp <= 0) return cudaSuccess;
   mlr_shard_finish_kernel<512><<<static_cast<unsigned>(nsamp), 512, 0, s>>>(
       Z, rows, ldz, labels, row_off, reinterpret_cast<const float4*>(parts), shards, nsamp, loss, status);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t sdca_dual_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows, int64_t ldz, const float* X, int64_t cols,
+                           const int32_t* labels, const int32_t* ids, float* Q, int64_t n_samples, float inv_lam_n,
+                           float gamma, float* coef, float* loss, uint32_t* status) {
+  if (nsamp <= 0) return cudaSuccess;
+  sdca_dual_kernel<512><<<static_cast<unsigned>(nsamp), 512, 0, s>>>(Z, rows, ldz, X, cols, labels, ids, Q, n_samples,
+                                                                  inv_lam_n, gamma, coef, loss, status);
   count_launch();
   return cudaGetLastError();
 }

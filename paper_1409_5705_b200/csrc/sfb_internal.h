@@ -58,6 +58,10 @@ struct sfb_ctx {
   int64_t row_offset;                 // row-sharded MLR: this context's W holds rows [row_offset, row_offset + rows)
   int64_t global_rows;                //   of a matrix with global_rows rows (class ids are global); 0, rows when unsharded
   bool partials_ready;                // sfb_forward_partials has run since the last update
+  bool sdca;                          // SFB_L2MLR: the factors are dual changes; cfg.model is kept as SFB_MLR internally
+  float* dualQ;                       // SDCA dual state [dual_n x rows], caller-owned
+  int64_t dual_n;
+  float step;                         // multiplier of sum u v^T in the update: eta, or eta / (lam N) for SDCA
   uint64_t committed;                 // bit p set: worker p has written its factors since the last update
   bool gathered;
   int last_cuda;
@@ -102,6 +106,12 @@ cudaError_t mlr_shard_partials(cudaStream_t s, const float* Z, int64_t nsamp, in
                                const int32_t* labels, int64_t row_off, float* part);
 cudaError_t mlr_shard_finish(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows, int64_t ldz, const int32_t* labels,
                              int64_t row_off, const float* parts, int shards, float* loss, uint32_t* status);
+// SDCA (l2-regularised MLR): per sample, from its logits z (row of Z, overwritten with du), its dual row of Q (advanced
+// by gamma * du) and its features x: the change of the dual vector that minimises the dual objective.  coef (may be
+// null) receives -du at the label entry.
+cudaError_t sdca_dual_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows, int64_t ldz, const float* X, int64_t cols,
+                           const int32_t* labels, const int32_t* ids, float* Q, int64_t n_samples, float inv_lam_n,
+                           float gamma, float* coef, float* loss, uint32_t* status);
 cudaError_t dml_scale_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows, int64_t ld,
                            const int32_t* similar, float margin);
 cudaError_t mean_of(cudaStream_t s, const float* v, int64_t n, float* out);

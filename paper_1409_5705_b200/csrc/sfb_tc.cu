@@ -515,6 +515,9 @@ __global__ void __launch_bounds__(256) mlr_shard_finish_tc_kernel(const float4* 
 // contiguous).  The factor is u_i = p_i - onehot(y_i); its label entry u_iy = p_iy - 1 is left out of the bf16
 // operand and applied to W in fp32 by label_rows_kernel, because bf16 cannot hold it when p_iy is close to 1
 // (spacing 2^-8 next to 1) and a rounded p_iy with an exact -1 would not cancel.
+// PLAIN: the values of Z themselves instead of exp(z - lse) (the dual changes of the SDCA step), same layout and
+// the same zero at the label entry.
+template <bool PLAIN>
 __global__ void __launch_bounds__(256) mlr_emit_ut_kernel(const float* __restrict__ Z, int64_t ldz, int64_t rows,
                                                           const float* __restrict__ lse, int64_t off, int64_t n,
                                                           const int32_t* __restrict__ labels,
@@ -529,7 +532,7 @@ __global__ void __launch_bounds__(256) mlr_emit_ut_kernel(const float* __restric
     const int i = idx / 16, rq = (idx % 16) * 4;
     if (i0 + i >= n) continue;
     const int64_t s = off + i0 + i;
-    const float l = lse[s];
+    const float l = PLAIN ? 0.f : lse[s];
     const int64_t yrel = static_cast<int64_t>(labels[i0 + i]) - (r0 + rq);     // label row relative to this quad
     const float* zp = Z + s * ldz + r0 + rq;
     float z[4] = {0.f, 0.f, 0.f, 0.f};
@@ -542,7 +545,7 @@ __global__ void __launch_bounds__(256) mlr_emit_ut_kernel(const float* __restric
     }
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      tile[i][rq + k] = k == yrel ? 0.f : __expf(z[k] - l);
+      tile[i][rq + k] = k == yrel ? 0.f : (PLAIN ? z[k] : __expf(z[k] - l));
     }
   }
   __syncthreads();
@@ -851,8 +854,30 @@ int tc_finish_factors(sfb_ctx* ctx, const float* parts, int shards) {
       ctx->at<float>(L.V), ctx->at<float>(L.loss), ctx->at<float>(L.coef), ctx->at<uint32_t>(L.status));
   count_launch();
   dim3 egrid(static_cast<unsigned>((c.rows + 63) / 64), static_cast<unsigned>((K + 63) / 64));
-  mlr_emit_ut_kernel<<<egrid, 256, 0, ctx->stream>>>(ctx->at<float>(L.ZT), round_up(c.rows, 32), c.rows, ctx->at<float>(L.V), 0, K,
+  mlr_emit_ut_kernel<false><<<egrid, 256, 0, ctx->stream>>>(ctx->at<float>(L.ZT), round_up(c.rows, 32), c.rows, ctx->at<float>(L.V), 0, K,
                                                      ctx->at<int32_t>(L.labels), ctx->at<__nv_bfloat16>(L.UT), L.Kp);
+  count_launch();
+  CKC(cudaGetLastError());
+  return SFB_OK;
+}
+
+// SDCA factors in bf16 mode: logits by the forward product, the dual changes in fp32 in place of the logits, then the
+// bf16 operand U^T = du (0 at the label entry, which goes to W in fp32 through coef, as for MLR).
+int tc_sdca_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const int32_t* labels, const int32_t* ids,
+                    float inv_lam_n) {
+  const sfb_config& c = ctx->cfg;
+  const Layout& L = ctx->lay;
+  const int64_t rows = c.rows;
+  const int64_t ldz = round_up(rows, 32);
+  float* Z = ctx->at<float>(L.ZT);
+  int tiles_n = 0;
+  const int rc = mlr_forward(ctx, off, n, X, labels, &tiles_n);
+  if (rc) return rc;
+  CKC(sdca_dual_rows(ctx->stream, Z + off * ldz, n, rows, ldz, X, c.cols, labels, ids, ctx->dualQ, ctx->dual_n, inv_lam_n,
+                     c.eta, ctx->at<float>(L.coef) + off, ctx->at<float>(L.loss) + off, ctx->at<uint32_t>(L.status)));
+  dim3 egrid(static_cast<unsigned>((rows + 63) / 64), static_cast<unsigned>((n + 63) / 64));
+  mlr_emit_ut_kernel<true><<<egrid, 256, 0, ctx->stream>>>(Z, ldz, rows, nullptr, off, n, labels, ctx->at<__nv_bfloat16>(L.UT),
+                                                           L.Kp);
   count_launch();
   CKC(cudaGetLastError());
   return SFB_OK;
@@ -874,7 +899,7 @@ int tc_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float
       ctx->at<uint32_t>(L.status));
   count_launch();
   dim3 egrid(static_cast<unsigned>((rows + 63) / 64), static_cast<unsigned>((n + 63) / 64));
-  mlr_emit_ut_kernel<<<egrid, 256, 0, ctx->stream>>>(Z, ldz, rows, lse, off, n, labels, ctx->at<__nv_bfloat16>(L.UT), L.Kp);
+  mlr_emit_ut_kernel<false><<<egrid, 256, 0, ctx->stream>>>(Z, ldz, rows, lse, off, n, labels, ctx->at<__nv_bfloat16>(L.UT), L.Kp);
   count_launch();
   CKC(cudaGetLastError());
   return SFB_OK;

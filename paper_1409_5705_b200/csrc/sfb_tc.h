@@ -18,6 +18,8 @@ int tc_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float
 // the partials of all shards.
 int tc_forward_partials(sfb_ctx* ctx, const float* X, const int32_t* labels, float* part_out);
 int tc_finish_factors(sfb_ctx* ctx, const float* parts, int shards);
+int tc_sdca_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const int32_t* labels, const int32_t* ids,
+                    float inv_lam_n);
 int tc_gather(sfb_ctx* ctx);
 int tc_update(sfb_ctx* ctx);
 int tc_get_factors(sfb_ctx* ctx, const void** U, const void** V, int32_t* dtype, int32_t* layout, int64_t* ldu,

@@ -404,7 +404,7 @@ int tc_update(sfb_ctx* ctx) {
   p.tilesM = static_cast<int32_t>((c.rows + 2 * UM - 1) / (2 * UM));
   p.tilesN = static_cast<int32_t>((c.cols + UN - 1) / UN);
   p.kseg = static_cast<int32_t>(L.Kp / UK);
-  p.alpha = -c.eta;
+  p.alpha = -ctx->step;
   p.status = ctx->at<uint32_t>(L.status);
   const int64_t tiles = static_cast<int64_t>(p.tilesM) * p.tilesN;
   const unsigned grid = 2u * static_cast<unsigned>(std::min<int64_t>(tiles, st->max_pairs));
@@ -427,7 +427,7 @@ int tc_update(sfb_ctx* ctx) {
   if ((c.cols + 1023) / 1024 > 65535) return SFB_ERR_SHAPE;
   dim3 lgrid(static_cast<unsigned>(ctx->K), static_cast<unsigned>((c.cols + 1023) / 1024));
   label_rows_kernel<<<lgrid, 256, 0, ctx->stream>>>(
-      ctx->W, c.rows, c.cols, ctx->at<float>(L.Xf), ctx->at<int32_t>(L.labels), ctx->at<float>(L.coef), static_cast<int>(ctx->K), c.eta,
+      ctx->W, c.rows, c.cols, ctx->at<float>(L.Xf), ctx->at<int32_t>(L.labels), ctx->at<float>(L.coef), static_cast<int>(ctx->K), ctx->step,
       ctx->at<__nv_bfloat16>(L.Wb), L.colsb);                // W[y_i] += eta * (1 - p_iy) * x_i
   count_launch();
   CKC(cudaGetLastError());
