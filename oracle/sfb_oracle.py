@@ -13,7 +13,8 @@ with u = d f_i / d (W a_i), v = a_i.  One step, for K = P*B samples drawn by P w
 
 Pins (tests/test_oracle_pins.py): finite differences of each loss, the independently coded dense gradient,
 the rank bound, closed forms (zero-init MLR, DML three-matmul form, orthonormal-dictionary ISTA), invariants
-(column sums conserved under MLR, ISTA objective non-increasing, prox idempotent), numpy's spectral norm.
+(column sums conserved under MLR, ISTA objective non-increasing, prox idempotent), numpy's spectral norm; the
+entry-wise proximal operators against scipy's scalar minimiser of their defining problem.
 Multi-step trajectories: parity unpinned beyond composing pinned single steps.
 """
 from __future__ import annotations
@@ -143,6 +144,33 @@ def prox_unit_columns(W):
 
 
 # ----------------------------------------------------------------------------------------------------------
+# Entry-wise proximal operators of proximal SGD (Section 2: the regulariser h "could be ... l1-, l2-, trace-norm";
+# Section 2.1: after W <- W - eta dW the operator prox_{eta h} is applied).  prox_{t h}(w) = argmin_v 1/2 (v - w)^2 + t h(v).
+#   h = lam ||W||_1           prox: shrink every entry towards 0 by t = eta*lam, entries within t of 0 become 0
+#   h = lam/2 ||W||_F^2       prox: every entry divided by 1 + t, t = eta*lam
+# (The trace norm needs the singular value decomposition of W and is not part of this step.)
+# ----------------------------------------------------------------------------------------------------------
+def prox_l1(W, t):
+    W = _f64(W)
+    return np.sign(W) * np.maximum(np.abs(W) - t, 0.0)
+
+
+def prox_l2sq(W, t):
+    return _f64(W) / (1.0 + t)
+
+
+def prox_entries(W, kind, t):
+    """kind: None, "l1" or "l2sq"."""
+    if kind is None:
+        return _f64(W)
+    if kind == "l1":
+        return prox_l1(W, t)
+    if kind == "l2sq":
+        return prox_l2sq(W, t)
+    raise ValueError(kind)
+
+
+# ----------------------------------------------------------------------------------------------------------
 # Broadcast, reconstruction, update (Section 3, Figure 1)
 # ----------------------------------------------------------------------------------------------------------
 def gather(factors_per_worker):
@@ -168,7 +196,7 @@ def worker_factors(model, W, X, Y=None, labels=None, margin=1.0, lam=0.1, L=None
 
 
 def sfb_step(model, W, X, Y=None, labels=None, workers=1, eta=1.0, margin=1.0, lam=0.1, L=None, iters=20,
-             prox=False, return_factors=False):
+             prox=False, return_factors=False, prox_kind=None, prox_weight=0.0):
     """One BSP step: every worker computes the SFs of its B samples against the same W, the SFs are
     gathered, every pair is reconstructed and applied, then the proximal operator (SC)."""
     K = X.shape[0]
@@ -181,6 +209,7 @@ def sfb_step(model, W, X, Y=None, labels=None, workers=1, eta=1.0, margin=1.0, l
                                          None if labels is None else labels[sl], margin, lam, L, iters))
     U, V = gather(per_worker)
     Wn = rank_k_update(W, U, V, eta)
+    Wn = prox_entries(Wn, prox_kind, eta * prox_weight)           # prox_{eta h} of an entry-wise regulariser, if any
     if prox:
         Wn = prox_unit_columns(Wn)
     return (Wn, U, V) if return_factors else Wn

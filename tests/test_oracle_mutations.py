@@ -15,7 +15,8 @@ def _pins():
              T.test_gather_is_worker_major_and_split_invariant, T.test_mlr_zero_init_closed_form,
              T.test_mlr_invariants, T.test_dml_three_matmul_closed_form, T.test_sc_closed_form_and_ista_properties,
              T.test_prox_properties, T.test_power_iteration_matches_spectral_norm,
-             T.test_comm_values_count_what_is_moved, T.test_sampled_mlr_helpers_match_the_plain_step]
+             T.test_comm_values_count_what_is_moved, T.test_sampled_mlr_helpers_match_the_plain_step,
+             T.test_entrywise_prox_operators_solve_their_defining_problem]
     pins += [lambda m=m: T.test_reconstruction_equals_dense_gradient_and_dense_sync(m) for m in (O.MLR, O.DML, O.SC)]
     return pins
 
@@ -54,7 +55,8 @@ def _dml_pair_sum(W, X, Y, similar, margin=1.0):
 
 
 ORIG = {n: getattr(O, n) for n in ("mlr_factors", "dml_factors", "soft_threshold", "rank_k_update",
-                                    "prox_unit_columns", "gather", "ista_codes", "lipschitz_power_iteration")}
+                                    "prox_unit_columns", "gather", "ista_codes", "lipschitz_power_iteration",
+                                    "prox_l1", "prox_l2sq")}
 
 MUTATIONS = {
     "mlr: onehot(y) not subtracted": ("mlr_factors", _mlr_without_onehot),
@@ -67,6 +69,8 @@ MUTATIONS = {
     "update: eta squared": ("rank_k_update", lambda W, U, V, eta: ORIG["rank_k_update"](W, U, V, eta * eta)),
     "update: U and V swapped": ("rank_k_update", lambda W, U, V, eta: ORIG["rank_k_update"](W, V, U, eta)),
     "prox: every column rescaled": ("prox_unit_columns", lambda W: np.asarray(W, dtype=np.float64) / np.sqrt((np.asarray(W, dtype=np.float64) ** 2).sum(axis=0))),
+    "prox l1: threshold halved": ("prox_l1", lambda W, t: ORIG["prox_l1"](W, 0.5 * t)),
+    "prox l2: divided by 1 + 2t": ("prox_l2sq", lambda W, t: ORIG["prox_l2sq"](W, 2 * t)),
     "gather: workers in reverse order": ("gather", lambda fs: ORIG["gather"](list(reversed(fs)))),
     "ista: one iteration too few": ("ista_codes", lambda W, X, lam, L, iters: ORIG["ista_codes"](W, X, lam, L, max(iters - 1, 0))),
     "power iteration: norm, not its square": ("lipschitz_power_iteration", lambda W, iters=50: float(np.sqrt(ORIG["lipschitz_power_iteration"](W, iters)))),

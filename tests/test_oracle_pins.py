@@ -288,3 +288,30 @@ def test_sampled_mlr_helpers_match_the_plain_step():
     Wn = O.sfb_step(O.MLR, W, X, None, y, workers=2, eta=0.05)
     rows = np.array([0, 5, 36, int(y[0])])
     np.testing.assert_allclose(O.mlr_updated_rows(W[rows], rows, X, y, lse, 0.05), Wn[rows], atol=1e-14)
+
+
+def test_entrywise_prox_operators_solve_their_defining_problem():
+    """prox_{t h}(w) = argmin_v 1/2 (v - w)^2 + t h(v) (Section 2.1, proximal SGD), entry by entry: checked against
+    scipy's bounded scalar minimiser, which the oracle does not use; plus what the definition implies."""
+    from scipy.optimize import minimize_scalar
+    rng = np.random.default_rng(12)
+    w = np.concatenate([rng.normal(size=12), [0.0, 0.3, -0.3, 0.3000001, 1e-9]])
+    for t in (0.0, 0.3, 2.0):
+        for kind, h in (("l1", abs), ("l2sq", lambda v: 0.5 * v * v)):
+            got = O.prox_entries(w, kind, t)
+            for wi, gi in zip(w, got):
+                r = minimize_scalar(lambda v: 0.5 * (v - wi) ** 2 + t * h(v), bounds=(-10, 10), method="bounded",
+                                    options={"xatol": 1e-12})
+                assert abs(gi - r.x) < 1e-6, (kind, t, wi)
+            assert np.all(np.abs(got) <= np.abs(w) + 1e-15) and np.all(got * w >= 0)       # shrinks, keeps the sign
+            w2 = w + 0.1 * rng.normal(size=w.shape)
+            assert np.linalg.norm(O.prox_entries(w2, kind, t) - got) <= np.linalg.norm(w2 - w) + 1e-15   # non-expansive
+    np.testing.assert_array_equal(O.prox_l1(w, 0.0), w)
+    assert np.all(O.prox_l1(w, 0.3)[np.abs(w) <= 0.3] == 0.0)                               # the dead zone of the l1 prox
+    np.testing.assert_allclose(O.prox_l2sq(w, 1.0), 0.5 * w)
+    assert O.prox_entries(w, None, 5.0) is not None and np.array_equal(O.prox_entries(w, None, 5.0), w)
+    # a step with a regulariser is the plain step followed by the operator with t = eta * weight
+    W, X, y = rng.normal(size=(5, 7)), rng.normal(size=(6, 7)), rng.integers(0, 5, size=6)
+    plain = O.sfb_step(O.MLR, W, X, None, y, workers=2, eta=0.2)
+    np.testing.assert_array_equal(O.sfb_step(O.MLR, W, X, None, y, workers=2, eta=0.2, prox_kind="l1", prox_weight=0.5),
+                                  O.prox_l1(plain, 0.1))
