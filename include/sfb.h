@@ -80,6 +80,11 @@ typedef struct sfb_config {
   int32_t sc_prox;        /* 0 none | 1 rescale columns of norm > 1 to norm 1 (Figure 3)               */
   float   sdca_lambda;    /* SFB_L2MLR: weight lam of the regulariser h(W) = lam/2 ||W||_F^2 (> 0)    */
   int64_t sdca_n;         /* SFB_L2MLR: N, the number of training samples (rows of the dual state)     */
+  int32_t prox_kind;      /* entry-wise proximal operator applied with the update (Section 2.1, proximal SGD):
+                             0 none | 1 h = w ||W||_1: entries shrunk towards 0 by eta*w | 2 h = w/2 ||W||_F^2:
+                             entries divided by 1 + eta*w.  Fused into the update pass; for SC it comes before
+                             the column rescaling.  Not for SFB_L2MLR (its regulariser lives in the dual).     */
+  float   prox_weight;    /* the weight w of that regulariser (>= 0)                                  */
   void*   stream;         /* cudaStream_t                                                              */
 } sfb_config;
 

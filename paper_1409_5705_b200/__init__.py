@@ -13,6 +13,7 @@ from .build import LIB, build
 
 MLR, DML, SC, L2MLR = 0, 1, 2, 3
 PREC_BF16, PREC_FP32 = 0, 1
+PROX_NONE, PROX_L1, PROX_L2SQ = 0, 1, 2
 STATUS_LABEL_RANGE, STATUS_TIMEOUT, STATUS_SAMPLE_RANGE = 0x1, 0x2, 0x4
 
 EXPORTS = ("sfb_workspace_bytes", "sfb_init", "sfb_compute_factors", "sfb_gather_factors", "sfb_apply_update",
@@ -29,7 +30,8 @@ class sfb_config(ctypes.Structure):
                 ("cols", ctypes.c_int64), ("workers", ctypes.c_int32), ("batch", ctypes.c_int32),
                 ("eta", ctypes.c_float), ("dml_margin", ctypes.c_float), ("sc_lambda", ctypes.c_float),
                 ("sc_ista_iters", ctypes.c_int32), ("sc_lipschitz", ctypes.c_float), ("sc_prox", ctypes.c_int32),
-                ("sdca_lambda", ctypes.c_float), ("sdca_n", ctypes.c_int64), ("stream", ctypes.c_void_p)]
+                ("sdca_lambda", ctypes.c_float), ("sdca_n", ctypes.c_int64), ("prox_kind", ctypes.c_int32),
+                ("prox_weight", ctypes.c_float), ("stream", ctypes.c_void_p)]
 
 
 class sfb_stats(ctypes.Structure):
@@ -98,9 +100,10 @@ def strerror(code: int) -> str:
 
 
 def make_config(model, rows, cols, workers, batch, eta, precision=PREC_FP32, dml_margin=1.0, sc_lambda=0.1,
-                sc_ista_iters=20, sc_lipschitz=0.0, sc_prox=0, stream=0, sdca_lambda=0.0, sdca_n=0) -> sfb_config:
+                sc_ista_iters=20, sc_lipschitz=0.0, sc_prox=0, stream=0, sdca_lambda=0.0, sdca_n=0, prox_kind=0,
+                prox_weight=0.0) -> sfb_config:
     return sfb_config(model, precision, rows, cols, workers, batch, eta, dml_margin, sc_lambda, sc_ista_iters,
-                      sc_lipschitz, sc_prox, sdca_lambda, sdca_n, stream)
+                      sc_lipschitz, sc_prox, sdca_lambda, sdca_n, prox_kind, prox_weight, stream)
 
 
 def sfb_workspace_bytes(cfg: sfb_config) -> int:

@@ -83,6 +83,8 @@ static int check_config(const sfb_config* c) {
   if (c->model == SFB_SC && c->sc_ista_iters < 0) return SFB_ERR_ARG;
   if (c->model == SFB_SC && !(c->sc_lambda >= 0.f)) return SFB_ERR_ARG;
   if (c->sc_prox < 0 || c->sc_prox > 1) return SFB_ERR_ARG;
+  if (c->prox_kind < 0 || c->prox_kind > 2 || !(c->prox_weight >= 0.f)) return SFB_ERR_ARG;
+  if (c->model == SFB_L2MLR && c->prox_kind != 0) return SFB_ERR_UNSUPPORTED;
   return SFB_OK;
 }
 
@@ -119,6 +121,10 @@ extern "C" int sfb_init(const sfb_config* cfg, float* W_dev, void* workspace_dev
   ctx->step = ctx->sdca ? static_cast<float>(static_cast<double>(cfg->eta) / (static_cast<double>(cfg->sdca_lambda) *
                                                                             static_cast<double>(cfg->sdca_n)))
                         : cfg->eta;
+  // prox_{eta h}: threshold eta*w for the l1 norm, factor 1 / (1 + eta*w) for the squared l2 norm
+  ctx->prox_kind = cfg->prox_kind;
+  ctx->prox_a = cfg->prox_kind == 1 ? cfg->eta * cfg->prox_weight
+              : cfg->prox_kind == 2 ? static_cast<float>(1.0 / (1.0 + static_cast<double>(cfg->eta) * cfg->prox_weight)) : 0.f;
   ctx->lay = lay;
   ctx->W = W_dev;
   ctx->ws = static_cast<char*>(workspace_dev);
@@ -206,6 +212,7 @@ static int update_fp32(sfb_ctx* ctx) {
   const sfb_config& c = ctx->cfg;
   EpiArgs e{};
   e.C = ctx->W; e.ldc = c.cols; e.alpha = -ctx->step;
+  e.prox_kind = ctx->prox_kind; e.prox_a = ctx->prox_a;
   CK(sgemm(ctx->stream, false, false, EPI_RMW, c.rows, c.cols, ctx->K, ctx->at<float>(ctx->lay.U), c.rows,
            ctx->at<float>(ctx->lay.V), c.cols, e));
   return SFB_OK;
@@ -505,6 +512,7 @@ extern "C" int sfb_dense_sync_step(sfb_ctx* ctx, const float* X_dev, const float
     if (p > 0) CK(axpy(ctx->stream, sum, one, 1.f, static_cast<int64_t>(mat)));          // server-side aggregation
   }
   CK(axpy(ctx->stream, ctx->W, sum, -c.eta, static_cast<int64_t>(mat)));                 // W <- W - eta * sum_p dW_p
+  CK(prox_entries(ctx->stream, ctx->W, static_cast<int64_t>(mat), ctx->prox_kind, ctx->prox_a));
   ctx->stats.flops += 2.0 * c.rows * c.cols * ctx->K;
   rc = apply_prox(ctx);
   if (rc) return rc;

@@ -68,6 +68,12 @@ __global__ void zero_kernel(float* __restrict__ dst, int64_t n) {
   for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < n; i += stride) dst[i] = 0.f;
 }
 
+__global__ void prox_entries_kernel(float* __restrict__ w, int64_t n, int kind, float a) {
+  const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+  for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < n; i += stride)
+    w[i] = prox_entry(w[i], kind, a);
+}
+
 __global__ void axpy_kernel(float* __restrict__ y, const float* __restrict__ x, float alpha, int64_t n) {
   const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
   for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < n; i += stride)
@@ -477,6 +483,13 @@ cudaError_t mlr_softmax_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t ro
                              float* loss, uint32_t* status) {
   if (nsamp <= 0) return cudaSuccess;
   mlr_softmax_kernel<512><<<static_cast<unsigned>(nsamp), 512, 0, s>>>(Z, rows, labels, loss, status);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t prox_entries(cudaStream_t s, float* w, int64_t n, int kind, float a) {
+  if (n <= 0 || kind == 0) return cudaSuccess;
+  prox_entries_kernel<<<grid_for(n, kThreads), kThreads, 0, s>>>(w, n, kind, a);
   count_launch();
   return cudaGetLastError();
 }

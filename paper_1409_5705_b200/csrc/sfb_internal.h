@@ -62,6 +62,8 @@ struct sfb_ctx {
   float* dualQ;                       // SDCA dual state [dual_n x rows], caller-owned
   int64_t dual_n;
   float step;                         // multiplier of sum u v^T in the update: eta, or eta / (lam N) for SDCA
+  int32_t prox_kind;                  // entry-wise prox of the update pass and its parameter (threshold or factor)
+  float prox_a;
   uint64_t committed;                 // bit p set: worker p has written its factors since the last update
   bool gathered;
   int last_cuda;
@@ -81,7 +83,18 @@ namespace sfb {
 // ---------------------------------------------------------------------------------------------------------
 enum Epilogue { EPI_STORE = 0, EPI_SUB = 1, EPI_RMW = 2, EPI_ISTA = 3 };
 
+// Entry-wise proximal operator fused into the update: kind 1 soft-threshold by a, kind 2 multiply by a.
+__host__ __device__ __forceinline__ float prox_entry(float w, int kind, float a) {
+  if (kind == 1) {
+    const float m = fabsf(w) - a;
+    return m > 0.f ? copysignf(m, w) : 0.f;
+  }
+  return kind == 2 ? w * a : w;
+}
+
 struct EpiArgs {
+  int32_t prox_kind;   // EPI_RMW: entry-wise prox applied to the updated value (0 none)
+  float prox_a;
   float* C;            // output, row-major [M x ldc]
   int64_t ldc;
   const float* aux;    // EPI_SUB: the matrix subtracted, same shape and ld as C
@@ -120,5 +133,6 @@ cudaError_t estimate_lipschitz(cudaStream_t s, const float* W, int64_t rows, int
                                float* colpart, Scalars* sc, int iters);
 cudaError_t set_lipschitz(cudaStream_t s, Scalars* sc, float L);
 cudaError_t axpy(cudaStream_t s, float* y, const float* x, float alpha, int64_t n);  // y += alpha*x
+cudaError_t prox_entries(cudaStream_t s, float* w, int64_t n, int kind, float a);      // w <- prox(w), entry-wise
 
 }  // namespace sfb

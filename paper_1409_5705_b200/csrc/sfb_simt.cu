@@ -74,7 +74,7 @@ template <int EPI>
 __device__ __forceinline__ float epi_one(float acc, float cur, float aux, const EpiArgs& e, float invL) {
   if (EPI == EPI_STORE) return acc;
   if (EPI == EPI_SUB) return acc - aux;
-  if (EPI == EPI_RMW) return fmaf(e.alpha, acc, cur);
+  if (EPI == EPI_RMW) return prox_entry(fmaf(e.alpha, acc, cur), e.prox_kind, e.prox_a);
   return soft(fmaf(-acc, invL, cur), e.lam * invL);   // EPI_ISTA
 }
 

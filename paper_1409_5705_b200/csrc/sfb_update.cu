@@ -54,6 +54,8 @@ struct UpdParams {
   // array of a kernel parameter with a run-time index moves the whole parameter block to local memory.
   int32_t a_off0, a_off1, a_off2, b_off0, b_off1, b_off2;
   float alpha;
+  int32_t prox_kind;           // entry-wise prox applied to the updated value (0 none, 1 soft-threshold, 2 scale)
+  float prox_a;
   __nv_bfloat16* shadow;       // bf16 copy of the updated W (or null), row pitch shadow_ld elements
   int64_t shadow_ld;
   uint32_t* status;
@@ -226,6 +228,10 @@ update_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
           w.y = fmaf(p.alpha, __uint_as_float(acc[4 * j + 1]), w.y);
           w.z = fmaf(p.alpha, __uint_as_float(acc[4 * j + 2]), w.z);
           w.w = fmaf(p.alpha, __uint_as_float(acc[4 * j + 3]), w.w);
+          if (p.prox_kind != 0) {
+            w.x = prox_entry(w.x, p.prox_kind, p.prox_a); w.y = prox_entry(w.y, p.prox_kind, p.prox_a);
+            w.z = prox_entry(w.z, p.prox_kind, p.prox_a); w.w = prox_entry(w.w, p.prox_kind, p.prox_a);
+          }
           *wp = w;
         }
         fence_proxy_async_smem();
@@ -405,6 +411,7 @@ int tc_update(sfb_ctx* ctx) {
   p.tilesN = static_cast<int32_t>((c.cols + UN - 1) / UN);
   p.kseg = static_cast<int32_t>(L.Kp / UK);
   p.alpha = -ctx->step;
+  p.prox_kind = ctx->prox_kind; p.prox_a = ctx->prox_a;
   p.status = ctx->at<uint32_t>(L.status);
   const int64_t tiles = static_cast<int64_t>(p.tilesM) * p.tilesN;
   const unsigned grid = 2u * static_cast<unsigned>(std::min<int64_t>(tiles, st->max_pairs));
@@ -421,16 +428,22 @@ int tc_update(sfb_ctx* ctx) {
   }
   p.nseg = 1;
   p.shadow = ctx->at<__nv_bfloat16>(L.Wb); p.shadow_ld = L.colsb;
-  update_pair_kernel<true><<<grid, kThreads, kSmem, ctx->stream>>>(ma, mb, mc, p);     // W += -eta * P^T V
-  count_launch();
-  CKC(cudaGetLastError());
   if ((c.cols + 1023) / 1024 > 65535) return SFB_ERR_SHAPE;
   dim3 lgrid(static_cast<unsigned>(ctx->K), static_cast<unsigned>((c.cols + 1023) / 1024));
-  label_rows_kernel<<<lgrid, 256, 0, ctx->stream>>>(
-      ctx->W, c.rows, c.cols, ctx->at<float>(L.Xf), ctx->at<int32_t>(L.labels), ctx->at<float>(L.coef), static_cast<int>(ctx->K), ctx->step,
-      ctx->at<__nv_bfloat16>(L.Wb), L.colsb);                // W[y_i] += eta * (1 - p_iy) * x_i
-  count_launch();
-  CKC(cudaGetLastError());
+  // With a fused prox the fp32 label-row term has to be in W before the pass that applies the operator, so it goes
+  // first (both terms are sums into W; the pass then also writes the bf16 copy of those rows).
+  const bool labels_first = ctx->prox_kind != 0;
+  for (int pass = 0; pass < 2; ++pass) {
+    if ((pass == 0) == labels_first) {
+      label_rows_kernel<<<lgrid, 256, 0, ctx->stream>>>(
+          ctx->W, c.rows, c.cols, ctx->at<float>(L.Xf), ctx->at<int32_t>(L.labels), ctx->at<float>(L.coef),
+          static_cast<int>(ctx->K), ctx->step, labels_first ? nullptr : ctx->at<__nv_bfloat16>(L.Wb), L.colsb);
+    } else {
+      update_pair_kernel<true><<<grid, kThreads, kSmem, ctx->stream>>>(ma, mb, mc, p);     // W += -eta * P^T V
+    }
+    count_launch();
+    CKC(cudaGetLastError());
+  }
   return SFB_OK;
 }
 
