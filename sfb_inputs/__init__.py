@@ -229,3 +229,18 @@ def _mlr_pool(wl: Workload):
         y = zipf_labels(wl.seed, _S_LABEL, 0, wl.n_samples, wl.rows, wl.zipf_s)
         _POOLS[key] = (X, y)
     return _POOLS[key]
+
+
+# ----------------------------------------------------------------------------------------------------------
+# Delivery delays for the stale-synchronous emulation (Section 4.1): delay[c][p][q] in [0, staleness] is how many clocks
+# beyond the next one the factors worker p produced at clock c take to reach worker q (0 on the diagonal).
+# ----------------------------------------------------------------------------------------------------------
+_S_DELAY = 9
+
+
+def ssp_delays(seed: int, clocks: int, workers: int, staleness: int) -> np.ndarray:
+    g = _gen(seed, _S_DELAY, 0)
+    d = g.integers(0, staleness + 1, size=(clocks, workers, workers), dtype=np.int64)
+    for p in range(workers):
+        d[:, p, p] = 0
+    return d
