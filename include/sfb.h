@@ -152,6 +152,18 @@ int sfb_sdca_compute_factors(sfb_ctx* ctx, int32_t worker, const float* X_dev, c
                              const int32_t* sample_ids_dev);
 int sfb_sdca_step(sfb_ctx* ctx, const float* X_dev, const int32_t* labels_dev, const int32_t* sample_ids_dev);
 
+/* The receiving side of the broadcast (Section 3: a worker applies the sufficient factors it has received from the
+ * others): the B pairs U_dev [B x rows], V_dev [B x cols] (fp32, pair-major, dense rows), computed elsewhere -- by
+ * another replica, under another consistency model (Section 4.1), on another machine -- take worker `worker`'s place
+ * in the gathered buffers and the worker counts as committed.  Pairs come out of a context through sfb_get_factors.
+ * Built for the layouts in which factors are fp32 pairs (SFB_PREC_FP32; DML and SC in either mode); SFB_ERR_UNSUPPORTED
+ * for MLR in bf16 mode (its u is held as bf16 probabilities plus an fp32 label term) and for SFB_L2MLR. */
+int sfb_set_factors(sfb_ctx* ctx, int32_t worker, const float* U_dev, const float* V_dev);
+
+/* Changes the step size eta of the following updates (step-size schedules, e.g. the decreasing eta_c of the
+ * convergence analysis in Section 5).  SFB_ERR_STATE between the factors of a step and their update. */
+int sfb_set_eta(sfb_ctx* ctx, float eta);
+
 /* The broadcast of Section 3 as an on-device gather: after it, U [K x rows] and V [K x cols] of all P workers
  * sit in one buffer in the operand layout of the update.  Fails with SFB_ERR_STATE unless every worker has
  * computed its factors since the last update.  Accounts the bytes of Section 5's cost table. */

@@ -21,7 +21,7 @@ EXPORTS = ("sfb_workspace_bytes", "sfb_init", "sfb_compute_factors", "sfb_gather
            "sfb_get_status", "sfb_strerror", "sfb_last_cuda_error", "sfb_destroy", "sfb_prox_columns_noalloc",
            "sfb_selftest_wait_timeout", "sfb_set_row_shard", "sfb_forward_partials", "sfb_finish_factors",
            "sfb_replay_update", "sfb_refresh_operands", "sfb_sdca_set_dual", "sfb_sdca_compute_factors",
-           "sfb_sdca_step")
+           "sfb_sdca_step", "sfb_set_factors", "sfb_set_eta")
 NOALLOC_MAX_COLS = 16384
 
 
@@ -88,6 +88,8 @@ def lib() -> ctypes.CDLL:
         L.sfb_sdca_set_dual.argtypes = [vp, vp, i64]
         L.sfb_sdca_compute_factors.argtypes = [vp, i32, vp, vp, vp]
         L.sfb_sdca_step.argtypes = [vp, vp, vp, vp]
+        L.sfb_set_factors.argtypes = [vp, i32, vp, vp]
+        L.sfb_set_eta.argtypes = [vp, ctypes.c_float]
         for name in EXPORTS:
             if name != "sfb_strerror":
                 getattr(L, name).restype = ctypes.c_int
@@ -167,14 +169,22 @@ class Context:
                  "sfb_sdca_compute_factors")
 
     def sfb_sdca_step(self, X, labels, sample_ids):
-        self._ck(lib().sfb_sdca_step(self._h, _ptr(X), _ptr(labels), _ptr(sample_ids)), "sfb_sdca_step")
+        self._ck(lib().sfb_sdca_step(self._h, _ptr(X), _ptr(labels), _ptr(sample_ids)), "sfb_sdca_step", "sfb_set_factors", "sfb_set_eta")
+
+    def sfb_set_factors(self, worker, U, V):
+        """U [B, rows], V [B, cols]: contiguous fp32 CUDA tensors of factors computed elsewhere."""
+        self._ck(lib().sfb_set_factors(self._h, worker, _ptr(U), _ptr(V)), "sfb_set_factors")
+
+    def sfb_set_eta(self, eta):
+        self._ck(lib().sfb_set_eta(self._h, eta), "sfb_set_eta")
+        self.cfg.eta = eta
 
     def sfb_refresh_operands(self):
         self._ck(lib().sfb_refresh_operands(self._h), "sfb_refresh_operands")
 
     def sfb_replay_update(self):
         self._ck(lib().sfb_replay_update(self._h), "sfb_replay_update", "sfb_refresh_operands", "sfb_sdca_set_dual", "sfb_sdca_compute_factors",
-           "sfb_sdca_step")
+           "sfb_sdca_step", "sfb_set_factors", "sfb_set_eta")
 
     def sfb_step(self, X, Y=None, labels=None):
         self._ck(lib().sfb_step(self._h, _ptr(X), _ptr(Y), _ptr(labels)), "sfb_step")

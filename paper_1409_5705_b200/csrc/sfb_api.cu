@@ -321,6 +321,39 @@ extern "C" int sfb_finish_factors(sfb_ctx* ctx, const float* partials_all_dev, i
   return SFB_OK;
 }
 
+// Sufficient factors computed elsewhere (another replica, another machine) take the place of a worker's own:
+// the receiving side of the broadcast of Section 3.
+extern "C" int sfb_set_factors(sfb_ctx* ctx, int32_t worker, const float* U_dev, const float* V_dev) {
+  if (!ctx || !U_dev || !V_dev) return SFB_ERR_ARG;
+  const sfb_config& c = ctx->cfg;
+  if (worker < 0 || worker >= c.workers) return SFB_ERR_SHAPE;
+  if (ctx->sdca || (c.precision == SFB_PREC_BF16 && c.model == SFB_MLR)) return SFB_ERR_UNSUPPORTED;
+  if (ctx->partials_ready) return SFB_ERR_STATE;
+  if (ctx->committed == 0) CK(cudaEventRecord(ctx->ev[0], ctx->stream));
+  const int64_t off = static_cast<int64_t>(worker) * c.batch;
+  const int64_t ldu = c.precision == SFB_PREC_FP32 ? c.rows : ctx->lay.ldu;
+  float* U = ctx->at<float>(ctx->lay.U) + off * ldu;
+  float* V = ctx->at<float>(ctx->lay.V) + off * c.cols;
+  CK(cudaMemcpy2DAsync(U, static_cast<size_t>(ldu) * 4, U_dev, static_cast<size_t>(c.rows) * 4, static_cast<size_t>(c.rows) * 4,
+                       static_cast<size_t>(c.batch), cudaMemcpyDeviceToDevice, ctx->stream));
+  CK(cudaMemcpyAsync(V, V_dev, static_cast<size_t>(c.batch) * c.cols * 4, cudaMemcpyDeviceToDevice, ctx->stream));
+  ctx->committed |= 1ull << worker;
+  ctx->gathered = false;
+  return SFB_OK;
+}
+
+extern "C" int sfb_set_eta(sfb_ctx* ctx, float eta) {
+  if (!ctx || !(eta >= 0.f)) return SFB_ERR_ARG;
+  if (ctx->committed != 0 || ctx->partials_ready) return SFB_ERR_STATE;       // not between the factors and their update
+  ctx->cfg.eta = eta;
+  ctx->step = ctx->sdca ? static_cast<float>(static_cast<double>(eta) / (static_cast<double>(ctx->cfg.sdca_lambda) *
+                                                                        static_cast<double>(ctx->cfg.sdca_n)))
+                        : eta;
+  ctx->prox_a = ctx->prox_kind == 1 ? eta * ctx->cfg.prox_weight
+              : ctx->prox_kind == 2 ? static_cast<float>(1.0 / (1.0 + static_cast<double>(eta) * ctx->cfg.prox_weight)) : 0.f;
+  return SFB_OK;
+}
+
 extern "C" int sfb_gather_factors(sfb_ctx* ctx) {
   if (!ctx) return SFB_ERR_ARG;
   const sfb_config& c = ctx->cfg;
