@@ -1,4 +1,11 @@
-"""Row-sharded multiclass logistic regression over several GPUs: host-side sequencing only.
+"""Sufficient-factor broadcasting over several GPUs: host-side sequencing only.  Two forms:
+
+* ``replica_step`` -- the paper's own (Section 3, Figure 1): every rank holds a full replica of W, computes the
+  factors of its logical workers, the ranks all-gather their factors (K*(rows+cols)*4 bytes in total, the linear volume
+  of Section 5), and every rank applies all K pairs to its replica.
+* ``sharded_step`` -- W partitioned by rows (multiclass logistic regression), described next.
+
+Row-sharded multiclass logistic regression:
 
 Each rank owns a contiguous block of the rows (classes) of W and a block of the K samples of a step (its logical
 workers).  One step is
@@ -80,3 +87,37 @@ def sharded_step(ctx, X_local, labels_local, partials, partials_all, X_all, labe
     ctx.sfb_gather_factors()
     ctx.sfb_apply_update()
     return moved
+
+
+def replica_step(ctx, my_workers, X_local, Y_local, labels_local, U_all, V_all, group=None, dist=None):
+    """One step of the replica form on this rank.
+
+    ctx          a context over this rank's replica of W with ALL P workers in its config (fp32 factor layout)
+    my_workers   the worker indices this rank computes, ascending and contiguous; X_local [len*B, in_dim] etc. hold
+                 their samples in that order
+    U_all, V_all [K, rows], [K, cols] fp32: receive every worker's factors (worker-major)
+    Returns the bytes this rank received.
+    """
+    B = ctx.cfg.batch
+    for k, p in enumerate(my_workers):
+        sl = slice(k * B, (k + 1) * B)
+        ctx.sfb_compute_factors(p, X_local[sl], None if Y_local is None else Y_local[sl],
+                                None if labels_local is None else labels_local[sl])
+    U, V = ctx.factors_as_tensors()
+    lo, hi = my_workers[0] * B, (my_workers[-1] + 1) * B
+    U_own, V_own = U[lo:hi].contiguous(), V[lo:hi].contiguous()
+    if dist is None:
+        U_all[lo:hi].copy_(U_own)
+        V_all[lo:hi].copy_(V_own)
+        received = 0
+    else:
+        dist.all_gather_into_tensor(U_all, U_own, group=group)
+        dist.all_gather_into_tensor(V_all, V_own, group=group)
+        received = (U_all.numel() - U_own.numel() + V_all.numel() - V_own.numel()) * U_all.element_size()
+    mine = set(my_workers)
+    for q in range(ctx.cfg.workers):
+        if q not in mine:
+            ctx.sfb_set_factors(q, U_all[q * B:(q + 1) * B], V_all[q * B:(q + 1) * B])
+    ctx.sfb_gather_factors()
+    ctx.sfb_apply_update()
+    return received

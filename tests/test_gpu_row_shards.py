@@ -150,3 +150,51 @@ def test_row_shard_call_order_and_argument_errors():
         cd.sfb_set_row_shard(0, 64)
     assert e.value.code == -10
     cd.close()
+
+
+@pytest.mark.parametrize("name", ["mlr", "dml"])
+def test_replica_form_two_ranks_on_one_gpu(name):
+    """The paper's own form: two replicas of W, each computes the factors of half of the workers, the factors are
+    exchanged (here: copied between the two contexts' buffers, as an all-gather would), both apply all K pairs.  Both
+    replicas must end at the oracle's step."""
+    from paper_1409_5705_b200.sharded import replica_step
+    if name == "mlr":
+        wl, prec = I.scaled(_workload(), "mlr_rep", workers=4, batch=20), S.PREC_FP32
+    else:
+        wl, prec = I.scaled(I.WORKLOADS["dml"], "dml_rep", rows=150, cols=388, workers=4, batch=33, eta=1e-3), S.PREC_BF16
+    W0 = I.initial_W(wl)
+    inp = I.step_inputs(wl, 0)
+    ref = oracle_step(wl, W0, inp)
+    G, B, K = 2, wl.batch, wl.K
+    Ws = [to_dev(W0, torch) for _ in range(G)]
+    ctxs = [S.Context(config_for(wl, prec), W) for W in Ws]
+    U_all = torch.zeros((K, wl.rows), dtype=torch.float32, device="cuda")
+    V_all = torch.zeros((K, wl.cols), dtype=torch.float32, device="cuda")
+    X, Y, lab = to_dev(inp.X, torch), to_dev(inp.Y, torch), to_dev(inp.labels, torch)
+    own = [list(range(g * 2, g * 2 + 2)) for g in range(G)]
+    # phase 1: every rank computes and publishes its own factors (what the all-gather delivers)
+    for g, ctx in enumerate(ctxs):
+        lo, hi = own[g][0] * B, (own[g][-1] + 1) * B
+        for p in own[g]:
+            sl = slice(p * B, (p + 1) * B)
+            ctx.sfb_compute_factors(p, X[sl], None if Y is None else Y[sl], lab[sl])
+        U, V = ctx.factors_as_tensors()
+        U_all[lo:hi].copy_(U[lo:hi])
+        V_all[lo:hi].copy_(V[lo:hi])
+    # phase 2: every rank takes the others' factors and applies all K pairs
+    for g, ctx in enumerate(ctxs):
+        for q in range(wl.workers):
+            if q not in own[g]:
+                ctx.sfb_set_factors(q, U_all[q * B:(q + 1) * B], V_all[q * B:(q + 1) * B])
+        ctx.sfb_gather_factors()
+        ctx.sfb_apply_update()
+        assert ctx.sfb_get_status() == 0
+        assert rel_err(Ws[g].cpu().numpy(), ref, W0) <= TOL[prec], g
+        ctx.close()
+    assert torch.equal(Ws[0], Ws[1])                         # the replicas stay bit-identical
+    # the single-rank form of the helper gives the same step
+    W = to_dev(W0, torch)
+    ctx = S.Context(config_for(wl, prec), W)
+    assert replica_step(ctx, list(range(wl.workers)), X, Y, lab, U_all, V_all) == 0
+    assert torch.equal(W, Ws[0])
+    ctx.close()

@@ -142,3 +142,85 @@ def test_single_shard_needs_no_process_group():
     ref = O.sfb_step(O.MLR, W0, inp.X, None, inp.labels, workers=wl.workers, eta=wl.eta)
     assert np.linalg.norm(ctx.W - ref) <= 1e-12 * np.linalg.norm(ref - W0)
     assert moved.total == 0
+
+
+class _FakeReplica:
+    """What the calls of the replica form do, in numpy fp64 (a test double): factors of a worker from the oracle's own
+    formula for MLR, factors taken from elsewhere, and the update with all of them."""
+
+    class _Cfg:
+        pass
+
+    def __init__(self, W, P, B, eta):
+        from oracle import sfb_oracle as O
+        self.O = O
+        self.W = W.astype(np.float64)
+        self.cfg = self._Cfg()
+        self.cfg.workers, self.cfg.batch = P, B
+        self.eta = eta
+        self.U = torch.zeros((P * B, W.shape[0]), dtype=torch.float64)
+        self.V = torch.zeros((P * B, W.shape[1]), dtype=torch.float64)
+        self.have = set()
+
+    def sfb_compute_factors(self, p, X, Y, labels):
+        B = self.cfg.batch
+        U, V = self.O.mlr_factors(self.W, X.numpy(), labels.numpy())
+        self.U[p * B:(p + 1) * B] = torch.from_numpy(U)
+        self.V[p * B:(p + 1) * B] = torch.from_numpy(V)
+        self.have.add(p)
+
+    def factors_as_tensors(self):
+        return self.U, self.V
+
+    def sfb_set_factors(self, q, U, V):
+        B = self.cfg.batch
+        self.U[q * B:(q + 1) * B] = U
+        self.V[q * B:(q + 1) * B] = V
+        self.have.add(q)
+
+    def sfb_gather_factors(self):
+        assert self.have == set(range(self.cfg.workers))
+
+    def sfb_apply_update(self):
+        self.W = self.O.rank_k_update(self.W, self.U.numpy(), self.V.numpy(), self.eta)
+
+
+def _replica_rank(rank, world, port, out_dir):
+    import torch.distributed as dist
+    sys.path.insert(0, ROOT)
+    import sfb_inputs as I
+    from paper_1409_5705_b200.sharded import replica_step
+    dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=rank, world_size=world)
+    wl = I.scaled(I.WORKLOADS["mlr_mid"], "mlr_rep", rows=15, cols=12, workers=4, batch=3, eta=0.1, w_std=0.2,
+                  x_scale="unit")
+    W0 = I.initial_W(wl)
+    inp = I.step_inputs(wl, 0)
+    B, K = wl.batch, wl.K
+    mine = [2 * rank, 2 * rank + 1]
+    lo, hi = mine[0] * B, (mine[-1] + 1) * B
+    ctx = _FakeReplica(W0, wl.workers, B, wl.eta)
+    U_all = torch.zeros((K, wl.rows), dtype=torch.float64)
+    V_all = torch.zeros((K, wl.cols), dtype=torch.float64)
+    got = replica_step(ctx, mine, torch.from_numpy(inp.X[lo:hi].astype(np.float64)), None, torch.from_numpy(inp.labels[lo:hi]),
+                       U_all, V_all, dist=dist)
+    np.save(os.path.join(out_dir, f"R{rank}.npy"), ctx.W)
+    assert got == (K - 2 * B) * (wl.rows + wl.cols) * 8
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_keep_identical_replicas_equal_to_the_oracle_step(tmp_path):
+    import torch.multiprocessing as mp
+    sys.path.insert(0, ROOT)
+    import sfb_inputs as I
+    from oracle import sfb_oracle as O
+    port = 33500 + os.getpid() % 2000
+    mp.spawn(_replica_rank, args=(2, port, str(tmp_path)), nprocs=2, join=True)
+    wl = I.scaled(I.WORKLOADS["mlr_mid"], "mlr_rep", rows=15, cols=12, workers=4, batch=3, eta=0.1, w_std=0.2,
+                  x_scale="unit")
+    W0 = I.initial_W(wl)
+    inp = I.step_inputs(wl, 0)
+    ref = O.sfb_step(O.MLR, W0, inp.X, None, inp.labels, workers=wl.workers, eta=wl.eta)
+    R0, R1 = np.load(tmp_path / "R0.npy"), np.load(tmp_path / "R1.npy")
+    assert np.array_equal(R0, R1)
+    assert np.linalg.norm(R0 - ref) <= 1e-12 * np.linalg.norm(ref - W0)
