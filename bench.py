@@ -244,11 +244,30 @@ def workload_config(wl, dtype):
             else "l2_flushed_between_steps"}
 
 
+def precision_code(S, name):
+    return {"bf16": S.PREC_BF16, "fp32": S.PREC_FP32, "tf32": S.PREC_TF32X3, "ffma": S.PREC_FP32_FFMA}[name]
+
+
+def dtype_name(wl, name):
+    """The arithmetic type of the products: bf16, f32 (FFMA) or tf32x3 (fp32 values as pairs of tf32 words)."""
+    if name == "bf16":
+        return "bf16"
+    return "tf32x3" if runs_tf32(wl, name) else "f32"
+
+
+def runs_tf32(wl, name):
+    """Whether the fp32 mode runs this workload's products on the tensor cores (the library's own rule)."""
+    if wl.model != I.MLR or name in ("bf16", "ffma"):
+        return False
+    return name == "tf32" or (wl.rows >= 2048 and wl.cols >= 512 and wl.K >= 128)
+
+
 NOMINAL_BF16_TFLOPS = 2250.0        # dense bf16, vendor figure (context only)
+NOMINAL_TF32_OVER_BF16 = 1100.0 / 2250.0   # nominal ratio of the dense tf32 and bf16 tensor rates
 NOMINAL_HBM_GBS = 7700.0
 
 
-def update_roofline(wl, prec_bf16, ms_u, peaks, clocks, sustained=True):
+def update_roofline(wl, prec_bf16, ms_u, peaks, clocks, sustained=True, tf32=False):
     """Roofline entry of the fused update W += -eta U^T V (one launch per step).  Algorithmic bytes per launch: W read
     and written once in fp32 plus U and V read once (what the method has to move).  The bf16 copy of W that this design
     writes alongside (the operand of the next forward product) is real traffic of the kernel and is reported beside
@@ -271,6 +290,13 @@ def update_roofline(wl, prec_bf16, ms_u, peaks, clocks, sustained=True):
             roof = {"bound": "tensor", "achieved": upd_flops / (ms_u * 1e-3) / 1e12, "peak": tf_peak,
                     "unit": "TFLOP/s"}
         roof["roof_ms"] = max(t_flop, t_mem) * 1e3
+    elif tf32:
+        # fp32 operands as tf32 pairs: three tf32 products per term.  Peak for that dtype = the measured bf16 figure
+        # times the nominal tf32/bf16 ratio; "achieved" counts the three products the kernel executes.
+        peak = tf_peak * NOMINAL_TF32_OVER_BF16
+        roof = {"bound": "tensor", "achieved": 3.0 * upd_flops / (ms_u * 1e-3) / 1e12, "peak": peak, "unit": "TFLOP/s",
+                "note": "tf32 peak = measured bf16 x nominal ratio 1.1/2.25; achieved = executed flops (3 products per term)"}
+        roof["roof_ms"] = max(3.0 * upd_flops / (peak * 1e12), upd_bytes / (peaks["hbm_gbs"] * 1e9)) * 1e3
     else:
         # fp32 FMA pipe: SMs x 128 lanes x 2 flop x max SM clock
         peak = 148 * 128 * 2 * ((clocks or {}).get("sm_max_mhz") or 1965.0) * 1e6 / 1e12
@@ -280,7 +306,7 @@ def update_roofline(wl, prec_bf16, ms_u, peaks, clocks, sustained=True):
     roof["traffic"] = ncu_traffic_per_launch(wl, 0 if prec_bf16 else 1)
     roof["traffic_captured_at"] = NCU_UPDATE_TRAFFIC["kernel_unchanged_since"] if roof["traffic"] else None
     roof["kernel"] = "update_pair_kernel + label_rows_kernel (sfb_apply_update)" if prec_bf16 \
-        else "sgemm_kernel EPI_RMW (sfb_apply_update)"
+        else "update_pair_kernel<tf32 pairs> (sfb_apply_update)" if tf32 else "sgemm_kernel EPI_RMW (sfb_apply_update)"
     roof["ms"] = ms_u
     roof["peaks"] = "of " + peaks["source"] + (" (sustained tensor figure: timed inside a long step)" if sustained
                                                else " (burst tensor figure: timed alone)")
@@ -349,7 +375,7 @@ def run_sharded(args, wl, rank, world, local):
     if world > 1:
         dist.init_process_group("nccl")
     dev = torch.device("cuda", local)
-    prec = S.PREC_BF16 if args.precision == "bf16" else S.PREC_FP32
+    prec = precision_code(S, args.precision)
     peaks = load_peaks()
     r0, r1 = row_shard_bounds(wl.rows, world, rank)
     W = draw_W(torch, wl, dev, 1234 + rank, rows=r1 - r0)
@@ -396,15 +422,15 @@ def run_sharded(args, wl, rank, world, local):
     if rank == 0:
         value = K * args.steps / (total_ms * 1e-3)                          # one problem: K samples per step in all
         shard = I.scaled(wl, wl.name, rows=r1 - r0)
-        roof = update_roofline(shard, prec == S.PREC_BF16, ms_u, peaks, clocks)
+        roof = update_roofline(shard, prec == S.PREC_BF16, ms_u, peaks, clocks, tf32=runs_tf32(shard, args.precision))
         roof["traffic"] = None
         roof["traffic_captured_at"] = None
         model = exchange_model_bytes(wl.workers, wl.batch, wl.rows, wl.cols, world)
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
-                "scaling": "strong", "vs_baseline": None, "dtype": "bf16" if prec == S.PREC_BF16 else "f32",
+                "scaling": "strong", "vs_baseline": None, "dtype": dtype_name(wl, args.precision),
                 "data": "synthetic",
-                "config": dict(workload_config(wl, "bf16" if prec == S.PREC_BF16 else "f32"),
+                "config": dict(workload_config(wl, dtype_name(wl, args.precision)),
                                parallelism=f"rows{world}", rows_per_rank=r1 - r0),
                 "roofline": roof, "cpu_baseline": None, "e2e": None, "gpu_launches": int(launches), "clocks": clocks,
                 "exchange": {"measured_bytes_received_per_rank": moved.total if moved else 0,
@@ -425,7 +451,9 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="sfb", choices=["sfb", "reference"])
-    ap.add_argument("--precision", default="bf16", choices=["bf16", "fp32"])
+    ap.add_argument("--precision", default="bf16", choices=["bf16", "fp32", "tf32", "ffma"],
+                    help="bf16 operands (default); fp32 = the 1e-5 mode (tensor cores with tf32 pairs at large MLR "
+                         "shapes, FFMA otherwise); tf32 / ffma force either kernel family of that mode")
     ap.add_argument("--workload", default="mlr_large", choices=sorted(I.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--rows", type=int, default=0,
@@ -462,7 +490,7 @@ def main():
     if world > 1:
         dist.init_process_group("nccl")
     dev = torch.device("cuda", local)
-    prec = S.PREC_BF16 if args.precision == "bf16" else S.PREC_FP32
+    prec = precision_code(S, args.precision)
     peaks = load_peaks()
 
     # ---- synthetic state: W drawn on the device; minibatches from the seeded input module (each rank its own
@@ -560,7 +588,8 @@ def main():
         ms_loop = e0.elapsed_time(e1) / reps
         update_loop = {"launches": reps, "ms": ms_loop, "seconds": ms_loop * reps * 1e-3, "clocks": ck,
                        "ms_x_sm_mhz": ms_loop * ck["sm_mhz"] if ck.get("sm_mhz") else None,
-                       "roofline": update_roofline(wl, prec == S.PREC_BF16, ms_loop, peaks, ck)}
+                       "roofline": update_roofline(wl, prec == S.PREC_BF16, ms_loop, peaks, ck,
+                                                   tf32=runs_tf32(wl, args.precision))}
 
     # ---- end to end: host minibatch -> sfb_step_host -> loss back on the host, every step
     for i in range(3):
@@ -586,7 +615,7 @@ def main():
     h2d = K * wl.in_dim * 4 + (K * wl.cols * 4 if wl.model == I.DML else 0) + (K * 4 if wl.model != I.SC else 0)
 
     # ---- roofline of the dominant kernel (the fused update), timed inside the long step: sustained tensor figure
-    roof = update_roofline(wl, prec == S.PREC_BF16, ms_u, peaks, clocks)
+    roof = update_roofline(wl, prec == S.PREC_BF16, ms_u, peaks, clocks, tf32=runs_tf32(wl, args.precision))
     roof_fwd, roof_step = (None, None)
     if prec == S.PREC_BF16 and wl.model == I.MLR:
         roof_fwd, roof_step = forward_and_step_rooflines(wl, ms_f, total_ms / args.steps, roof["roof_ms"], peaks)
@@ -608,8 +637,8 @@ def main():
     one_copy = K * (wl.rows + wl.cols) * esz
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if prec == S.PREC_BF16 else "f32",
-            "data": "synthetic", "config": workload_config(wl, "bf16" if prec == S.PREC_BF16 else "f32"),
+            "scaling": "weak", "vs_baseline": None, "dtype": dtype_name(wl, args.precision),
+            "data": "synthetic", "config": workload_config(wl, dtype_name(wl, args.precision)),
             "roofline": roof, "roofline_forward": roof_fwd, "roofline_step": roof_step, "cpu_baseline": cpu,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 8,
                     "ms_per_step": e2e_ms / e2e_steps, "last_loss": loss},

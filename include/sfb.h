@@ -42,8 +42,14 @@ enum sfb_model { SFB_MLR = 0, SFB_DML = 1, SFB_SC = 2, SFB_L2MLR = 3 };
  *                that cancels, so every product -- the forward W v, the products of the ISTA coder and the update --
  *                runs on the tensor cores with each value carried as a (hi, lo) pair of bf16, three bf16 products
  *                per term (about 2^-16 relative error per product).
- * SFB_PREC_FP32: fp32 operands, fp32 FMA accumulation. */
-enum sfb_precision { SFB_PREC_BF16 = 0, SFB_PREC_FP32 = 1 };
+ * SFB_PREC_FP32: fp32 operands.  MLR and SFB_L2MLR contexts of at least 2048 x 512 with K >= 128 run their two
+ *                products on the tensor cores as SFB_PREC_TF32X3 does; everything else uses fp32 FMA kernels.
+ * SFB_PREC_TF32X3: (MLR, SFB_L2MLR) fp32 operands on the tensor cores at any shape: every fp32 value x is carried as
+ *                two tf32 words, big = tf32(x) and small = tf32(x - big), and a product runs as
+ *                big*big + big*small + small*big with fp32 accumulation (relative error about 2^-21 per product);
+ *                softmax, loss and the factors stay in fp32.  SFB_ERR_UNSUPPORTED for the other models.
+ * SFB_PREC_FP32_FFMA: fp32 FMA kernels at any shape (the on-device cross-check of the tensor-core paths). */
+enum sfb_precision { SFB_PREC_BF16 = 0, SFB_PREC_FP32 = 1, SFB_PREC_TF32X3 = 2, SFB_PREC_FP32_FFMA = 3 };
 
 enum sfb_error {
   SFB_OK = 0,

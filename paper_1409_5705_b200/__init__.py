@@ -12,7 +12,7 @@ import os
 from .build import LIB, build
 
 MLR, DML, SC, L2MLR = 0, 1, 2, 3
-PREC_BF16, PREC_FP32 = 0, 1
+PREC_BF16, PREC_FP32, PREC_TF32X3, PREC_FP32_FFMA = 0, 1, 2, 3
 PROX_NONE, PROX_L1, PROX_L2SQ = 0, 1, 2
 STATUS_LABEL_RANGE, STATUS_TIMEOUT, STATUS_SAMPLE_RANGE = 0x1, 0x2, 0x4
 
@@ -169,7 +169,7 @@ class Context:
                  "sfb_sdca_compute_factors")
 
     def sfb_sdca_step(self, X, labels, sample_ids):
-        self._ck(lib().sfb_sdca_step(self._h, _ptr(X), _ptr(labels), _ptr(sample_ids)), "sfb_sdca_step", "sfb_set_factors", "sfb_set_eta")
+        self._ck(lib().sfb_sdca_step(self._h, _ptr(X), _ptr(labels), _ptr(sample_ids)), "sfb_sdca_step")
 
     def sfb_set_factors(self, worker, U, V):
         """U [B, rows], V [B, cols]: contiguous fp32 CUDA tensors of factors computed elsewhere."""

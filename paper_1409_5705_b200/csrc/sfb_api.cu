@@ -45,7 +45,9 @@ Layout make_layout(const sfb_config& cfg) {
   L.Kp = static_cast<int64_t>(K);
   L.colsb = static_cast<int64_t>(cols);
   L.ldu = static_cast<int64_t>(rows);
-  if (c.precision == SFB_PREC_FP32) {
+  if (use_tf32(cfg)) {
+    tc32_extend_layout(c, L, off);
+  } else if (c.precision != SFB_PREC_BF16) {
     L.V = take(K * cols * 4);
     L.U = take(K * rows * 4);
   } else {
@@ -74,7 +76,8 @@ static int check_config(const sfb_config* c) {
   if (!c) return SFB_ERR_ARG;
   if (c->model < SFB_MLR || c->model > SFB_L2MLR) return SFB_ERR_ARG;
   if (c->model == SFB_L2MLR && (!(c->sdca_lambda > 0.f) || c->sdca_n < 1)) return SFB_ERR_ARG;
-  if (c->precision != SFB_PREC_BF16 && c->precision != SFB_PREC_FP32) return SFB_ERR_ARG;
+  if (c->precision < SFB_PREC_BF16 || c->precision > SFB_PREC_FP32_FFMA) return SFB_ERR_ARG;
+  if (c->precision == SFB_PREC_TF32X3 && c->model != SFB_MLR && c->model != SFB_L2MLR) return SFB_ERR_UNSUPPORTED;
   if (c->rows <= 0 || c->cols <= 0 || c->workers <= 0 || c->batch <= 0) return SFB_ERR_ARG;
   if (c->workers > 64) return SFB_ERR_SHAPE;
   if (c->cols % 4 != 0) return SFB_ERR_SHAPE;
@@ -114,6 +117,8 @@ extern "C" int sfb_init(const sfb_config* cfg, float* W_dev, void* workspace_dev
   sfb_ctx* ctx = new (std::nothrow) sfb_ctx();
   if (!ctx) return SFB_ERR_ARG;
   ctx->cfg = *cfg;
+  ctx->tf32 = use_tf32(*cfg);
+  if (cfg->precision != SFB_PREC_BF16) ctx->cfg.precision = SFB_PREC_FP32;      // one fp32 family; tf32 says which kernels
   ctx->sdca = cfg->model == SFB_L2MLR;
   if (ctx->sdca) ctx->cfg.model = SFB_MLR;            // the products, buffers and the update are those of MLR
   ctx->dualQ = nullptr;
@@ -151,7 +156,7 @@ extern "C" int sfb_init(const sfb_config* cfg, float* W_dev, void* workspace_dev
     ce = set_lipschitz(ctx->stream, ctx->at<Scalars>(lay.scalars), cfg->sc_lipschitz);
     if (ce != cudaSuccess) { sfb_destroy(ctx); return SFB_ERR_CUDA; }
   }
-  if (cfg->precision == SFB_PREC_BF16) {
+  if (cfg->precision == SFB_PREC_BF16 || ctx->tf32) {
     rc = tc_init(ctx);
     if (rc) { sfb_destroy(ctx); return rc; }
   }
@@ -246,8 +251,9 @@ extern "C" int sfb_compute_factors(sfb_ctx* ctx, int32_t worker, const float* X_
   }
   // bf16 mode: every product runs on the tensor cores; DML and SC, whose u comes from a cancelling residual,
   // carry each value as a (hi, lo) pair of bf16 (fp32-class products)
-  rc = c.precision == SFB_PREC_FP32 ? factors_fp32(ctx, off, n, X_dev, Y_dev, labels_dev)
-                                    : tc_factors(ctx, off, n, X_dev, Y_dev, labels_dev);
+  rc = ctx->tf32 ? tc32_factors(ctx, off, n, X_dev, labels_dev, nullptr, 0.f)
+       : c.precision == SFB_PREC_FP32 ? factors_fp32(ctx, off, n, X_dev, Y_dev, labels_dev)
+                                      : tc_factors(ctx, off, n, X_dev, Y_dev, labels_dev);
   if (rc) return rc;
   const uint64_t all = c.workers == 64 ? ~0ull : ((1ull << c.workers) - 1);
   ctx->committed |= worker < 0 ? all : (1ull << worker);
@@ -362,8 +368,8 @@ extern "C" int sfb_gather_factors(sfb_ctx* ctx) {
   CK(cudaEventRecord(ctx->ev[1], ctx->stream));
   // Every worker wrote its pairs at row offset p*B of the shared buffers, so the gathered operands are
   // complete; what remains is the per-step read-out over all K pairs.
-  if (c.precision == SFB_PREC_BF16) {
-    int rc = tc_gather(ctx);
+  if (c.precision == SFB_PREC_BF16 || ctx->tf32) {
+    int rc = ctx->tf32 ? tc32_gather(ctx) : tc_gather(ctx);
     if (rc) return rc;
   }
   if (c.model == SFB_MLR)
@@ -391,7 +397,7 @@ extern "C" int sfb_apply_update(sfb_ctx* ctx) {
   if (!ctx) return SFB_ERR_ARG;
   if (!ctx->gathered) return SFB_ERR_STATE;
   const sfb_config& c = ctx->cfg;
-  int rc = c.precision == SFB_PREC_FP32 ? update_fp32(ctx) : tc_update(ctx);
+  int rc = ctx->tf32 ? tc32_update(ctx) : c.precision == SFB_PREC_FP32 ? update_fp32(ctx) : tc_update(ctx);
   if (rc) return rc;
   ctx->stats.flops += 2.0 * c.rows * c.cols * ctx->K;
   rc = apply_prox(ctx);
@@ -431,7 +437,10 @@ extern "C" int sfb_sdca_compute_factors(sfb_ctx* ctx, int32_t worker, const floa
   const float inv_lam_n = static_cast<float>(1.0 / (static_cast<double>(c.sdca_lambda) * static_cast<double>(c.sdca_n)));
   uint32_t* status = ctx->at<uint32_t>(ctx->lay.status);
   float* loss = ctx->at<float>(ctx->lay.loss) + off;
-  if (c.precision == SFB_PREC_FP32) {
+  if (ctx->tf32) {
+    const int rc = tc32_factors(ctx, off, n, X_dev, labels_dev, sample_ids_dev, inv_lam_n);
+    if (rc) return rc;
+  } else if (c.precision == SFB_PREC_FP32) {
     float* V = ctx->at<float>(ctx->lay.V) + off * c.cols;
     float* U = ctx->at<float>(ctx->lay.U) + off * c.rows;
     CK(pack_copy(ctx->stream, V, X_dev, nullptr, n * c.cols));                                        // v = a_i
@@ -473,7 +482,7 @@ extern "C" int sfb_replay_update(sfb_ctx* ctx) {
   if (ctx->stats.steps < 1 || ctx->committed != 0 || ctx->partials_ready) return SFB_ERR_STATE;
   const sfb_config& c = ctx->cfg;
   CK(cudaEventRecord(ctx->ev[2], ctx->stream));
-  int rc = c.precision == SFB_PREC_FP32 ? update_fp32(ctx) : tc_update(ctx);
+  int rc = ctx->tf32 ? tc32_update(ctx) : c.precision == SFB_PREC_FP32 ? update_fp32(ctx) : tc_update(ctx);
   if (rc) return rc;
   ctx->stats.flops += 2.0 * c.rows * c.cols * ctx->K;
   rc = apply_prox(ctx);

@@ -26,7 +26,7 @@ constexpr int kProxSlabs = 64;        // row slabs of the deterministic column r
 struct Layout {
   size_t status, scalars, loss, V, U, colpart, pib, piy, stageX, stageY, stageL;
   // bf16 tensor-core mode
-  size_t Wb, Xb, VT, ZT, UT, part, Xf, labels, coef;
+  size_t Wb, Xb, VT, ZT, UT, part, Xf, labels, coef, lse;
   // bf16 mode, DML and SC: (hi | lo) bf16 operands of the split products
   size_t Ws, WTs, As, Rs;             // W by rows, W transposed, the A operand (v or the codes), the residual
   int64_t ldu;                        // row pitch of the fp32 U buffer (rows rounded up to 4 in bf16 mode)
@@ -37,6 +37,16 @@ struct Layout {
 };
 
 Layout make_layout(const sfb_config& c);
+
+// fp32 mode runs its products of multiclass logistic regression on the tensor cores (every fp32 value as a pair of
+// tf32 words, three products per term) when asked to, or by itself when the shape is large enough to be worth the
+// operand copies; small shapes and the other models use the FFMA kernels.
+inline bool use_tf32(const sfb_config& c) {
+  const bool mlr = c.model == SFB_MLR || c.model == SFB_L2MLR;
+  if (c.precision == SFB_PREC_TF32X3) return mlr;
+  if (c.precision != SFB_PREC_FP32 || !mlr) return false;
+  return c.rows >= 2048 && c.cols >= 512 && static_cast<int64_t>(c.workers) * c.batch >= 128;
+}
 
 struct Scalars {                      // device-resident scalars
   float loss_mean;
@@ -58,6 +68,7 @@ struct sfb_ctx {
   int64_t row_offset;                 // row-sharded MLR: this context's W holds rows [row_offset, row_offset + rows)
   int64_t global_rows;                //   of a matrix with global_rows rows (class ids are global); 0, rows when unsharded
   bool partials_ready;                // sfb_forward_partials has run since the last update
+  bool tf32;                          // fp32 mode with its products on the tensor cores (see use_tf32)
   bool sdca;                          // SFB_L2MLR: the factors are dual changes; cfg.model is kept as SFB_MLR internally
   float* dualQ;                       // SDCA dual state [dual_n x rows], caller-owned
   int64_t dual_n;

@@ -77,7 +77,9 @@ __device__ __forceinline__ float soft_threshold(float w, float t) {
   return a > 0.f ? copysignf(a, w) : 0.f;
 }
 
-template <int EPI>
+// TF32: the operands are 32-bit words read as tf32 (a k-block of 128 bytes is then 32 elements and one MMA contracts
+// 8 of them); everything else -- stages, descriptors, epilogues -- is the same.
+template <int EPI, bool TF32 = false>
 __global__ void __launch_bounds__(kThreads, 1)
 forward_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmC, const TcParams p) {
@@ -128,8 +130,8 @@ forward_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t s = it % S, ph = (it / S) & 1;
             if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
             mbar_expect_tx(&full[s], kBytesA + p.bn * BK * 2);
-            tma_load_2d_hint(sA + s * kBytesA, &tmA, xa0 + kl * BK, m0, &full[s], pol_keep);
-            tma_load_2d(sB + s * kBytesB, &tmB, xb0 + kl * BK, n0, &full[s]);
+            tma_load_2d_hint(sA + s * kBytesA, &tmA, xa0 + kl * (TF32 ? BK / 2 : BK), m0, &full[s], pol_keep);
+            tma_load_2d(sB + s * kBytesB, &tmB, xb0 + kl * (TF32 ? BK / 2 : BK), n0, &full[s]);
           }
         }
       }
@@ -137,7 +139,7 @@ forward_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
-      const uint32_t idesc = umma_idesc_bf16(BM, p.bn);
+      const uint32_t idesc = TF32 ? umma_idesc_tf32(BM, p.bn) : umma_idesc_bf16(BM, p.bn);
       uint32_t it = 0, tl = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++tl) {
@@ -152,9 +154,11 @@ forward_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const uint64_t da = umma_desc_k128(smem_u32(sA + s * kBytesA));
           const uint64_t db = umma_desc_k128(smem_u32(sB + s * kBytesB));
 #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k)
-            umma_bf16(d_tmem, da + static_cast<uint64_t>(k * UMMA_K * 2 / 16), db + static_cast<uint64_t>(k * UMMA_K * 2 / 16),
-                      idesc, (kb | k) != 0 ? 1u : 0u);
+          for (int k = 0; k < BK / UMMA_K; ++k) {          // four MMAs of 32 bytes of contraction each, either kind
+            const uint64_t adv = static_cast<uint64_t>(k * UMMA_K * 2 / 16);
+            if (TF32) umma_tf32(d_tmem, da + adv, db + adv, idesc, (kb | k) != 0 ? 1u : 0u);
+            else umma_bf16(d_tmem, da + adv, db + adv, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
           umma_commit(&empty[s]);          // the stage is free once these MMAs have read it
         }
         if (ok) umma_commit(&tfull[a]);    // the accumulator is complete once every MMA of the tile is
@@ -567,15 +571,85 @@ __global__ void __launch_bounds__(256) mlr_emit_ut_kernel(const float* __restric
 }
 
 // ---------------------------------------------------------------------------------------------------------
+// fp32 mode on the tensor cores: every fp32 value x is carried as two tf32 words, big = tf32(x) and
+// small = tf32(x - big) (x = big + small to about 2^-22 |x|), and a product runs as big*big + big*small + small*big.
+// ---------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float to_tf32(float x) {
+  uint32_t u;
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(u) : "f"(x));
+  return __uint_as_float(u);
+}
+
+// fp32 [n x dim] (row pitch ld) -> [n x 2*dimp] fp32 words: dst[r][c] = big, dst[r][dimp + c] = small.  Columns
+// dim..dimp-1 keep the zeros of set-up.  dim and ld are multiples of 4.
+__global__ void __launch_bounds__(256) split32_rows_kernel(const float* __restrict__ F, int64_t n, int64_t dim, int64_t ld,
+                                                           float* __restrict__ dst, int64_t dimp) {
+  const int64_t quads = dim / 4, total = n * quads;
+  const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+  for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total; i += stride) {
+    const int64_t r = i / quads, qd = i % quads;
+    const float4 v = *reinterpret_cast<const float4*>(F + r * ld + qd * 4);
+    const float4 b = make_float4(to_tf32(v.x), to_tf32(v.y), to_tf32(v.z), to_tf32(v.w));
+    float* d = dst + r * 2 * dimp + qd * 4;
+    *reinterpret_cast<float4*>(d) = b;
+    *reinterpret_cast<float4*>(d + dimp) = make_float4(to_tf32(v.x - b.x), to_tf32(v.y - b.y), to_tf32(v.z - b.z),
+                                                       to_tf32(v.w - b.w));
+  }
+}
+
+// Gathered fp32 factors F [n x dim] (pair-major, row pitch ld) -> FT [dim x 2*Kp] (pairs contiguous):
+// FT[c][i] = big, FT[c][Kp + i] = small; pairs n..Kp-1 are written as zeros.  64 x 64 tiles through shared memory.
+__global__ void __launch_bounds__(256) split32_t_kernel(const float* __restrict__ F, int64_t n, int64_t dim, int64_t ld,
+                                                        float* __restrict__ FT, int64_t Kp) {
+  __shared__ float tile[64][65];
+  const int64_t i0 = static_cast<int64_t>(blockIdx.y) * 64, c0 = static_cast<int64_t>(blockIdx.x) * 64;
+  const int t = threadIdx.x;
+#pragma unroll
+  for (int v = 0; v < 16; ++v) {
+    const int idx = t + v * 256;            // 64 pairs x 64 columns
+    const int i = idx / 64, c = idx % 64;
+    tile[i][c] = (i0 + i < n && c0 + c < dim) ? F[(i0 + i) * ld + c0 + c] : 0.f;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int v = 0; v < 4; ++v) {
+    const int idx = t + v * 256;            // 64 columns x 16 groups of 4 pairs
+    const int c = idx / 16, ig = (idx % 16) * 4;
+    if (c0 + c >= dim || i0 + ig >= Kp) continue;
+    const float f0 = tile[ig][c], f1 = tile[ig + 1][c], f2 = tile[ig + 2][c], f3 = tile[ig + 3][c];
+    const float4 b = make_float4(to_tf32(f0), to_tf32(f1), to_tf32(f2), to_tf32(f3));
+    float* dst = FT + (c0 + c) * 2 * Kp + i0 + ig;          // Kp is a multiple of 32: 16-byte aligned
+    *reinterpret_cast<float4*>(dst) = b;
+    *reinterpret_cast<float4*>(dst + Kp) = make_float4(to_tf32(f0 - b.x), to_tf32(f1 - b.y), to_tf32(f2 - b.z), to_tf32(f3 - b.w));
+  }
+}
+
+// u_ij = exp(z_ij - lse_i) - [j = y_i], from the logits Z [n x ldz] to the pair-major fp32 factors U [n x rows]
+// (Section 2.1: u = d f / d (W a)).  PLAIN copies Z instead (the dual changes of the SDCA step already are the factors).
+template <bool PLAIN>
+__global__ void __launch_bounds__(256) mlr_finish_u_kernel(const float* __restrict__ Z, int64_t ldz, int64_t rows,
+                                                           const float* __restrict__ lse, const int32_t* __restrict__ labels,
+                                                           float* __restrict__ U) {
+  const int64_t i = blockIdx.y;
+  const float l = PLAIN ? 0.f : lse[i];
+  const int64_t y = PLAIN ? -1 : static_cast<int64_t>(labels[i]);
+  const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+  for (int64_t j = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; j < rows; j += stride) {
+    const float z = Z[i * ldz + j];
+    U[i * rows + j] = PLAIN ? z : expf(z - l) - (j == y ? 1.f : 0.f);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------------------
-template <int EPI>
+template <int EPI, bool TF32 = false>
 cudaError_t launch_forward(sfb_ctx* ctx, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c, TcParams p) {
   const TcState* st = static_cast<const TcState*>(ctx->tc);
   const int64_t tiles = static_cast<int64_t>(p.tilesM) * p.tilesN;
   if (tiles <= 0) return cudaSuccess;
   const int grid = static_cast<int>(tiles < st->sms ? tiles : st->sms);
-  forward_kernel<EPI><<<grid, kThreads, kSmem, ctx->stream>>>(a, b, c, p);
+  forward_kernel<EPI, TF32><<<grid, kThreads, kSmem, ctx->stream>>>(a, b, c, p);
   count_launch();
   return cudaGetLastError();
 }
@@ -587,6 +661,8 @@ cudaError_t prepare_forward_kernels() {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(forward_kernel<F_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(forward_kernel<F_SUB>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(forward_kernel<F_ISTA>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(forward_kernel<F_SOFTMAX, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
   return e;
 }
 
@@ -600,6 +676,28 @@ cudaError_t prepare_forward_kernels() {
       return SFB_ERR_CUDA;                              \
     }                                                   \
   } while (0)
+
+// fp32 mode on the tensor cores (MLR): fp32 pair-major factors as in the FFMA path, plus the (big | small) tf32
+// operands of the two products and the logits.
+void tc32_extend_layout(const sfb_config& c, Layout& L, size_t& off) {
+  auto take = [&](size_t bytes) { size_t o = off; off += (bytes + kAlign - 1) / kAlign * kAlign; return o; };
+  const size_t K = static_cast<size_t>(c.workers) * c.batch;
+  L.Kp = round_up(static_cast<int64_t>(K), 32);
+  L.colsp = round_up(c.cols, 32);
+  const size_t ldz = static_cast<size_t>(round_up(c.rows, 32));
+  const size_t nblk = static_cast<size_t>((c.rows + BN - 1) / BN);
+  L.V = take(K * static_cast<size_t>(c.cols) * 4);
+  L.U = take(K * static_cast<size_t>(c.rows) * 4);
+  L.Ws = take(static_cast<size_t>(c.rows) * 2 * L.colsp * 4);        // W, rows x (big | small)
+  L.As = take(K * 2 * static_cast<size_t>(L.colsp) * 4);             // the samples, K x (big | small)
+  L.VT = take(static_cast<size_t>(c.cols) * 2 * L.Kp * 4);
+  L.UT = take(static_cast<size_t>(c.rows) * 2 * L.Kp * 4);
+  L.ZT = take(K * ldz * 4);
+  L.part = take(nblk * K * 8);
+  L.lse = take(K * 4);
+  L.coef = take(K * 4);
+  L.labels = take(K * 4);
+}
 
 void tc_extend_layout(const sfb_config& c, Layout& L, size_t& off) {
   auto take = [&](size_t bytes) { size_t o = off; off += (bytes + kAlign - 1) / kAlign * kAlign; return o; };
@@ -657,6 +755,13 @@ int tc_init(sfb_ctx* ctx) {
     if (rc) return rc;
   }
   const sfb_config& c = ctx->cfg;
+  if (ctx->tf32) {
+    // pad columns of the split operands are never written by the kernels: clear the buffers once
+    const Layout& L = ctx->lay;
+    CKC(cudaMemsetAsync(ctx->at<char>(L.Ws), 0, static_cast<size_t>(c.rows) * 2 * L.colsp * 4, ctx->stream));
+    CKC(cudaMemsetAsync(ctx->at<char>(L.As), 0, static_cast<size_t>(ctx->K) * 2 * L.colsp * 4, ctx->stream));
+    return SFB_OK;
+  }
   if (c.model != SFB_MLR) {
     // pad columns of the split operands are never written by the kernels: clear the buffers once
     const Layout& L = ctx->lay;
@@ -796,6 +901,81 @@ int factors_split(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const fl
 }
 
 }  // namespace
+
+// fp32 mode on the tensor cores: factors of n MLR samples at pair offset off.  The logits are the three-term tf32
+// product of the (big | small) samples and the (big | small) rows of W; softmax, loss and the factors in fp32.
+// sdca_ids != nullptr: the dual changes of the SDCA step instead of softmax - onehot.
+int tc32_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const int32_t* labels, const int32_t* sdca_ids,
+                 float inv_lam_n) {
+  const sfb_config& c = ctx->cfg;
+  const TcState* st = static_cast<const TcState*>(ctx->tc);
+  const Layout& L = ctx->lay;
+  const int64_t rows = c.rows, cols = c.cols, K = ctx->K;
+  const int64_t ldz = round_up(rows, 32);
+  cudaStream_t s = ctx->stream;
+  float* Ws = ctx->at<float>(L.Ws);
+  float* As = ctx->at<float>(L.As);
+  float* Z = ctx->at<float>(L.ZT);
+  float* V = ctx->at<float>(L.V) + off * cols;
+  float* U = ctx->at<float>(L.U) + off * rows;
+  if (ctx->committed == 0) {
+    // first factors of the step: the (big | small) copy of the W every worker sees (BSP)
+    split32_rows_kernel<<<grid1d(rows * cols / 4, 256), 256, 0, s>>>(ctx->W, rows, cols, cols, Ws, L.colsp);
+    count_launch();
+  }
+  CKC(pack_copy(s, V, X, nullptr, n * cols));                                              // v = x
+  split32_rows_kernel<<<grid1d(n * cols / 4, 256), 256, 0, s>>>(X, n, cols, cols, As + off * 2 * L.colsp, L.colsp);
+  count_launch();
+  CKC(cudaGetLastError());
+  CUtensorMap ma, mb, mc;
+  if (!make_map(st, &ma, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, As, 2 * L.colsp, off + n, 2 * L.colsp * 4, BK / 2, BM) ||
+      !make_map(st, &mb, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, Ws, 2 * L.colsp, rows, 2 * L.colsp * 4, BK / 2, BN) ||
+      !make_map(st, &mc, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, Z, rows, off + n, ldz * 4, kChunk, 32))
+    return SFB_ERR_CUDA;
+  TcParams p{};
+  p.M = static_cast<int32_t>(off + n); p.N = static_cast<int32_t>(rows); p.Kc = static_cast<int32_t>(L.colsp);
+  p.m_off = static_cast<int32_t>(off);
+  p.tilesM = static_cast<int32_t>((n + BM - 1) / BM);
+  p.bn = BN;
+  p.tilesN = static_cast<int32_t>((rows + BN - 1) / BN);
+  p.part = ctx->at<float2>(L.part); p.part_ld = K; p.status = ctx->at<uint32_t>(L.status);
+  p.nseg = 3; p.kseg = static_cast<int32_t>(L.colsp / (BK / 2));          // cross terms first, big*big last
+  p.a_off0 = 0; p.a_off1 = static_cast<int32_t>(L.colsp); p.a_off2 = 0;
+  p.b_off0 = static_cast<int32_t>(L.colsp); p.b_off1 = 0; p.b_off2 = 0;
+  CKC((launch_forward<F_SOFTMAX, true>(ctx, ma, mb, mc, p)));                                // z_i = W x_i
+  ctx->stats.flops += 3.0 * 2.0 * n * rows * cols;
+  dim3 ugrid(static_cast<unsigned>(std::min<int64_t>((rows + 255) / 256, 64)), static_cast<unsigned>(n));
+  if (sdca_ids) {
+    CKC(sdca_dual_rows(s, Z + off * ldz, n, rows, ldz, X, cols, labels, sdca_ids, ctx->dualQ, ctx->dual_n, inv_lam_n, c.eta,
+                       nullptr, ctx->at<float>(L.loss) + off, ctx->at<uint32_t>(L.status)));
+    mlr_finish_u_kernel<true><<<ugrid, 256, 0, s>>>(Z + off * ldz, ldz, rows, nullptr, nullptr, U);
+  } else {
+    float* lse = ctx->at<float>(L.lse);
+    mlr_lse_kernel<<<static_cast<unsigned>((n + 7) / 8), 256, 0, s>>>(ctx->at<float2>(L.part), K, p.tilesN, Z, ldz, rows, labels,
+                                                                     off, n, lse, ctx->at<float>(L.loss),
+                                                                     ctx->at<float>(L.coef), ctx->at<uint32_t>(L.status));
+    count_launch();
+    mlr_finish_u_kernel<false><<<ugrid, 256, 0, s>>>(Z + off * ldz, ldz, rows, lse + off, labels, U);
+  }
+  count_launch();
+  CKC(cudaGetLastError());
+  return SFB_OK;
+}
+
+// The gathered fp32 pairs (computed here or received) become the (big | small) operands of the update product.
+int tc32_gather(sfb_ctx* ctx) {
+  const sfb_config& c = ctx->cfg;
+  const Layout& L = ctx->lay;
+  const unsigned gy = static_cast<unsigned>((L.Kp + 63) / 64);
+  split32_t_kernel<<<dim3(static_cast<unsigned>((c.rows + 63) / 64), gy), 256, 0, ctx->stream>>>(
+      ctx->at<float>(L.U), ctx->K, c.rows, c.rows, ctx->at<float>(L.UT), L.Kp);
+  count_launch();
+  split32_t_kernel<<<dim3(static_cast<unsigned>((c.cols + 63) / 64), gy), 256, 0, ctx->stream>>>(
+      ctx->at<float>(L.V), ctx->K, c.cols, c.cols, ctx->at<float>(L.VT), L.Kp);
+  count_launch();
+  CKC(cudaGetLastError());
+  return SFB_OK;
+}
 
 // Pack of n samples at pair offset off and their logits against the rows of this context's W:
 // Z[off .. off+n) = X W^T with the per-(sample, 256-row block) softmax partials.

@@ -9,6 +9,12 @@ namespace sfb {
 
 // Appends the bf16-mode buffers to the workspace layout.
 void tc_extend_layout(const sfb_config& c, Layout& L, size_t& off);
+// fp32 mode on the tensor cores (MLR and its SDCA form): layout, factors, operand packing of the gathered pairs, update.
+void tc32_extend_layout(const sfb_config& c, Layout& L, size_t& off);
+int tc32_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const int32_t* labels, const int32_t* sdca_ids,
+                 float inv_lam_n);
+int tc32_gather(sfb_ctx* ctx);
+int tc32_update(sfb_ctx* ctx);
 int tc_init(sfb_ctx* ctx);
 void tc_destroy(sfb_ctx* ctx);
 // Rebuilds the bf16 operand copy of W from the caller's fp32 W (MLR; the other models rebuild theirs every step).

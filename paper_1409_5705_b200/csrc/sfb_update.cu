@@ -81,7 +81,8 @@ __device__ __forceinline__ void tile_origin(const UpdParams& p, int tile, int& m
   n0 = tn * UN;
 }
 
-template <bool SHADOW>
+// TF32: the operands are 32-bit words read as tf32 (32 elements per 128-byte k-block), see the forward kernel.
+template <bool SHADOW, bool TF32 = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 update_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                    const __grid_constant__ CUtensorMap tmC, const UpdParams p) {
@@ -137,8 +138,8 @@ update_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
             if (rank == 0) mbar_expect_tx(&full[s], 2 * kStageBytes);
             const uint32_t full_leader = mapa_u32(smem_u32(&full[s]), 0);
-            const int xa = (seg == 0 ? p.a_off0 : seg == 1 ? p.a_off1 : p.a_off2) + kl * UK;
-            const int xb = (seg == 0 ? p.b_off0 : seg == 1 ? p.b_off1 : p.b_off2) + kl * UK;
+            const int xa = (seg == 0 ? p.a_off0 : seg == 1 ? p.a_off1 : p.a_off2) + kl * (TF32 ? UK / 2 : UK);
+            const int xb = (seg == 0 ? p.b_off0 : seg == 1 ? p.b_off1 : p.b_off2) + kl * (TF32 ? UK / 2 : UK);
             tma_load_2d_pair(sA + s * kBytesA, &tmA, xa, m0 + static_cast<int>(rank) * UM, full_leader, pol_norm);
             tma_load_2d_pair(sB + s * kBytesB, &tmB, xb, n0 + static_cast<int>(rank) * (UN / 2), full_leader, pol_keep);
           }
@@ -148,7 +149,7 @@ update_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
   } else if (warp == 1) {
     // ---------------- MMA issuer: one thread of the leader CTA drives both SMs ----------------
     if (lane == 0 && rank == 0) {
-      const uint32_t idesc = umma_idesc_bf16(2 * UM, UN);
+      const uint32_t idesc = TF32 ? umma_idesc_tf32(2 * UM, UN) : umma_idesc_bf16(2 * UM, UN);
       uint32_t it = 0;
       bool ok = true;
       for (int tl = 0; tl < my_tiles && ok; ++tl) {
@@ -163,9 +164,11 @@ update_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
           const uint64_t da = umma_desc_k128(smem_u32(sA + s * kBytesA));
           const uint64_t db = umma_desc_k128(smem_u32(sB + s * kBytesB));
 #pragma unroll
-          for (int k = 0; k < UK / UMMA_K; ++k)
-            umma_bf16_pair(d_tmem, da + static_cast<uint64_t>(k * UMMA_K * 2 / 16),
-                           db + static_cast<uint64_t>(k * UMMA_K * 2 / 16), idesc, (kb | k) != 0 ? 1u : 0u);
+          for (int k = 0; k < UK / UMMA_K; ++k) {          // four MMAs of 32 bytes of contraction each, either kind
+            const uint64_t adv = static_cast<uint64_t>(k * UMMA_K * 2 / 16);
+            if (TF32) umma_tf32_pair(d_tmem, da + adv, db + adv, idesc, (kb | k) != 0 ? 1u : 0u);
+            else umma_bf16_pair(d_tmem, da + adv, db + adv, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
           umma_commit_pair(&empty[s], 3);          // both CTAs' stage s is free once these MMAs have read it
         }
         if (ok) umma_commit_pair(&tfull[a], 3);    // both CTAs' halves of the accumulator are complete
@@ -364,9 +367,9 @@ __global__ void __launch_bounds__(256) label_rows_kernel(float* __restrict__ W, 
     }                                                   \
   } while (0)
 
-template <bool SHADOW>
+template <bool SHADOW, bool TF32 = false>
 static cudaError_t prepare_kernel(int* max_pairs) {
-  cudaError_t e = cudaFuncSetAttribute(update_pair_kernel<SHADOW>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+  cudaError_t e = cudaFuncSetAttribute(update_pair_kernel<SHADOW, TF32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(2, 1, 1);
@@ -378,18 +381,55 @@ static cudaError_t prepare_kernel(int* max_pairs) {
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
   int n = 0;
-  e = cudaOccupancyMaxActiveClusters(&n, update_pair_kernel<SHADOW>, &cfg);
+  e = cudaOccupancyMaxActiveClusters(&n, update_pair_kernel<SHADOW, TF32>, &cfg);
   if (e != cudaSuccess) return e;
   *max_pairs = n;
   return cudaSuccess;
 }
 
 int tc_update_init(sfb_ctx* ctx, TcState* st) {
-  int a = 0, b = 0;
+  int a = 0, b = 0, t = 0;
   CKC(prepare_kernel<true>(&a));
   CKC(prepare_kernel<false>(&b));
-  st->max_pairs = std::min(a, b);
+  CKC((prepare_kernel<false, true>(&t)));
+  st->max_pairs = std::min(std::min(a, b), t);
   if (st->max_pairs < 1) return SFB_ERR_ARCH;     // the device cannot host a CTA pair of this kernel
+  return SFB_OK;
+}
+
+// fp32 mode on the tensor cores (MLR): U^T and V^T are (big | small) pairs of tf32 words, [rows x 2 Kp] and
+// [cols x 2 Kp] with Kp the pair count rounded up to 32;  U^T V = Ub Vb + Ub Vs + Us Vb  (Us Vs, 2^-22 of the product,
+// is dropped).  The label entries are part of U here: no separate label-row pass, no bf16 copy of W.
+int tc32_update(sfb_ctx* ctx) {
+  const sfb_config& c = ctx->cfg;
+  const TcState* st = static_cast<const TcState*>(ctx->tc);
+  const Layout& L = ctx->lay;
+  const int64_t Kp = L.Kp;                                  // a multiple of 32
+  CUtensorMap ma, mb, mc;
+  if (!make_map(st, &ma, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, ctx->at<float>(L.UT), 2 * Kp, c.rows, 2 * Kp * 4, UK / 2, UM) ||
+      !make_map(st, &mb, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, ctx->at<float>(L.VT), 2 * Kp, c.cols, 2 * Kp * 4, UK / 2, UN / 2) ||
+      !make_map(st, &mc, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, ctx->W, c.cols, c.rows, c.cols * 4, kChunk, 32))
+    return SFB_ERR_CUDA;
+  UpdParams p{};
+  p.rows = static_cast<int32_t>(c.rows); p.cols = static_cast<int32_t>(c.cols);
+  p.tilesM = static_cast<int32_t>((c.rows + 2 * UM - 1) / (2 * UM));
+  p.tilesN = static_cast<int32_t>((c.cols + UN - 1) / UN);
+  p.kseg = static_cast<int32_t>(Kp / (UK / 2));
+  p.alpha = -ctx->step;
+  p.prox_kind = ctx->prox_kind; p.prox_a = ctx->prox_a;
+  p.status = ctx->at<uint32_t>(L.status);
+  // The two cross terms first, big*big last: the tensor core rounds its fp32 accumulator at every instruction, by an
+  // amount relative to what the accumulator holds, so the many roundings of the small terms should happen while it is
+  // still small (measured: 3 times less error than with big*big first).
+  p.nseg = 3;
+  p.a_off0 = 0; p.a_off1 = static_cast<int32_t>(Kp); p.a_off2 = 0;
+  p.b_off0 = static_cast<int32_t>(Kp); p.b_off1 = 0; p.b_off2 = 0;
+  p.shadow = nullptr; p.shadow_ld = 0;
+  const int64_t tiles = static_cast<int64_t>(p.tilesM) * p.tilesN;
+  const unsigned grid = 2u * static_cast<unsigned>(std::min<int64_t>(tiles, st->max_pairs));
+  update_pair_kernel<false, true><<<grid, kThreads, kSmem, ctx->stream>>>(ma, mb, mc, p);
+  count_launch();
+  CKC(cudaGetLastError());
   return SFB_OK;
 }
 
