@@ -123,7 +123,8 @@ int sfb_init(const sfb_config* cfg, float* W_dev, void* workspace_dev, size_t wo
  * Factors are written at the worker's row offset p*B of the gathered buffers.  All P workers of a step see the
  * same W (bulk-synchronous consistency, Section 4.1).
  * Copies of W that the library derives: in bf16 mode the forward product reads a bf16 operand copy of W.  DML and SC
- * rebuild theirs from W in the first factors call of every step.  MLR builds it once in sfb_init and afterwards the
+ * rebuild theirs from W in the first factors call of every step.  MLR (and the tensor-core fp32 mode, whose copy is
+ * the pair of tf32 words per entry) builds it once in sfb_init and afterwards the
  * update pass rewrites it together with W (W makes one trip through the SM per step), so it tracks every change the
  * LIBRARY makes to W -- but not writes the caller makes to W_dev between steps (loading weights, rescaling, a prox of
  * its own): after such a write call sfb_refresh_operands, or the next forward product runs on the stale copy. */
@@ -181,7 +182,8 @@ int sfb_apply_update(sfb_ctx* ctx);
 
 /* Re-derives the library's operand copies of W from the caller's W_dev (enqueued on the stream): to be called after
  * the caller itself has written W_dev between two steps.  MLR in bf16 mode: one conversion pass over W (reads 4,
- * writes 2 bytes per entry); a no-op for the other models and for fp32 mode.  SFB_ERR_STATE in the middle of a step. */
+ * writes 2 bytes per entry; 8 bytes in the tensor-core fp32 mode); a no-op for the other models and for the FFMA
+ * kernels.  SFB_ERR_STATE in the middle of a step. */
 int sfb_refresh_operands(sfb_ctx* ctx);
 
 /* Measurement hook (the paper has no counterpart): applies the factors gathered by the last completed step once

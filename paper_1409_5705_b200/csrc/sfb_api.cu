@@ -473,7 +473,7 @@ extern "C" int sfb_sdca_step(sfb_ctx* ctx, const float* X_dev, const int32_t* la
 extern "C" int sfb_refresh_operands(sfb_ctx* ctx) {
   if (!ctx) return SFB_ERR_ARG;
   if (ctx->committed != 0 || ctx->partials_ready) return SFB_ERR_STATE;      // not in the middle of a step
-  if (ctx->cfg.precision != SFB_PREC_BF16) return SFB_OK;                     // fp32 mode reads W itself
+  if (ctx->cfg.precision != SFB_PREC_BF16 && !ctx->tf32) return SFB_OK;       // the FFMA kernels read W itself
   return tc_refresh_operands(ctx);
 }
 

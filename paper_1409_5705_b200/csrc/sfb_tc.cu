@@ -760,7 +760,7 @@ int tc_init(sfb_ctx* ctx) {
     const Layout& L = ctx->lay;
     CKC(cudaMemsetAsync(ctx->at<char>(L.Ws), 0, static_cast<size_t>(c.rows) * 2 * L.colsp * 4, ctx->stream));
     CKC(cudaMemsetAsync(ctx->at<char>(L.As), 0, static_cast<size_t>(ctx->K) * 2 * L.colsp * 4, ctx->stream));
-    return SFB_OK;
+    return tc_refresh_operands(ctx);
   }
   if (c.model != SFB_MLR) {
     // pad columns of the split operands are never written by the kernels: clear the buffers once
@@ -782,6 +782,13 @@ int tc_refresh_operands(sfb_ctx* ctx) {
   const sfb_config& c = ctx->cfg;
   if (c.model != SFB_MLR) return SFB_OK;          // the split copies of W are rebuilt by the first factors call of a step
   const TcState* st = static_cast<const TcState*>(ctx->tc);
+  if (ctx->tf32) {
+    split32_rows_kernel<<<static_cast<unsigned>(st->sms * 16), 256, 0, ctx->stream>>>(ctx->W, c.rows, c.cols, c.cols,
+                                                                                     ctx->at<float>(ctx->lay.Ws), ctx->lay.colsp);
+    count_launch();
+    CKC(cudaGetLastError());
+    return SFB_OK;
+  }
   convert_rows_kernel<<<st->sms * 8, 256, 0, ctx->stream>>>(ctx->W, c.rows, c.cols, ctx->at<__nv_bfloat16>(ctx->lay.Wb),
                                                             ctx->lay.colsb);
   count_launch();
@@ -918,11 +925,7 @@ int tc32_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const int
   float* Z = ctx->at<float>(L.ZT);
   float* V = ctx->at<float>(L.V) + off * cols;
   float* U = ctx->at<float>(L.U) + off * rows;
-  if (ctx->committed == 0) {
-    // first factors of the step: the (big | small) copy of the W every worker sees (BSP)
-    split32_rows_kernel<<<grid1d(rows * cols / 4, 256), 256, 0, s>>>(ctx->W, rows, cols, cols, Ws, L.colsp);
-    count_launch();
-  }
+  // Ws, the (big | small) copy of W, is built at set-up and rewritten by the update's epilogue together with W
   CKC(pack_copy(s, V, X, nullptr, n * cols));                                              // v = x
   split32_rows_kernel<<<grid1d(n * cols / 4, 256), 256, 0, s>>>(X, n, cols, cols, As + off * 2 * L.colsp, L.colsp);
   count_launch();

@@ -57,9 +57,17 @@ struct UpdParams {
   int32_t prox_kind;           // entry-wise prox applied to the updated value (0 none, 1 soft-threshold, 2 scale)
   float prox_a;
   __nv_bfloat16* shadow;       // bf16 copy of the updated W (or null), row pitch shadow_ld elements
+  float* shadow32;             // (big | small) tf32 copy of the updated W: big at column c, small at shadow_half + c
   int64_t shadow_ld;
+  int64_t shadow_half;
   uint32_t* status;
 };
+
+__device__ __forceinline__ float to_tf32(float x) {
+  uint32_t u;
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(u) : "f"(x));
+  return __uint_as_float(u);
+}
 
 __device__ __forceinline__ uint32_t pack2(float a, float b) {
   __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
@@ -82,7 +90,9 @@ __device__ __forceinline__ void tile_origin(const UpdParams& p, int tile, int& m
 }
 
 // TF32: the operands are 32-bit words read as tf32 (32 elements per 128-byte k-block), see the forward kernel.
-template <bool SHADOW, bool TF32 = false>
+// SHADOW: the operand copy of the new W that the epilogue writes beside it for the next forward product:
+// 0 none, 1 bf16, 2 the (big | small) pair of tf32 words of the fp32-on-tensor-cores mode.
+template <int SHADOW, bool TF32 = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 update_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                    const __grid_constant__ CUtensorMap tmC, const UpdParams p) {
@@ -245,7 +255,24 @@ update_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
           if (g >= kPend) tma_wait_group_read<kPend>();      // the store of chunk g-kPend has read its slot:
           issue_load();                                      // refill it with chunk g + kRing - kPend
         }
-        if (SHADOW) {
+        if (SHADOW == 2) {
+          // (big | small) tf32 copy of the chunk, read back from the slot with 8 lanes per row: 128-byte row pieces
+          const int sub = lane >> 3, jj = lane & 7;
+#pragma unroll
+          for (int r0 = 0; r0 < 32; r0 += 4) {
+            const int r = r0 + sub;
+            const float4 w = *reinterpret_cast<const float4*>(sl + r * 128 + ((jj ^ (r & 7)) << 4));
+            const int col = x0 + 4 * jj;
+            if (y0 + r < p.rows && col < p.cols) {
+              const float4 b = make_float4(to_tf32(w.x), to_tf32(w.y), to_tf32(w.z), to_tf32(w.w));
+              float* d = p.shadow32 + static_cast<int64_t>(y0 + r) * p.shadow_ld + col;
+              *reinterpret_cast<float4*>(d) = b;
+              *reinterpret_cast<float4*>(d + p.shadow_half) =
+                  make_float4(to_tf32(w.x - b.x), to_tf32(w.y - b.y), to_tf32(w.z - b.z), to_tf32(w.w - b.w));
+            }
+          }
+        }
+        if (SHADOW == 1) {
           // bf16 copy of the chunk, read back from the slot with 8 lanes per row (4 rows per pass): each row's
           // 32 values leave as one 64-byte piece instead of 32 lanes storing 16 bytes to 32 different rows.
           const int sub = lane >> 3, jj = lane & 7;
@@ -367,7 +394,7 @@ __global__ void __launch_bounds__(256) label_rows_kernel(float* __restrict__ W, 
     }                                                   \
   } while (0)
 
-template <bool SHADOW, bool TF32 = false>
+template <int SHADOW, bool TF32 = false>
 static cudaError_t prepare_kernel(int* max_pairs) {
   cudaError_t e = cudaFuncSetAttribute(update_pair_kernel<SHADOW, TF32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
   if (e != cudaSuccess) return e;
@@ -389,9 +416,9 @@ static cudaError_t prepare_kernel(int* max_pairs) {
 
 int tc_update_init(sfb_ctx* ctx, TcState* st) {
   int a = 0, b = 0, t = 0;
-  CKC(prepare_kernel<true>(&a));
-  CKC(prepare_kernel<false>(&b));
-  CKC((prepare_kernel<false, true>(&t)));
+  CKC(prepare_kernel<1>(&a));
+  CKC(prepare_kernel<0>(&b));
+  CKC((prepare_kernel<2, true>(&t)));
   st->max_pairs = std::min(std::min(a, b), t);
   if (st->max_pairs < 1) return SFB_ERR_ARCH;     // the device cannot host a CTA pair of this kernel
   return SFB_OK;
@@ -424,10 +451,11 @@ int tc32_update(sfb_ctx* ctx) {
   p.nseg = 3;
   p.a_off0 = 0; p.a_off1 = static_cast<int32_t>(Kp); p.a_off2 = 0;
   p.b_off0 = static_cast<int32_t>(Kp); p.b_off1 = 0; p.b_off2 = 0;
-  p.shadow = nullptr; p.shadow_ld = 0;
+  // the epilogue also writes the (big | small) copy of the new W, the operand of the next forward product
+  p.shadow = nullptr; p.shadow32 = ctx->at<float>(L.Ws); p.shadow_ld = 2 * L.colsp; p.shadow_half = L.colsp;
   const int64_t tiles = static_cast<int64_t>(p.tilesM) * p.tilesN;
   const unsigned grid = 2u * static_cast<unsigned>(std::min<int64_t>(tiles, st->max_pairs));
-  update_pair_kernel<false, true><<<grid, kThreads, kSmem, ctx->stream>>>(ma, mb, mc, p);
+  update_pair_kernel<2, true><<<grid, kThreads, kSmem, ctx->stream>>>(ma, mb, mc, p);
   count_launch();
   CKC(cudaGetLastError());
   return SFB_OK;
@@ -461,7 +489,7 @@ int tc_update(sfb_ctx* ctx) {
     p.a_off0 = 0; p.a_off1 = 0; p.a_off2 = static_cast<int32_t>(L.Kp);
     p.b_off0 = 0; p.b_off1 = static_cast<int32_t>(L.Kp); p.b_off2 = 0;
     p.shadow = nullptr; p.shadow_ld = 0;
-    update_pair_kernel<false><<<grid, kThreads, kSmem, ctx->stream>>>(ma, mb, mc, p);
+    update_pair_kernel<0><<<grid, kThreads, kSmem, ctx->stream>>>(ma, mb, mc, p);
     count_launch();
     CKC(cudaGetLastError());
     return SFB_OK;
@@ -479,7 +507,7 @@ int tc_update(sfb_ctx* ctx) {
           ctx->W, c.rows, c.cols, ctx->at<float>(L.Xf), ctx->at<int32_t>(L.labels), ctx->at<float>(L.coef),
           static_cast<int>(ctx->K), ctx->step, labels_first ? nullptr : ctx->at<__nv_bfloat16>(L.Wb), L.colsb);
     } else {
-      update_pair_kernel<true><<<grid, kThreads, kSmem, ctx->stream>>>(ma, mb, mc, p);     // W += -eta * P^T V
+      update_pair_kernel<1><<<grid, kThreads, kSmem, ctx->stream>>>(ma, mb, mc, p);     // W += -eta * P^T V
     }
     count_launch();
     CKC(cudaGetLastError());

@@ -105,8 +105,10 @@ def test_zero_matrix_mlr_matches_the_closed_form_in_bf16():
     assert np.linalg.norm(Wg - ref) / np.linalg.norm(ref) <= TOL[S.PREC_BF16]
 
 
-def test_caller_writes_to_W_between_steps_need_a_refresh_of_the_bf16_operand():
-    """MLR in bf16 mode keeps a bf16 copy of W for the forward product.  The library keeps it current through its own
+@pytest.mark.parametrize("prec", [pytest.param(S.PREC_BF16, id="bf16"), pytest.param(S.PREC_TF32X3, id="tf32x3")])
+def test_caller_writes_to_W_between_steps_need_a_refresh_of_the_operand_copy(prec):
+    """MLR keeps an operand copy of W for the forward product (bf16, or the pair of tf32 words of the tensor-core
+    fp32 mode).  The library keeps it current through its own
     updates; after the CALLER rewrites W, sfb_refresh_operands brings it up to date: the next step is then the oracle's
     step from the new W.  Without the refresh the forward runs on the old copy, which this test also shows."""
     wl = I.scaled(I.WORKLOADS["mlr_mid"], "mlr_refresh", rows=300, cols=260, workers=2, batch=64, eta=0.05,
@@ -116,9 +118,10 @@ def test_caller_writes_to_W_between_steps_need_a_refresh_of_the_bf16_operand():
     inp0, inp1 = I.step_inputs(wl, 0), I.step_inputs(wl, 1)
     ref = oracle_step(wl, W1, inp1)
     errs = {}
+    tol = TOL[S.PREC_BF16] if prec == S.PREC_BF16 else TOL[S.PREC_FP32]
     for refresh in (True, False):
         W = to_dev(W0, torch)
-        ctx = S.Context(config_for(wl, S.PREC_BF16), W)
+        ctx = S.Context(config_for(wl, prec), W)
         ctx.sfb_step(to_dev(inp0.X, torch), None, to_dev(inp0.labels, torch))
         W.copy_(torch.from_numpy(W1))                          # the caller's own write to W
         if refresh:
@@ -127,5 +130,5 @@ def test_caller_writes_to_W_between_steps_need_a_refresh_of_the_bf16_operand():
         assert ctx.sfb_get_status() == 0
         errs[refresh] = rel_err(W.cpu().numpy(), ref, W1)
         ctx.close()
-    assert errs[True] <= TOL[S.PREC_BF16], errs
+    assert errs[True] <= tol, errs
     assert errs[False] > 10 * TOL[S.PREC_BF16], errs           # the stale copy gives another step altogether

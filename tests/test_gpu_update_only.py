@@ -50,6 +50,8 @@ def test_update_matrix_alone_meets_the_stated_tolerance(name, prec):
     print(f"{name}: update-only rel err {err:.3e} (tol {TOL[prec]})")
     assert err <= TOL[prec]
     # entry-wise: nothing is absorbed by a large W, so every entry is held to the tolerance, relative to its own size
-    # plus 16 rms entries of the update (label rows of MLR carry entries a hundred times the rms)
+    # plus 16 rms entries of its row of the update (the rows of frequent classes of MLR sum a hundred terms a hundred
+    # times the matrix rms, and an fp32 accumulator rounds relative to what it holds)
     rms = np.sqrt((ref * ref).mean())
-    assert (np.abs(dW - ref) - TOL[prec] * np.abs(ref)).max() <= 16 * TOL[prec] * rms
+    rms_row = np.maximum(np.sqrt((ref * ref).mean(axis=1, keepdims=True)), rms)
+    assert ((np.abs(dW - ref) - TOL[prec] * np.abs(ref)) / rms_row).max() <= 16 * TOL[prec]
