@@ -226,8 +226,8 @@ def run_reference(args, wl, rank):
 # profiles/ncu_update_pair_kernel_mlr_rows16384.md (a slab of 16384 rows of the paper-scale MLR shape; traffic is
 # proportional to the rows, see that file).  "kernel_unchanged_since" names the commit of csrc/sfb_update.cu the
 # counters were taken at: when the kernel is edited this entry has to be re-captured or set to None.
-NCU_UPDATE_TRAFFIC = {"rows": 16384, "cols": 10000, "K": 1024, "bytes": 764645888 + 933098496,
-                      "kernel_unchanged_since": "cf145f9"}
+NCU_UPDATE_TRAFFIC = {"rows": 16384, "cols": 10000, "K": 1024, "bytes": 758433280 + 932738048,
+                      "kernel_unchanged_since": "1339426"}
 
 
 def ncu_traffic_per_launch(wl, prec):
