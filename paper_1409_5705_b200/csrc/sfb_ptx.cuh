@@ -81,6 +81,12 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, const void* s
                ::"l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(src)), "r"(x), "r"(y)
                : "memory");
 }
+// Asks L2 to fetch the box at (x, y) of a tiled tensor ahead of the load that will want it (no shared memory, no
+// barrier: a hint).  Same alignment rule for x as the loads.
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* m, int32_t x, int32_t y) {
+  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
+               ::"l"(reinterpret_cast<uint64_t>(m)), "r"(x), "r"(y) : "memory");
+}
 // L2 eviction-priority policy for TMA traffic: operands that every tile re-reads stay.
 __device__ __forceinline__ uint64_t policy_evict_last() {
   uint64_t pol;

@@ -17,6 +17,10 @@
 #include "sfb_ptx.cuh"
 #include "sfb_tc.h"
 
+#ifndef SFB_SPLIT_PREFETCH
+#define SFB_SPLIT_PREFETCH 4
+#endif
+
 namespace sfb {
 namespace {
 
@@ -35,7 +39,8 @@ constexpr int kBars = 2 * S + 4;
 constexpr int kSmem = S * (kBytesA + kBytesB) + kEpiWarps * R * kSlotBytes + kBars * 8 + 16 + 1024;
 
 // Epilogues of the product  D (samples x N) = A * B^T:
-//   F_SOFTMAX  store D as fp32 logits and the per (sample, 256-column block) softmax partials      (MLR)
+//   F_SOFTMAX  store D as fp32 logits and the per (sample, 256-column block) softmax partials      (MLR; forward_kernel)
+// and, in forward_split_kernel:
 //   F_STORE    store D as fp32                                                                     (DML: z = W v)
 //   F_SUB      store D - aux as fp32 and as a (hi | lo) bf16 pair                                  (SC: r = W a - x)
 //   F_ISTA     C <- soft(C - D / L, lambda / L) in place, also as a (hi | lo) bf16 pair            (SC: ISTA step)
@@ -56,6 +61,7 @@ struct TcParams {
   int64_t part_ld;
   const float* aux;            // F_SUB: the matrix subtracted, [M x ldaux]; F_ISTA: the matrix updated, [M x ldaux]
   int64_t ldaux;
+  int32_t prefetch;            // k-blocks by which the producer asks L2 for the B operand ahead of its loads (0: off)
   const Scalars* sc;           // F_ISTA: 1 / L
   float lam;                   // F_ISTA: lambda
   __nv_bfloat16* split;        // F_SUB, F_ISTA: [M x ld_split] receives hi at column n and lo at column split_half + n
@@ -129,6 +135,10 @@ forward_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int kl = 0; kl < p.kseg; ++kl, ++it) {
             const uint32_t s = it % S, ph = (it / S) & 1;
             if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
+            // B streams from HBM when it is larger than L2: with the box asked for a few k-blocks early, the load
+            // that fills the stage finds it in L2 and the four stages cover the latency
+            if (p.prefetch > 0 && kl + p.prefetch < p.kseg)
+              tma_prefetch_2d(&tmB, xb0 + (kl + p.prefetch) * (TF32 ? BK / 2 : BK), n0);
             mbar_expect_tx(&full[s], kBytesA + p.bn * BK * 2);
             tma_load_2d_hint(sA + s * kBytesA, &tmA, xa0 + kl * (TF32 ? BK / 2 : BK), m0, &full[s], pol_keep);
             tma_load_2d(sB + s * kBytesB, &tmB, xb0 + kl * (TF32 ? BK / 2 : BK), n0, &full[s]);
@@ -202,51 +212,6 @@ forward_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               sum = sum * __expf(mx - nm) + cs;
               mx = nm;
             }
-            if constexpr (EPI == F_SUB || EPI == F_ISTA) {
-              // the sample's 32 values of aux (x, or the current code a) are contiguous: 128 bytes per lane
-              float xv[32];
-              const float* ap = p.aux + static_cast<int64_t>(row) * p.ldaux + col0;
-              const bool vec = row < p.M && col0 + 32 <= p.N && ((reinterpret_cast<uintptr_t>(ap) & 15u) == 0);
-              if (vec) {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                  const float4 v4 = *reinterpret_cast<const float4*>(ap + 4 * j);
-                  xv[4 * j] = v4.x; xv[4 * j + 1] = v4.y; xv[4 * j + 2] = v4.z; xv[4 * j + 3] = v4.w;
-                }
-              } else {
-#pragma unroll
-                for (int j = 0; j < 32; ++j) xv[j] = (row < p.M && col0 + j < p.N) ? ap[j] : 0.f;
-              }
-              float invL = 0.f, thr = 0.f;
-              if (EPI == F_ISTA) { invL = p.sc->invL; thr = p.lam * invL; }
-#pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                const float d = __uint_as_float(acc[j]);
-                const float v = EPI == F_SUB ? d - xv[j] : soft_threshold(fmaf(-d, invL, xv[j]), thr);
-                acc[j] = __float_as_uint((row < p.M && col0 + j < p.N) ? v : 0.f);
-              }
-              if (row < p.M) {
-                // (hi | lo) bf16 pair of the result: the operand of the next product
-                __nv_bfloat16* hp = p.split + static_cast<int64_t>(row) * p.ld_split + col0;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  if (col0 + 8 * j < p.split_half) {
-                    uint32_t hi[4], lo[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                      const float f0 = __uint_as_float(acc[8 * j + 2 * e]), f1 = __uint_as_float(acc[8 * j + 2 * e + 1]);
-                      const __nv_bfloat16 h0 = __float2bfloat16_rn(f0), h1 = __float2bfloat16_rn(f1);
-                      hi[e] = static_cast<uint32_t>(__bfloat16_as_ushort(h0)) |
-                              (static_cast<uint32_t>(__bfloat16_as_ushort(h1)) << 16);
-                      const __nv_bfloat162 l2 = __floats2bfloat162_rn(f0 - __bfloat162float(h0), f1 - __bfloat162float(h1));
-                      lo[e] = *reinterpret_cast<const uint32_t*>(&l2);
-                    }
-                    *reinterpret_cast<uint4*>(hp + 8 * j) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                    *reinterpret_cast<uint4*>(hp + p.split_half + 8 * j) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-                  }
-                }
-              }
-            }
             if (lane == 0) tma_wait_group_read<R - 1>();   // the store that last used this slot has read it
             __syncwarp();
 #pragma unroll
@@ -277,6 +242,204 @@ forward_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __syncthreads();
   if (*abort_flag) {
     // A wait ran out: report it, give copies in flight a bounded time to land, then release TMEM.
+    if (threadIdx.x == 0) atomicOr(p.status, SFB_STATUS_TIMEOUT);
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, kTmemCols); }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Split-bf16 products of distance metric learning and sparse coding:  D (samples x N) = A * B^T  with both operands
+// stored as [hi | lo] bf16 halves,  A_hi B_hi + A_lo B_hi + A_hi B_lo  (fp32-class accuracy; A_lo B_lo, 2^-16 of the
+// product, is dropped).  One pipeline stage holds the k-block of all four halves, and the three products of that
+// k-block are issued from it: 72 KB of operands per three k-blocks of tensor work instead of 108 KB when the three
+// products run as separate passes over the contraction (these products are bound by their operand loads: a 128 x 160
+// tile takes 36 KB per 320 cycles of MMA).  Three stages of 72 KB fill the shared memory, so the epilogue writes its
+// results straight from registers (the outputs are small: samples x N).
+// Roles as in forward_kernel: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-5 epilogue.
+// ---------------------------------------------------------------------------------------------------------
+constexpr int FS_BN = 160;                          // widest tile of this kernel (columns of the accumulator)
+constexpr int FS_STAGES = 3;
+constexpr int kFsBytesB = FS_BN * BK * 2;           // 20 KB
+constexpr int kFsStage = 2 * kBytesA + 2 * kFsBytesB;
+constexpr int kFsBars = 2 * FS_STAGES + 4;
+constexpr int kFsSmem = FS_STAGES * kFsStage + kFsBars * 8 + 16 + 1024;
+
+template <int EPI>
+__global__ void __launch_bounds__(kThreads, 1)
+forward_split_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, float* __restrict__ C,
+                     int64_t ldc, const TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + FS_STAGES * kFsStage);
+  uint64_t* full = bars;
+  uint64_t* empty = bars + FS_STAGES;
+  uint64_t* tfull = bars + 2 * FS_STAGES;
+  uint64_t* tempty = bars + 2 * FS_STAGES + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kFsBars);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int ntiles = p.tilesM * p.tilesN;
+  const int numK = p.kseg;                          // k-blocks of the contraction (each serves three products)
+  const int a_hi = p.a_off0, a_lo = p.a_off2, b_hi = p.b_off0, b_lo = p.b_off1;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < FS_STAGES; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&tfull[i], 1); mbar_init(&tempty[i], 4); }
+    *abort_flag = 0;
+    fence_barrier_init();
+    prefetch_tmap(&tmA); prefetch_tmap(&tmB);
+  }
+  if (warp == 1) { tmem_alloc(tmem_slot, kTmemCols); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer: the four operand halves of a k-block per stage ----------------
+    if (lane == 0) {
+      const uint64_t pol_keep = policy_evict_last();
+      const uint32_t stage_bytes = 2 * kBytesA + 2 * static_cast<uint32_t>(p.bn) * BK * 2;
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+        int m0, n0;
+        tile_coords(p, tile, m0, n0);
+        for (int kl = 0; kl < numK; ++kl, ++it) {
+          const uint32_t s = it % FS_STAGES, ph = (it / FS_STAGES) & 1;
+          if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
+          if (p.prefetch > 0 && kl + p.prefetch < numK) {          // B streams from HBM when it is larger than L2
+            tma_prefetch_2d(&tmB, b_hi + (kl + p.prefetch) * BK, n0);
+            tma_prefetch_2d(&tmB, b_lo + (kl + p.prefetch) * BK, n0);
+          }
+          uint8_t* st = smem + s * kFsStage;
+          mbar_expect_tx(&full[s], stage_bytes);
+          tma_load_2d_hint(st, &tmA, a_hi + kl * BK, m0, &full[s], pol_keep);
+          tma_load_2d_hint(st + kBytesA, &tmA, a_lo + kl * BK, m0, &full[s], pol_keep);
+          tma_load_2d(st + 2 * kBytesA, &tmB, b_hi + kl * BK, n0, &full[s]);
+          tma_load_2d(st + 2 * kBytesA + kFsBytesB, &tmB, b_lo + kl * BK, n0, &full[s]);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer: three products per stage ----------------
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_bf16(BM, p.bn);
+      uint32_t it = 0, tl = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++tl) {
+        const uint32_t a = tl & 1, aph = (tl >> 1) & 1;
+        if (!mbar_wait(&tempty[a], aph ^ 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + a * BN;
+        for (int kb = 0; kb < numK; ++kb, ++it) {
+          const uint32_t s = it % FS_STAGES, ph = (it / FS_STAGES) & 1;
+          if (!mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          uint8_t* st = smem + s * kFsStage;
+          const uint64_t dah = umma_desc_k128(smem_u32(st));
+          const uint64_t dal = umma_desc_k128(smem_u32(st + kBytesA));
+          const uint64_t dbh = umma_desc_k128(smem_u32(st + 2 * kBytesA));
+          const uint64_t dbl = umma_desc_k128(smem_u32(st + 2 * kBytesA + kFsBytesB));
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            const uint64_t adv = static_cast<uint64_t>(k * UMMA_K * 2 / 16);
+            umma_bf16(d_tmem, dal + adv, dbh + adv, idesc, (kb | k) != 0 ? 1u : 0u);     // A_lo B_hi
+            umma_bf16(d_tmem, dah + adv, dbl + adv, idesc, 1u);                          // A_hi B_lo
+            umma_bf16(d_tmem, dah + adv, dbh + adv, idesc, 1u);                          // A_hi B_hi
+          }
+          umma_commit(&empty[s]);
+        }
+        if (ok) umma_commit(&tfull[a]);
+      }
+    }
+  } else {
+    // ---------------- epilogue: warps 2..5, TMEM lane quarter q; results leave straight from registers ----------------
+    const int q = warp & 3;
+    const int my_tiles = blockIdx.x < ntiles ? (ntiles - 1 - blockIdx.x) / gridDim.x + 1 : 0;
+    bool ok = true;
+    float invL = 0.f, thr = 0.f;
+    if (EPI == F_ISTA) { invL = p.sc->invL; thr = p.lam * invL; }
+    for (int tl = 0; tl < my_tiles && ok; ++tl) {
+      int m0, n0;
+      tile_coords(p, blockIdx.x + tl * gridDim.x, m0, n0);
+      const uint32_t a = tl & 1, aph = (tl >> 1) & 1;
+      if (!__all_sync(0xffffffffu, mbar_wait(&tfull[a], aph, abort_flag))) { ok = false; break; }
+      tc_fence_after();
+      const int row = m0 + q * 32 + lane;
+      for (int c = 0; c < p.bn / kChunk; ++c) {
+        uint32_t acc[32];
+        tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + a * BN + c * kChunk, acc);
+        tmem_ld_wait();
+        const int col0 = n0 + c * kChunk;
+        if (col0 >= p.N || row >= p.M) continue;
+        const bool whole = col0 + 32 <= p.N;
+        if constexpr (EPI == F_SUB || EPI == F_ISTA) {
+          // the sample's 32 values of aux (x, or the current code a) are contiguous: 128 bytes per lane
+          float xv[32];
+          const float* ap = p.aux + static_cast<int64_t>(row) * p.ldaux + col0;
+          if (whole && ((reinterpret_cast<uintptr_t>(ap) & 15u) == 0)) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const float4 v4 = *reinterpret_cast<const float4*>(ap + 4 * j);
+              xv[4 * j] = v4.x; xv[4 * j + 1] = v4.y; xv[4 * j + 2] = v4.z; xv[4 * j + 3] = v4.w;
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) xv[j] = col0 + j < p.N ? ap[j] : 0.f;
+          }
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const float d = __uint_as_float(acc[j]);
+            const float v = EPI == F_SUB ? d - xv[j] : soft_threshold(fmaf(-d, invL, xv[j]), thr);
+            acc[j] = __float_as_uint(col0 + j < p.N ? v : 0.f);
+          }
+          // (hi | lo) bf16 pair of the result: the operand of the next product
+          __nv_bfloat16* hp = p.split + static_cast<int64_t>(row) * p.ld_split + col0;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            if (col0 + 8 * j < p.split_half) {
+              uint32_t hi[4], lo[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float f0 = __uint_as_float(acc[8 * j + 2 * e]), f1 = __uint_as_float(acc[8 * j + 2 * e + 1]);
+                const __nv_bfloat16 h0 = __float2bfloat16_rn(f0), h1 = __float2bfloat16_rn(f1);
+                hi[e] = static_cast<uint32_t>(__bfloat16_as_ushort(h0)) |
+                        (static_cast<uint32_t>(__bfloat16_as_ushort(h1)) << 16);
+                const __nv_bfloat162 l2 = __floats2bfloat162_rn(f0 - __bfloat162float(h0), f1 - __bfloat162float(h1));
+                lo[e] = *reinterpret_cast<const uint32_t*>(&l2);
+              }
+              *reinterpret_cast<uint4*>(hp + 8 * j) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+              *reinterpret_cast<uint4*>(hp + p.split_half + 8 * j) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+            }
+          }
+        }
+        // the fp32 result: this lane's 32 consecutive columns of its row
+        float* cp = C + static_cast<int64_t>(row) * ldc + col0;
+        if (whole && ((reinterpret_cast<uintptr_t>(cp) & 15u) == 0)) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            *reinterpret_cast<uint4*>(cp + 4 * j) = make_uint4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (col0 + j < p.N) cp[j] = __uint_as_float(acc[j]);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tempty[a]);
+    }
+  }
+
+  // ---------------- teardown ----------------
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
     if (threadIdx.x == 0) atomicOr(p.status, SFB_STATUS_TIMEOUT);
     for (int i = 0; i < 64; ++i) __nanosleep(1000);
     __syncthreads();
@@ -654,13 +817,24 @@ cudaError_t launch_forward(sfb_ctx* ctx, const CUtensorMap& a, const CUtensorMap
   return cudaGetLastError();
 }
 
+template <int EPI>
+cudaError_t launch_forward_split(sfb_ctx* ctx, const CUtensorMap& a, const CUtensorMap& b, float* C, int64_t ldc, TcParams p) {
+  const TcState* st = static_cast<const TcState*>(ctx->tc);
+  const int64_t tiles = static_cast<int64_t>(p.tilesM) * p.tilesN;
+  if (tiles <= 0) return cudaSuccess;
+  const int grid = static_cast<int>(tiles < st->sms ? tiles : st->sms);
+  forward_split_kernel<EPI><<<grid, kThreads, kFsSmem, ctx->stream>>>(a, b, C, ldc, p);
+  count_launch();
+  return cudaGetLastError();
+}
+
 // The shared-memory opt-in is a per-device attribute of each kernel: set for every instantiation when a context is
 // created (with its device current), not once per process.
 cudaError_t prepare_forward_kernels() {
   cudaError_t e = cudaFuncSetAttribute(forward_kernel<F_SOFTMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(forward_kernel<F_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(forward_kernel<F_SUB>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(forward_kernel<F_ISTA>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(forward_split_kernel<F_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFsSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(forward_split_kernel<F_SUB>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFsSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(forward_split_kernel<F_ISTA>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFsSmem);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(forward_kernel<F_SOFTMAX, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
   return e;
@@ -813,10 +987,10 @@ inline unsigned grid1d(int64_t items, int per_block) {
 // column-equivalents (below 128 columns a k-block is bound by the latency of its operand loads, not by the MMA).
 // Narrower tiles fill the SMs of small products, where 256-wide ones leave many idle or need a nearly empty
 // second round; ties go to the wider tile.
-inline int pick_tile_width(int sms, int64_t tilesM, int64_t N) {
-  int best = BN;
+inline int pick_tile_width(int sms, int64_t tilesM, int64_t N, int widest) {
+  int best = widest;
   int64_t best_cost = INT64_MAX;
-  for (int bn = BN; bn >= 128; bn -= 32) {
+  for (int bn = widest; bn >= 128; bn -= 32) {
     const int64_t tiles = tilesM * ((N + bn - 1) / bn);
     const int64_t cost = ((tiles + sms - 1) / sms) * (bn + 16);
     if (cost < best_cost) { best_cost = cost; best = bn; }
@@ -824,17 +998,18 @@ inline int pick_tile_width(int sms, int64_t tilesM, int64_t N) {
   return best;
 }
 
+constexpr int kSplitPrefetch = SFB_SPLIT_PREFETCH;    // k-blocks of look-ahead of the L2 prefetch in the split products
+
 // One split-bf16 product  D[off..off+n) = A * B^T  with A = [*, 2*Cp] and B = [N x 2*Cp] (hi | lo) operands:
 // hi*hi + hi*lo + lo*hi over a contraction of Cp.
 template <int EPI>
 int split_product(sfb_ctx* ctx, int64_t off, int64_t n, __nv_bfloat16* A, __nv_bfloat16* B, int64_t N, int64_t Cp,
                   float* C, int64_t ldc, TcParams p) {
   const TcState* st = static_cast<const TcState*>(ctx->tc);
-  const int bn = pick_tile_width(st->sms, (n + BM - 1) / BM, N);
-  CUtensorMap ma, mb, mc;
+  const int bn = pick_tile_width(st->sms, (n + BM - 1) / BM, N, FS_BN);
+  CUtensorMap ma, mb;
   if (!make_map(st, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, A, 2 * Cp, off + n, 2 * Cp * 2, BK, BM) ||
-      !make_map(st, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, B, 2 * Cp, N, 2 * Cp * 2, BK, bn) ||
-      !make_map(st, &mc, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, C, N, off + n, ldc * 4, kChunk, 32))
+      !make_map(st, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, B, 2 * Cp, N, 2 * Cp * 2, BK, bn))
     return SFB_ERR_CUDA;
   p.M = static_cast<int32_t>(off + n); p.N = static_cast<int32_t>(N); p.Kc = static_cast<int32_t>(Cp);
   p.m_off = static_cast<int32_t>(off);
@@ -842,10 +1017,11 @@ int split_product(sfb_ctx* ctx, int64_t off, int64_t n, __nv_bfloat16* A, __nv_b
   p.bn = bn;
   p.tilesN = static_cast<int32_t>((N + bn - 1) / bn);
   p.nseg = 3; p.kseg = static_cast<int32_t>(Cp / BK);
+  p.prefetch = kSplitPrefetch;
   p.a_off0 = 0; p.a_off1 = 0; p.a_off2 = static_cast<int32_t>(Cp);
   p.b_off0 = 0; p.b_off1 = static_cast<int32_t>(Cp); p.b_off2 = 0;
   p.status = ctx->at<uint32_t>(ctx->lay.status);
-  CKC(launch_forward<EPI>(ctx, ma, mb, mc, p));
+  CKC(launch_forward_split<EPI>(ctx, ma, mb, C, ldc, p));
   ctx->stats.flops += 3.0 * 2.0 * n * N * Cp;
   return SFB_OK;
 }
