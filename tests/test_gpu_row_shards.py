@@ -198,3 +198,19 @@ def test_replica_form_two_ranks_on_one_gpu(name):
     assert replica_step(ctx, list(range(wl.workers)), X, Y, lab, U_all, V_all) == 0
     assert torch.equal(W, Ws[0])
     ctx.close()
+
+
+def test_a_shard_that_owns_no_class_of_the_batch():
+    """Every class id of the batch lies in the first shard: the other shards contribute softmax mass only, their
+    owner flags are all 0, and their rows still receive the (small) update of the non-label classes."""
+    wl = _workload()
+    W0 = I.initial_W(wl)
+    inp = I.step_inputs(wl, 0)
+    inp.labels = (inp.labels % 50).astype(np.int32)            # 3 shards of 111 rows: all labels in shard 0
+    ref = oracle_step(wl, W0, inp)
+    for prec in (S.PREC_FP32, S.PREC_BF16):
+        W, parts, losses, status = _sharded_step(wl, W0, inp, prec, 3)
+        assert status == [0, 0, 0]
+        assert rel_err(W, ref, W0) <= TOL[prec]
+        assert parts[0, :, 3].sum() == wl.K and parts[1:, :, 3].sum() == 0
+        assert np.abs(W[111:] - W0[111:]).max() > 0            # the other shards' rows moved too

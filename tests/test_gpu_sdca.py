@@ -113,3 +113,23 @@ def test_sdca_argument_and_state_errors():
         plain.sfb_sdca_step(X, lab, ids)
     assert e.value.code == -10
     plain.close()
+
+
+def test_a_sample_without_features_moves_its_dual_row_to_the_softmax_and_leaves_W_alone():
+    """a_i = 0: kappa = 0, the coordinate problem has no quadratic term and its minimiser is softmax(z) = softmax(0),
+    the uniform distribution; the factor pair (du_i, 0) changes nothing in W."""
+    N, J, Dm = 8, 20, 12
+    cfg = S.make_config(S.L2MLR, J, Dm, 1, 2, 1.0, S.PREC_FP32, sdca_lambda=0.1, sdca_n=N)
+    W = torch.zeros((J, Dm), dtype=torch.float32, device="cuda")
+    y = np.array([3, 7], dtype=np.int32)
+    Q = to_dev(D.initial_dual(np.arange(N) % J, J).astype(np.float32), torch)
+    ctx = S.Context(cfg, W)
+    ctx.sfb_sdca_set_dual(Q)
+    X = torch.zeros((2, Dm), dtype=torch.float32, device="cuda")
+    ctx.sfb_sdca_step(X, to_dev(y, torch), to_dev(np.array([3, 7], dtype=np.int32), torch))
+    assert ctx.sfb_get_status() == 0
+    Qh = Q.cpu().numpy()
+    np.testing.assert_allclose(Qh[3], np.full(J, 1.0 / J), atol=1e-6)
+    np.testing.assert_allclose(Qh[7], np.full(J, 1.0 / J), atol=1e-6)
+    assert float(W.abs().max()) == 0.0
+    ctx.close()

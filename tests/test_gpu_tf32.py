@@ -103,3 +103,16 @@ def test_tensor_core_fp32_mode_is_for_the_logistic_models():
     with pytest.raises(S.SfbError) as e:
         S.sfb_workspace_bytes(S.make_config(S.DML, 64, 64, 1, 8, 0.1, S.PREC_TF32X3))
     assert e.value.code == -10
+
+
+@pytest.mark.parametrize("shape", [(5, 8, 1, 3), (40, 36, 2, 17), (257, 68, 1, 1)])
+def test_degenerate_shapes_on_the_tensor_cores(shape):
+    """Matrices smaller than one tile, a contraction shorter than one k-block, one sample: everything is padding."""
+    rows, cols, P, B = shape
+    wl = I.scaled(I.WORKLOADS["mlr_mid"], "mlr_tf32_tiny", rows=rows, cols=cols, workers=P, batch=B, eta=0.1, w_std=0.3,
+                  x_scale="unit")
+    W0, inp = I.initial_W(wl), I.step_inputs(wl, 0)
+    ref = oracle_step(wl, W0, inp)
+    W, _, _, st, _ = _step(wl, W0, inp, S.PREC_TF32X3)
+    assert st == 0
+    assert rel_err(W, ref, W0) <= TOL32
