@@ -284,8 +284,9 @@ extern "C" int sfb_forward_partials(sfb_ctx* ctx, const float* X_dev, const int3
   ctx->committed = 0;
   ctx->gathered = false;
   CK(cudaEventRecord(ctx->ev[0], ctx->stream));
-  if (c.precision == SFB_PREC_BF16) {
-    rc = tc_forward_partials(ctx, X_dev, labels_dev, partials_dev);
+  if (c.precision == SFB_PREC_BF16 || ctx->tf32) {
+    rc = ctx->tf32 ? tc32_forward_partials(ctx, X_dev, labels_dev, partials_dev)
+                   : tc_forward_partials(ctx, X_dev, labels_dev, partials_dev);
     if (rc) return rc;
   } else {
     const int64_t K = ctx->K;
@@ -313,8 +314,9 @@ extern "C" int sfb_finish_factors(sfb_ctx* ctx, const float* partials_all_dev, i
   if (!al16(partials_all_dev)) return SFB_ERR_ALIGN;
   if (!ctx->partials_ready) return SFB_ERR_STATE;
   const sfb_config& c = ctx->cfg;
-  if (c.precision == SFB_PREC_BF16) {
-    const int rc = tc_finish_factors(ctx, partials_all_dev, shards);
+  if (c.precision == SFB_PREC_BF16 || ctx->tf32) {
+    const int rc = ctx->tf32 ? tc32_finish_factors(ctx, partials_all_dev, shards)
+                             : tc_finish_factors(ctx, partials_all_dev, shards);
     if (rc) return rc;
   } else {
     CK(mlr_shard_finish(ctx->stream, ctx->at<float>(ctx->lay.U), ctx->K, c.rows, c.rows, ctx->at<int32_t>(ctx->lay.stageL),

@@ -1085,11 +1085,9 @@ int factors_split(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const fl
 
 }  // namespace
 
-// fp32 mode on the tensor cores: factors of n MLR samples at pair offset off.  The logits are the three-term tf32
-// product of the (big | small) samples and the (big | small) rows of W; softmax, loss and the factors in fp32.
-// sdca_ids != nullptr: the dual changes of the SDCA step instead of softmax - onehot.
-int tc32_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const int32_t* labels, const int32_t* sdca_ids,
-                 float inv_lam_n) {
+// v = x, the (big | small) samples, and the logits of n samples at pair offset off against this context's rows as
+// the three-term tf32 product, with the per-(sample, 256-row block) softmax partials.
+static int mlr32_forward(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, int* tiles_n) {
   const sfb_config& c = ctx->cfg;
   const TcState* st = static_cast<const TcState*>(ctx->tc);
   const Layout& L = ctx->lay;
@@ -1100,7 +1098,6 @@ int tc32_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const int
   float* As = ctx->at<float>(L.As);
   float* Z = ctx->at<float>(L.ZT);
   float* V = ctx->at<float>(L.V) + off * cols;
-  float* U = ctx->at<float>(L.U) + off * rows;
   // Ws, the (big | small) copy of W, is built at set-up and rewritten by the update's epilogue together with W
   CKC(pack_copy(s, V, X, nullptr, n * cols));                                              // v = x
   split32_rows_kernel<<<grid1d(n * cols / 4, 256), 256, 0, s>>>(X, n, cols, cols, As + off * 2 * L.colsp, L.colsp);
@@ -1123,6 +1120,60 @@ int tc32_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const int
   p.b_off0 = static_cast<int32_t>(L.colsp); p.b_off1 = 0; p.b_off2 = 0;
   CKC((launch_forward<F_SOFTMAX, true>(ctx, ma, mb, mc, p)));                                // z_i = W x_i
   ctx->stats.flops += 3.0 * 2.0 * n * rows * cols;
+  *tiles_n = p.tilesN;
+  return SFB_OK;
+}
+
+// Row-sharded form in the tensor-core fp32 mode: partials of all K samples against this shard's rows ...
+int tc32_forward_partials(sfb_ctx* ctx, const float* X, const int32_t* labels, float* part_out) {
+  const sfb_config& c = ctx->cfg;
+  const Layout& L = ctx->lay;
+  int tiles_n = 0;
+  const int rc = mlr32_forward(ctx, 0, ctx->K, X, &tiles_n);
+  if (rc) return rc;
+  CKC(cudaMemcpyAsync(ctx->at<int32_t>(L.labels), labels, static_cast<size_t>(ctx->K) * 4, cudaMemcpyDeviceToDevice, ctx->stream));
+  mlr_shard_partials_tc_kernel<<<static_cast<unsigned>((ctx->K + 7) / 8), 256, 0, ctx->stream>>>(
+      ctx->at<float2>(L.part), ctx->K, tiles_n, ctx->at<float>(L.ZT), round_up(c.rows, 32), c.rows,
+      ctx->at<int32_t>(L.labels), ctx->row_offset, ctx->K, reinterpret_cast<float4*>(part_out));
+  count_launch();
+  CKC(cudaGetLastError());
+  return SFB_OK;
+}
+
+// ... and the fp32 factors from the partials of all shards.
+int tc32_finish_factors(sfb_ctx* ctx, const float* parts, int shards) {
+  const sfb_config& c = ctx->cfg;
+  const Layout& L = ctx->lay;
+  const int64_t K = ctx->K, rows = c.rows;
+  mlr_shard_finish_tc_kernel<<<static_cast<unsigned>((K + 255) / 256), 256, 0, ctx->stream>>>(
+      reinterpret_cast<const float4*>(parts), shards, K, rows, ctx->row_offset, ctx->at<int32_t>(L.labels),
+      ctx->at<float>(L.lse), ctx->at<float>(L.loss), ctx->at<float>(L.coef), ctx->at<uint32_t>(L.status));
+  count_launch();
+  dim3 ugrid(static_cast<unsigned>(std::min<int64_t>((rows + 255) / 256, 64)), static_cast<unsigned>(K));
+  mlr_finish_u_kernel<false><<<ugrid, 256, 0, ctx->stream>>>(ctx->at<float>(L.ZT), round_up(rows, 32), rows, ctx->at<float>(L.lse),
+                                                             ctx->at<int32_t>(L.labels), ctx->at<float>(L.U));
+  count_launch();
+  CKC(cudaGetLastError());
+  return SFB_OK;
+}
+
+// fp32 mode on the tensor cores: factors of n MLR samples at pair offset off.  The logits are the three-term tf32
+// product of the (big | small) samples and the (big | small) rows of W; softmax, loss and the factors in fp32.
+// sdca_ids != nullptr: the dual changes of the SDCA step instead of softmax - onehot.
+int tc32_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const int32_t* labels, const int32_t* sdca_ids,
+                 float inv_lam_n) {
+  const sfb_config& c = ctx->cfg;
+  const Layout& L = ctx->lay;
+  const int64_t rows = c.rows, cols = c.cols, K = ctx->K;
+  const int64_t ldz = round_up(rows, 32);
+  cudaStream_t s = ctx->stream;
+  float* Z = ctx->at<float>(L.ZT);
+  float* U = ctx->at<float>(L.U) + off * rows;
+  int tiles_n = 0;
+  {
+    const int rc = mlr32_forward(ctx, off, n, X, &tiles_n);
+    if (rc) return rc;
+  }
   dim3 ugrid(static_cast<unsigned>(std::min<int64_t>((rows + 255) / 256, 64)), static_cast<unsigned>(n));
   if (sdca_ids) {
     CKC(sdca_dual_rows(s, Z + off * ldz, n, rows, ldz, X, cols, labels, sdca_ids, ctx->dualQ, ctx->dual_n, inv_lam_n, c.eta,
@@ -1130,7 +1181,7 @@ int tc32_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const int
     mlr_finish_u_kernel<true><<<ugrid, 256, 0, s>>>(Z + off * ldz, ldz, rows, nullptr, nullptr, U);
   } else {
     float* lse = ctx->at<float>(L.lse);
-    mlr_lse_kernel<<<static_cast<unsigned>((n + 7) / 8), 256, 0, s>>>(ctx->at<float2>(L.part), K, p.tilesN, Z, ldz, rows, labels,
+    mlr_lse_kernel<<<static_cast<unsigned>((n + 7) / 8), 256, 0, s>>>(ctx->at<float2>(L.part), K, tiles_n, Z, ldz, rows, labels,
                                                                      off, n, lse, ctx->at<float>(L.loss),
                                                                      ctx->at<float>(L.coef), ctx->at<uint32_t>(L.status));
     count_launch();

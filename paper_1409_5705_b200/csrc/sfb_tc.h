@@ -13,6 +13,8 @@ void tc_extend_layout(const sfb_config& c, Layout& L, size_t& off);
 void tc32_extend_layout(const sfb_config& c, Layout& L, size_t& off);
 int tc32_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const int32_t* labels, const int32_t* sdca_ids,
                  float inv_lam_n);
+int tc32_forward_partials(sfb_ctx* ctx, const float* X, const int32_t* labels, float* part_out);
+int tc32_finish_factors(sfb_ctx* ctx, const float* parts, int shards);
 int tc32_gather(sfb_ctx* ctx);
 int tc32_update(sfb_ctx* ctx);
 int tc_init(sfb_ctx* ctx);

@@ -8,7 +8,7 @@ import paper_1409_5705_b200 as S
 import sfb_inputs as I
 from oracle import sfb_oracle as O
 
-TOL = {S.PREC_FP32: 1e-5, S.PREC_BF16: 2e-3}
+TOL = {S.PREC_FP32: 1e-5, S.PREC_BF16: 2e-3, S.PREC_TF32X3: 1e-5, S.PREC_FP32_FFMA: 1e-5}
 
 
 def config_for(wl: I.Workload, precision, L=0.0, prox=None):
