@@ -549,7 +549,8 @@ def main():
     sampler, sfile = clocks_sampler(local) if rank == 0 else (None, None)
     for i in range(args.warmup):
         phased_step(i)
-    launches0 = ctx.sfb_get_stats().kernel_launches
+    st0 = ctx.sfb_get_stats()
+    launches0 = st0.kernel_launches
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
     barrier()
     wall0 = time.time()
@@ -562,7 +563,12 @@ def main():
     barrier()
     clocks = clocks_summary(sampler, sfile, wall0, time.time()) if rank == 0 else None
     total_ms = t_start.elapsed_time(t_end)
-    launches = ctx.sfb_get_stats().kernel_launches - launches0
+    st1 = ctx.sfb_get_stats()
+    launches = st1.kernel_launches - launches0
+    copy_stats = {"row_pieces_per_step": (st1.copy_pieces - st0.copy_pieces) / args.steps,
+                  "rewritten_per_step": (st1.copy_written - st0.copy_written) / args.steps,
+                  "fraction_rewritten": (st1.copy_written - st0.copy_written) / max(1, st1.copy_pieces - st0.copy_pieces)} \
+        if st1.copy_pieces > st0.copy_pieces else None
     status = ctx.sfb_get_status()
     ms_f = sum(e[0].elapsed_time(e[1]) for e in evs) / args.steps
     ms_g = sum(e[1].elapsed_time(e[2]) for e in evs) / args.steps
@@ -648,7 +654,7 @@ def main():
                       "sf_broadcast_p2p": wl.workers * (wl.workers - 1) * wl.batch * (wl.rows + wl.cols) * esz,
                       "dense_sync": wl.workers * wl.rows * wl.cols * 4,
                       "dense_over_sf": wl.workers * wl.rows * wl.cols * 4 / one_copy},
-            "status_word": status}
+            "operand_copy": copy_stats, "status_word": status}
     if update_loop is not None:
         line["update_loop"] = update_loop
     print(json.dumps(line), flush=True)

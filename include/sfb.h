@@ -105,6 +105,10 @@ typedef struct sfb_stats {
   float   last_loss;          /* MLR: mean over the last step's K samples of -log p(y_i); else 0        */
   float   sc_lipschitz;       /* SC: the L = ||W||_2^2 the coder used in the last step                  */
   int64_t kernel_launches;    /* kernels this library has launched in this process                      */
+  int64_t copy_pieces;        /* MLR, bf16 mode: 64-byte row pieces of the bf16 operand copy of W that the update
+                                 passes went over since sfb_init, and                                          */
+  int64_t copy_written;       /* how many of them they rewrote (a piece whose 32 bf16 roundings did not change
+                                 already holds bf16 of the new values and is left alone)                      */
 } sfb_stats;
 
 /* Bytes of device workspace a context with this config needs.  Host-only; no CUDA call. */
@@ -243,6 +247,12 @@ int sfb_dense_sync_step(sfb_ctx* ctx, const float* X_dev, const float* Y_dev, co
  * (bf16 cannot hold it when p_iy is close to 1). */
 int sfb_get_factors(sfb_ctx* ctx, const void** U_dev, const void** V_dev, int32_t* dtype, int32_t* layout,
                     int64_t* ldu, int64_t* ldv);
+
+/* The library's operand copy of W, for inspection: MLR in bf16 mode: dtype 1, the bf16 matrix [rows x ld]; the
+ * tensor-core fp32 mode: dtype 2, fp32 words [rows x ld] holding tf32(w) at column c and tf32(w - tf32(w)) at column
+ * ld/2 + c.  SFB_ERR_UNSUPPORTED where no persistent copy exists (the other models rebuild theirs every step; the FFMA
+ * kernels read W itself). */
+int sfb_get_operand_copy(sfb_ctx* ctx, const void** copy_dev, int32_t* dtype, int64_t* ld);
 
 /* Waits for the stream, then fills the counters. */
 int sfb_get_stats(sfb_ctx* ctx, sfb_stats* out);

@@ -21,7 +21,7 @@ EXPORTS = ("sfb_workspace_bytes", "sfb_init", "sfb_compute_factors", "sfb_gather
            "sfb_get_status", "sfb_strerror", "sfb_last_cuda_error", "sfb_destroy", "sfb_prox_columns_noalloc",
            "sfb_selftest_wait_timeout", "sfb_set_row_shard", "sfb_forward_partials", "sfb_finish_factors",
            "sfb_replay_update", "sfb_refresh_operands", "sfb_sdca_set_dual", "sfb_sdca_compute_factors",
-           "sfb_sdca_step", "sfb_set_factors", "sfb_set_eta")
+           "sfb_sdca_step", "sfb_set_factors", "sfb_set_eta", "sfb_get_operand_copy")
 NOALLOC_MAX_COLS = 16384
 
 
@@ -39,7 +39,8 @@ class sfb_stats(ctypes.Structure):
                 ("gather_bytes", ctypes.c_double), ("gather_bytes_p2p", ctypes.c_double),
                 ("dense_sync_bytes", ctypes.c_double), ("ms_factors", ctypes.c_float),
                 ("ms_gather", ctypes.c_float), ("ms_update", ctypes.c_float), ("last_loss", ctypes.c_float),
-                ("sc_lipschitz", ctypes.c_float), ("kernel_launches", ctypes.c_int64)]
+                ("sc_lipschitz", ctypes.c_float), ("kernel_launches", ctypes.c_int64),
+                ("copy_pieces", ctypes.c_int64), ("copy_written", ctypes.c_int64)]
 
 
 class SfbError(RuntimeError):
@@ -90,6 +91,7 @@ def lib() -> ctypes.CDLL:
         L.sfb_sdca_step.argtypes = [vp, vp, vp, vp]
         L.sfb_set_factors.argtypes = [vp, i32, vp, vp]
         L.sfb_set_eta.argtypes = [vp, ctypes.c_float]
+        L.sfb_get_operand_copy.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(i32), ctypes.POINTER(i64)]
         for name in EXPORTS:
             if name != "sfb_strerror":
                 getattr(L, name).restype = ctypes.c_int
@@ -183,8 +185,7 @@ class Context:
         self._ck(lib().sfb_refresh_operands(self._h), "sfb_refresh_operands")
 
     def sfb_replay_update(self):
-        self._ck(lib().sfb_replay_update(self._h), "sfb_replay_update", "sfb_refresh_operands", "sfb_sdca_set_dual", "sfb_sdca_compute_factors",
-           "sfb_sdca_step", "sfb_set_factors", "sfb_set_eta")
+        self._ck(lib().sfb_replay_update(self._h), "sfb_replay_update")
 
     def sfb_step(self, X, Y=None, labels=None):
         self._ck(lib().sfb_step(self._h, _ptr(X), _ptr(Y), _ptr(labels)), "sfb_step")
@@ -225,6 +226,17 @@ class Context:
         if lo == 0:
             return view(U, K, ldu)[:, :rows].float(), view(V, K, ldv)[:, :cols].float()
         return view(U, rows, ldu)[:, :K].t().float(), view(V, cols, ldv)[:, :K].t().float()
+
+    def operand_copy_as_tensor(self):
+        """The library's operand copy of W as a torch view into the workspace: bf16 [rows, ld] (MLR, bf16 mode) or
+        fp32 [rows, ld] with the (big | small) tf32 halves side by side (tensor-core fp32 mode)."""
+        import torch
+        ptr, dt, ld = ctypes.c_void_p(), ctypes.c_int32(), ctypes.c_int64()
+        self._ck(lib().sfb_get_operand_copy(self._h, ctypes.byref(ptr), ctypes.byref(dt), ctypes.byref(ld)),
+                 "sfb_get_operand_copy")
+        tdt, esz = (torch.bfloat16, 2) if dt.value == 1 else (torch.float32, 4)
+        off = ptr.value - self.workspace.data_ptr()
+        return self.workspace[off:off + self.cfg.rows * ld.value * esz].view(tdt).view(self.cfg.rows, ld.value)
 
     def sfb_get_stats(self) -> sfb_stats:
         st = sfb_stats()

@@ -583,6 +583,22 @@ extern "C" int sfb_get_factors(sfb_ctx* ctx, const void** U_dev, const void** V_
   return tc_get_factors(ctx, U_dev, V_dev, dtype, layout, ldu, ldv);
 }
 
+extern "C" int sfb_get_operand_copy(sfb_ctx* ctx, const void** copy_dev, int32_t* dtype, int64_t* ld) {
+  if (!ctx || !copy_dev) return SFB_ERR_ARG;
+  if (ctx->cfg.model != SFB_MLR) return SFB_ERR_UNSUPPORTED;
+  if (ctx->tf32) {
+    *copy_dev = ctx->at<float>(ctx->lay.Ws);
+    if (dtype) *dtype = 2;
+    if (ld) *ld = 2 * ctx->lay.colsp;
+    return SFB_OK;
+  }
+  if (ctx->cfg.precision != SFB_PREC_BF16) return SFB_ERR_UNSUPPORTED;
+  *copy_dev = ctx->at<char>(ctx->lay.Wb);
+  if (dtype) *dtype = 1;
+  if (ld) *ld = ctx->lay.colsb;
+  return SFB_OK;
+}
+
 extern "C" int sfb_get_stats(sfb_ctx* ctx, sfb_stats* out) {
   if (!ctx || !out) return SFB_ERR_ARG;
   CK(cudaStreamSynchronize(ctx->stream));
@@ -596,6 +612,8 @@ extern "C" int sfb_get_stats(sfb_ctx* ctx, sfb_stats* out) {
     CK(cudaMemcpy(&h, ctx->at<Scalars>(ctx->lay.scalars), sizeof(h), cudaMemcpyDeviceToHost));
     ctx->stats.last_loss = h.loss_mean;
     ctx->stats.sc_lipschitz = h.L;
+    ctx->stats.copy_pieces = static_cast<int64_t>(h.copy_pieces);
+    ctx->stats.copy_written = static_cast<int64_t>(h.copy_written);
   }
   ctx->stats.kernel_launches = g_kernel_launches.load(std::memory_order_relaxed);
   *out = ctx->stats;

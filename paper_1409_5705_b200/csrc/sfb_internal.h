@@ -53,6 +53,8 @@ struct Scalars {                      // device-resident scalars
   float L;                            // ||W||_2^2 used by the coder
   float invL;
   float tmp;
+  unsigned long long copy_pieces;     // 64-byte row pieces of the bf16 operand copy the update passes went over ...
+  unsigned long long copy_written;    // ... and how many of them they had to rewrite (the others already held bf16(W))
 };
 
 }  // namespace sfb

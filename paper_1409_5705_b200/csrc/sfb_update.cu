@@ -61,6 +61,7 @@ struct UpdParams {
   int64_t shadow_ld;
   int64_t shadow_half;
   uint32_t* status;
+  unsigned long long* copy_counters;   // [0] row pieces of the bf16 copy visited, [1] of them rewritten (or null)
 };
 
 __device__ __forceinline__ float to_tf32(float x) {
@@ -196,6 +197,7 @@ update_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     const uint32_t tempty_leader0 = mapa_u32(smem_u32(&tempty[0]), 0), tempty_leader1 = mapa_u32(smem_u32(&tempty[1]), 0);
     const int row_in_tile = static_cast<int>(rank) * UM + q * 32;
     bool ok = true;
+    uint32_t copy_written = 0;           // row pieces of the bf16 copy this warp rewrote
     uint32_t lg = 0;                     // next chunk to request
     auto issue_load = [&]() {
       if (lg >= nchunks) return;
@@ -233,10 +235,13 @@ update_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         uint8_t* sl = ring + slot * kSlotBytes;
         if (!__all_sync(0xffffffffu, mbar_wait(&rf[slot], (g / kRing) & 1, abort_flag))) return false;
         const int x0 = n0 + h * (UN / 2) + c * kChunk;
+        uint32_t differs = 0;      // SHADOW == 1: does the bf16 rounding of any of this row's 32 values change?
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           float4* wp = reinterpret_cast<float4*>(sl + lane * 128 + ((j ^ (lane & 7)) << 4));
           float4 w = *wp;
+          uint32_t o01 = 0, o23 = 0;
+          if (SHADOW == 1) { o01 = pack2(w.x, w.y); o23 = pack2(w.z, w.w); }
           w.x = fmaf(p.alpha, __uint_as_float(acc[4 * j + 0]), w.x);
           w.y = fmaf(p.alpha, __uint_as_float(acc[4 * j + 1]), w.y);
           w.z = fmaf(p.alpha, __uint_as_float(acc[4 * j + 2]), w.z);
@@ -246,7 +251,12 @@ update_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             w.z = prox_entry(w.z, p.prox_kind, p.prox_a); w.w = prox_entry(w.w, p.prox_kind, p.prox_a);
           }
           *wp = w;
+          if (SHADOW == 1) differs |= (o01 ^ pack2(w.x, w.y)) | (o23 ^ pack2(w.z, w.w));
         }
+        // The bf16 copy holds bf16(W) when the pass starts (set-up, refresh, label rows and this kernel keep it so): a
+        // row piece whose 32 roundings all stay the same already holds bf16 of the new values and is not rewritten.
+        // With updates of a few fp32 spacings per entry that is most of the matrix; the copy stays exact either way.
+        const uint32_t rowmask = SHADOW == 1 ? __ballot_sync(0xffffffffu, differs != 0) : 0u;
         fence_proxy_async_smem();
         __syncwarp();                                        // every lane has rewritten its row of the slot
         if (lane == 0) {
@@ -276,14 +286,19 @@ update_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
           // bf16 copy of the chunk, read back from the slot with 8 lanes per row (4 rows per pass): each row's
           // 32 values leave as one 64-byte piece instead of 32 lanes storing 16 bytes to 32 different rows.
           const int sub = lane >> 3, jj = lane & 7;
-#pragma unroll
-          for (int r0 = 0; r0 < 32; r0 += 4) {
-            const int r = r0 + sub;
-            const float4 w = *reinterpret_cast<const float4*>(sl + r * 128 + ((jj ^ (r & 7)) << 4));
-            const int col = x0 + 4 * jj;
-            if (y0 + r < p.rows && col < p.shadow_ld)
-              *reinterpret_cast<uint2*>(p.shadow + static_cast<int64_t>(y0 + r) * p.shadow_ld + col) =
-                  make_uint2(pack2(w.x, w.y), pack2(w.z, w.w));
+          copy_written += __popc(rowmask);
+          // the changed rows, four per pass: lane group `sub` takes the (sub+1)-th changed row still to do
+#pragma unroll 1
+          for (uint32_t todo = rowmask; todo != 0;) {
+            const uint32_t r = __fns(todo, 0, sub + 1);           // 0xffffffff when fewer than sub+1 rows are left
+            if (r < 32u) {
+              const float4 w = *reinterpret_cast<const float4*>(sl + r * 128 + ((jj ^ (r & 7)) << 4));
+              const int col = x0 + 4 * jj;
+              if (y0 + static_cast<int>(r) < p.rows && col < p.shadow_ld)
+                *reinterpret_cast<uint2*>(p.shadow + static_cast<int64_t>(y0 + r) * p.shadow_ld + col) =
+                    make_uint2(pack2(w.x, w.y), pack2(w.z, w.w));
+            }
+            todo &= todo - 1; todo &= todo - 1; todo &= todo - 1; todo &= todo - 1;    // drop the four lowest set bits
           }
         }
         ++g;
@@ -296,6 +311,10 @@ update_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
       }
     }
     if (lane == 0) tma_wait_group<0>();
+    if (SHADOW == 1 && lane == 0 && p.copy_counters) {
+      atomicAdd(&p.copy_counters[0], 32ull * nchunks);
+      atomicAdd(&p.copy_counters[1], static_cast<unsigned long long>(copy_written));
+    }
   }
 
   // ---------------- teardown ----------------
@@ -496,16 +515,18 @@ int tc_update(sfb_ctx* ctx) {
   }
   p.nseg = 1;
   p.shadow = ctx->at<__nv_bfloat16>(L.Wb); p.shadow_ld = L.colsb;
+  p.copy_counters = &ctx->at<Scalars>(L.scalars)->copy_pieces;
   if ((c.cols + 1023) / 1024 > 65535) return SFB_ERR_SHAPE;
   dim3 lgrid(static_cast<unsigned>(ctx->K), static_cast<unsigned>((c.cols + 1023) / 1024));
   // With a fused prox the fp32 label-row term has to be in W before the pass that applies the operator, so it goes
-  // first (both terms are sums into W; the pass then also writes the bf16 copy of those rows).
+  // first (both terms are sums into W).  Either way the label-row kernel rewrites the bf16 copy of its rows, so the
+  // copy equals bf16(W) whenever the main pass starts.
   const bool labels_first = ctx->prox_kind != 0;
   for (int pass = 0; pass < 2; ++pass) {
     if ((pass == 0) == labels_first) {
       label_rows_kernel<<<lgrid, 256, 0, ctx->stream>>>(
           ctx->W, c.rows, c.cols, ctx->at<float>(L.Xf), ctx->at<int32_t>(L.labels), ctx->at<float>(L.coef),
-          static_cast<int>(ctx->K), ctx->step, labels_first ? nullptr : ctx->at<__nv_bfloat16>(L.Wb), L.colsb);
+          static_cast<int>(ctx->K), ctx->step, ctx->at<__nv_bfloat16>(L.Wb), L.colsb);   // keeps the copy = bf16(W)
     } else {
       update_pair_kernel<1><<<grid, kThreads, kSmem, ctx->stream>>>(ma, mb, mc, p);     // W += -eta * P^T V
     }
