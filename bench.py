@@ -222,19 +222,21 @@ def run_reference(args, wl, rank):
     print(json.dumps(line), flush=True)
 
 
-# DRAM bytes per launch of the update kernel from the ncu capture summarised in
-# profiles/ncu_update_pair_kernel_mlr_rows16384.md (a slab of 16384 rows of the paper-scale MLR shape; traffic is
-# proportional to the rows, see that file).  "kernel_unchanged_since" names the commit of csrc/sfb_update.cu the
-# counters were taken at: when the kernel is edited this entry has to be re-captured or set to None.
-NCU_UPDATE_TRAFFIC = {"rows": 16384, "cols": 10000, "K": 1024, "bytes": 758433280 + 932738048,
-                      "kernel_unchanged_since": "1339426"}
+# DRAM bytes per launch of the update kernel at the paper-scale MLR shape, from the one-pass ncu capture summarised in
+# profiles/ncu_update_pair_kernel_mlr_large_dram.md (dram__bytes_read.sum + dram__bytes_write.sum of one launch of the
+# full-size bench).  The bf16 copy of W is rewritten only where its rounding changed, so the traffic depends on the data
+# and does not scale with the rows: the figure applies to this workload only.  "kernel_unchanged_since" names the
+# commit of csrc/sfb_update.cu the counters were taken at: when the kernel is edited this entry has to be re-captured
+# or set to None.
+NCU_UPDATE_TRAFFIC = {"rows": 325000, "cols": 10000, "K": 1024, "bytes": 15.90e9 + 13.85e9,
+                      "kernel_unchanged_since": "318561f"}
 
 
 def ncu_traffic_per_launch(wl, prec):
     t = NCU_UPDATE_TRAFFIC
-    if t["bytes"] is None or wl.model != I.MLR or wl.cols != t["cols"] or wl.K != t["K"] or prec != 0:
+    if t["bytes"] is None or wl.model != I.MLR or wl.cols != t["cols"] or wl.K != t["K"] or wl.rows != t["rows"]             or prec != 0:
         return None
-    return t["bytes"] * wl.rows / t["rows"]
+    return t["bytes"]
 
 
 def workload_config(wl, dtype):
@@ -267,7 +269,7 @@ NOMINAL_TF32_OVER_BF16 = 1100.0 / 2250.0   # nominal ratio of the dense tf32 and
 NOMINAL_HBM_GBS = 7700.0
 
 
-def update_roofline(wl, prec_bf16, ms_u, peaks, clocks, sustained=True, tf32=False):
+def update_roofline(wl, prec_bf16, ms_u, peaks, clocks, sustained=True, tf32=False, copy_fraction=1.0):
     """Roofline entry of the fused update W += -eta U^T V (one launch per step).  Algorithmic bytes per launch: W read
     and written once in fp32 plus U and V read once (what the method has to move).  The bf16 copy of W that this design
     writes alongside (the operand of the next forward product) is real traffic of the kernel and is reported beside
@@ -278,7 +280,7 @@ def update_roofline(wl, prec_bf16, ms_u, peaks, clocks, sustained=True, tf32=Fal
         esz = 4                                                               # (hi, lo) pairs of bf16
     upd_flops = 2.0 * wl.rows * wl.cols * K
     upd_bytes = 8.0 * wl.rows * wl.cols + K * (wl.rows + wl.cols) * esz
-    shadow_bytes = 2.0 * wl.rows * wl.cols if (prec_bf16 and wl.model == I.MLR) else 0.0
+    shadow_bytes = 2.0 * wl.rows * wl.cols * copy_fraction if (prec_bf16 and wl.model == I.MLR) else 0.0
     tf_peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
     if prec_bf16:
         t_flop = upd_flops / (tf_peak * 1e12)
@@ -621,7 +623,9 @@ def main():
     h2d = K * wl.in_dim * 4 + (K * wl.cols * 4 if wl.model == I.DML else 0) + (K * 4 if wl.model != I.SC else 0)
 
     # ---- roofline of the dominant kernel (the fused update), timed inside the long step: sustained tensor figure
-    roof = update_roofline(wl, prec == S.PREC_BF16, ms_u, peaks, clocks, tf32=runs_tf32(wl, args.precision))
+    roof = update_roofline(wl, prec == S.PREC_BF16, ms_u, peaks, clocks, tf32=runs_tf32(wl, args.precision),
+                           copy_fraction=min(1.0, copy_stats["rewritten_per_step"] / (wl.rows * math.ceil(wl.cols / 32)))
+                           if copy_stats else 1.0)
     roof_fwd, roof_step = (None, None)
     if prec == S.PREC_BF16 and wl.model == I.MLR:
         roof_fwd, roof_step = forward_and_step_rooflines(wl, ms_f, total_ms / args.steps, roof["roof_ms"], peaks)
