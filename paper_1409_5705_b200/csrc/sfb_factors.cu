@@ -278,10 +278,16 @@ __global__ void __launch_bounds__(NTHREADS) sdca_dual_kernel(float* __restrict__
 
 // One block per pair: q = ||z||^2; similar: u = 2z; dissimilar: u = -2z if q < margin else 0 (Section 2, DML).
 template <int NTHREADS>
-__global__ void __launch_bounds__(NTHREADS) dml_scale_kernel(float* __restrict__ Z, int64_t rows, int64_t ld,
+__global__ void __launch_bounds__(NTHREADS) dml_scale_kernel(float* __restrict__ Z, const float* __restrict__ Z2,
+                                                             int64_t rows, int64_t ld,
                                                              const int32_t* __restrict__ similar, float margin) {
   __shared__ float sh[32];
   float* z = Z + static_cast<int64_t>(blockIdx.x) * ld;
+  if (Z2) {                      // z arrives as two partial sums over halves of the contraction (fixed order: Z + Z2)
+    const float* z2 = Z2 + static_cast<int64_t>(blockIdx.x) * ld;
+    for (int64_t j = threadIdx.x; j < rows; j += NTHREADS) z[j] += z2[j];
+    __syncthreads();
+  }
   float q = 0.f;
   for (int64_t j = threadIdx.x; j < rows; j += NTHREADS) q = fmaf(z[j], z[j], q);
   q = block_sum<NTHREADS>(q, sh);
@@ -523,9 +529,9 @@ cudaError_t sdca_dual_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows
 }
 
 cudaError_t dml_scale_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows, int64_t ld,
-                           const int32_t* similar, float margin) {
+                           const int32_t* similar, float margin, const float* Z2) {
   if (nsamp <= 0) return cudaSuccess;
-  dml_scale_kernel<256><<<static_cast<unsigned>(nsamp), 256, 0, s>>>(Z, rows, ld, similar, margin);
+  dml_scale_kernel<256><<<static_cast<unsigned>(nsamp), 256, 0, s>>>(Z, Z2, rows, ld, similar, margin);
   count_launch();
   return cudaGetLastError();
 }

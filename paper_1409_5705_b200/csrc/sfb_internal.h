@@ -29,6 +29,7 @@ struct Layout {
   size_t Wb, Xb, VT, ZT, UT, part, Xf, labels, coef, lse;
   // bf16 mode, DML and SC: (hi | lo) bf16 operands of the split products
   size_t Ws, WTs, As, Rs;             // W by rows, W transposed, the A operand (v or the codes), the residual
+  size_t U2;                          // DML: second partial of z when the forward product splits its contraction
   int64_t ldu;                        // row pitch of the fp32 U buffer (rows rounded up to 4 in bf16 mode)
   int64_t colsp, rowsp;               // cols, rows rounded up to 64
   int64_t Kp;                         // K rounded up to the contraction block of the update product
@@ -138,8 +139,9 @@ cudaError_t mlr_shard_finish(cudaStream_t s, float* Z, int64_t nsamp, int64_t ro
 cudaError_t sdca_dual_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows, int64_t ldz, const float* X, int64_t cols,
                            const int32_t* labels, const int32_t* ids, float* Q, int64_t n_samples, float inv_lam_n,
                            float gamma, float* coef, float* loss, uint32_t* status);
+// Z2 (may be null): a second partial of z (the other half of the contraction), added to Z first.
 cudaError_t dml_scale_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows, int64_t ld,
-                           const int32_t* similar, float margin);
+                           const int32_t* similar, float margin, const float* Z2 = nullptr);
 cudaError_t mean_of(cudaStream_t s, const float* v, int64_t n, float* out);
 cudaError_t prox_unit_columns(cudaStream_t s, float* W, int64_t rows, int64_t cols, float* colpart);
 cudaError_t estimate_lipschitz(cudaStream_t s, const float* W, int64_t rows, int64_t cols, float* b, float* y,

@@ -62,6 +62,8 @@ struct TcParams {
   const float* aux;            // F_SUB: the matrix subtracted, [M x ldaux]; F_ISTA: the matrix updated, [M x ldaux]
   int64_t ldaux;
   int32_t prefetch;            // k-blocks by which the producer asks L2 for the B operand ahead of its loads (0: off)
+  int32_t ksplit;              // forward_split_kernel, F_STORE: the contraction is cut into this many parts, each a work
+  int64_t c_split_stride;      //   unit of its own writing its partial product to C + part * c_split_stride (else 1, 0)
   const Scalars* sc;           // F_ISTA: 1 / L
   float lam;                   // F_ISTA: lambda
   __nv_bfloat16* split;        // F_SUB, F_ISTA: [M x ld_split] receives hi at column n and lo at column split_half + n
@@ -281,8 +283,9 @@ forward_split_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int ntiles = p.tilesM * p.tilesN;
-  const int numK = p.kseg;                          // k-blocks of the contraction (each serves three products)
+  const int S = p.ksplit > 1 ? p.ksplit : 1;
+  const int ntiles = p.tilesM * p.tilesN * S;       // work units: (tile, part of the contraction), parts of a tile adjacent
+  const int numKall = p.kseg;                       // k-blocks of the contraction (each serves three products)
   const int a_hi = p.a_off0, a_lo = p.a_off2, b_hi = p.b_off0, b_lo = p.b_off1;
 
   if (threadIdx.x == 0) {
@@ -307,8 +310,9 @@ forward_split_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       bool ok = true;
       for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
         int m0, n0;
-        tile_coords(p, tile, m0, n0);
-        for (int kl = 0; kl < numK; ++kl, ++it) {
+        tile_coords(p, tile / S, m0, n0);
+        const int part = tile % S, kbeg = part * numKall / S, numK = (part + 1) * numKall / S;
+        for (int kl = kbeg; kl < numK; ++kl, ++it) {
           const uint32_t s = it % FS_STAGES, ph = (it / FS_STAGES) & 1;
           if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
           if (p.prefetch > 0 && kl + p.prefetch < numK) {          // B streams from HBM when it is larger than L2
@@ -335,6 +339,7 @@ forward_split_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         if (!mbar_wait(&tempty[a], aph ^ 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + a * BN;
+        const int part = tile % S, numK = (part + 1) * numKall / S - part * numKall / S;
         for (int kb = 0; kb < numK; ++kb, ++it) {
           const uint32_t s = it % FS_STAGES, ph = (it / FS_STAGES) & 1;
           if (!mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
@@ -365,7 +370,9 @@ forward_split_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     if (EPI == F_ISTA) { invL = p.sc->invL; thr = p.lam * invL; }
     for (int tl = 0; tl < my_tiles && ok; ++tl) {
       int m0, n0;
-      tile_coords(p, blockIdx.x + tl * gridDim.x, m0, n0);
+      const int unit = blockIdx.x + tl * gridDim.x;
+      tile_coords(p, unit / S, m0, n0);
+      float* Cp = C + static_cast<int64_t>(unit % S) * p.c_split_stride;
       const uint32_t a = tl & 1, aph = (tl >> 1) & 1;
       if (!__all_sync(0xffffffffu, mbar_wait(&tfull[a], aph, abort_flag))) { ok = false; break; }
       tc_fence_after();
@@ -418,7 +425,7 @@ forward_split_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           }
         }
         // the fp32 result: this lane's 32 consecutive columns of its row
-        float* cp = C + static_cast<int64_t>(row) * ldc + col0;
+        float* cp = Cp + static_cast<int64_t>(row) * ldc + col0;
         if (whole && ((reinterpret_cast<uintptr_t>(cp) & 15u) == 0)) {
 #pragma unroll
           for (int j = 0; j < 8; ++j)
@@ -820,7 +827,7 @@ cudaError_t launch_forward(sfb_ctx* ctx, const CUtensorMap& a, const CUtensorMap
 template <int EPI>
 cudaError_t launch_forward_split(sfb_ctx* ctx, const CUtensorMap& a, const CUtensorMap& b, float* C, int64_t ldc, TcParams p) {
   const TcState* st = static_cast<const TcState*>(ctx->tc);
-  const int64_t tiles = static_cast<int64_t>(p.tilesM) * p.tilesN;
+  const int64_t tiles = static_cast<int64_t>(p.tilesM) * p.tilesN * (p.ksplit > 1 ? p.ksplit : 1);
   if (tiles <= 0) return cudaSuccess;
   const int grid = static_cast<int>(tiles < st->sms ? tiles : st->sms);
   forward_split_kernel<EPI><<<grid, kThreads, kFsSmem, ctx->stream>>>(a, b, C, ldc, p);
@@ -886,6 +893,7 @@ void tc_extend_layout(const sfb_config& c, Layout& L, size_t& off) {
     L.ldu = round_up(c.rows, 4);                                        // TMA stores need a 16-byte row pitch
     L.V = take(K * static_cast<size_t>(c.cols) * 4);
     L.U = take(K * static_cast<size_t>(L.ldu) * 4);
+    L.U2 = take(c.model == SFB_DML ? K * static_cast<size_t>(L.ldu) * 4 : 0);
     L.UT = take(static_cast<size_t>(c.rows) * 2 * L.Kp * 2);
     L.VT = take(static_cast<size_t>(c.cols) * 2 * L.Kp * 2);
     L.Ws = take(static_cast<size_t>(c.rows) * 2 * L.colsp * 2);         // W, rows x (hi | lo)
@@ -1004,7 +1012,7 @@ constexpr int kSplitPrefetch = SFB_SPLIT_PREFETCH;    // k-blocks of look-ahead 
 // hi*hi + hi*lo + lo*hi over a contraction of Cp.
 template <int EPI>
 int split_product(sfb_ctx* ctx, int64_t off, int64_t n, __nv_bfloat16* A, __nv_bfloat16* B, int64_t N, int64_t Cp,
-                  float* C, int64_t ldc, TcParams p) {
+                  float* C, int64_t ldc, TcParams p, int64_t c_split_stride = 0, int* parts_out = nullptr) {
   const TcState* st = static_cast<const TcState*>(ctx->tc);
   const int bn = pick_tile_width(st->sms, (n + BM - 1) / BM, N, FS_BN);
   CUtensorMap ma, mb;
@@ -1018,6 +1026,12 @@ int split_product(sfb_ctx* ctx, int64_t off, int64_t n, __nv_bfloat16* A, __nv_b
   p.tilesN = static_cast<int32_t>((N + bn - 1) / bn);
   p.nseg = 3; p.kseg = static_cast<int32_t>(Cp / BK);
   p.prefetch = kSplitPrefetch;
+  // a product whose tiles fill less than half of the SMs is cut along its contraction (plain store epilogue only: the
+  // partial products are added, in a fixed order, by the kernel that consumes them)
+  const int64_t tiles = static_cast<int64_t>(p.tilesM) * p.tilesN;
+  p.ksplit = (EPI == F_STORE && c_split_stride > 0 && 2 * tiles <= st->sms && p.kseg >= 8) ? 2 : 1;
+  p.c_split_stride = p.ksplit > 1 ? c_split_stride : 0;
+  if (parts_out) *parts_out = p.ksplit;
   p.a_off0 = 0; p.a_off1 = 0; p.a_off2 = static_cast<int32_t>(Cp);
   p.b_off0 = 0; p.b_off1 = static_cast<int32_t>(Cp); p.b_off2 = 0;
   p.status = ctx->at<uint32_t>(ctx->lay.status);
@@ -1056,9 +1070,11 @@ int factors_split(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const fl
                                                                      As + off * 2 * L.colsp, L.colsp);
     count_launch();
     CKC(cudaGetLastError());
-    int rc = split_product<F_STORE>(ctx, off, n, As, Ws, rows, L.colsp, U, L.ldu, p);   // z_i = W v_i
+    float* U2 = ctx->at<float>(L.U2);
+    int parts = 1;
+    int rc = split_product<F_STORE>(ctx, off, n, As, Ws, rows, L.colsp, U, L.ldu, p, U2 - U, &parts);   // z_i = W v_i
     if (rc) return rc;
-    CKC(dml_scale_rows(s, U + off * L.ldu, n, rows, L.ldu, labels, c.dml_margin));
+    CKC(dml_scale_rows(s, U + off * L.ldu, n, rows, L.ldu, labels, c.dml_margin, parts > 1 ? U2 + off * L.ldu : nullptr));
     return SFB_OK;
   }
   // sparse coding: ISTA from a = 0, then u = W a - x, v = a
