@@ -50,7 +50,8 @@ struct TcParams {
   int32_t M, N, Kc;            // extents of the product: samples, output columns, contraction
   int32_t m_off;               // first sample handled by this launch (per-worker slices)
   int32_t tilesM, tilesN;
-  int32_t bn;                  // columns per tile: a multiple of 32, at most BN (chosen so that the tiles fill the SMs)
+  int32_t bn;                  // columns per tile, at most BN (chosen so that the tiles fill the SMs): a multiple of 32
+                               // in forward_kernel, of 16 in forward_split_kernel
   // The contraction runs over nseg segments of kseg k-blocks; segment s reads A from column a_off<s> and B from
   // column b_off<s> of their tensors: one segment is the plain product, three segments over [hi | lo] operand
   // halves form the split-bf16 product hi*hi + hi*lo + lo*hi.  (Scalars: an indexed array would send the whole
@@ -377,26 +378,28 @@ forward_split_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       if (!__all_sync(0xffffffffu, mbar_wait(&tfull[a], aph, abort_flag))) { ok = false; break; }
       tc_fence_after();
       const int row = m0 + q * 32 + lane;
-      for (int c = 0; c < p.bn / kChunk; ++c) {
+      // the tile's columns end at nlim; its width is a multiple of 16, so the last 32-column chunk may be half used
+      const int nlim = min(p.N, n0 + p.bn);
+      for (int c = 0; c < (p.bn + kChunk - 1) / kChunk; ++c) {
         uint32_t acc[32];
         tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + a * BN + c * kChunk, acc);
         tmem_ld_wait();
         const int col0 = n0 + c * kChunk;
-        if (col0 >= p.N || row >= p.M) continue;
-        const bool whole = col0 + 32 <= p.N;
+        if (col0 >= nlim || row >= p.M) continue;
         if constexpr (EPI == F_SUB || EPI == F_ISTA) {
-          // the sample's 32 values of aux (x, or the current code a) are contiguous: 128 bytes per lane
+          // the sample's values of aux (x, or the current code a) are contiguous: up to 128 bytes per lane
           float xv[32];
           const float* ap = p.aux + static_cast<int64_t>(row) * p.ldaux + col0;
-          if (whole && ((reinterpret_cast<uintptr_t>(ap) & 15u) == 0)) {
+          const bool ap16 = (reinterpret_cast<uintptr_t>(ap) & 15u) == 0;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
+          for (int j = 0; j < 8; ++j) {
+            if (ap16 && col0 + 4 * j + 4 <= nlim) {
               const float4 v4 = *reinterpret_cast<const float4*>(ap + 4 * j);
               xv[4 * j] = v4.x; xv[4 * j + 1] = v4.y; xv[4 * j + 2] = v4.z; xv[4 * j + 3] = v4.w;
-            }
-          } else {
+            } else {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) xv[j] = col0 + j < p.N ? ap[j] : 0.f;
+              for (int e = 0; e < 4; ++e) xv[4 * j + e] = col0 + 4 * j + e < nlim ? ap[4 * j + e] : 0.f;
+            }
           }
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
@@ -404,11 +407,13 @@ forward_split_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             const float v = EPI == F_SUB ? d - xv[j] : soft_threshold(fmaf(-d, invL, xv[j]), thr);
             acc[j] = __float_as_uint(col0 + j < p.N ? v : 0.f);
           }
-          // (hi | lo) bf16 pair of the result: the operand of the next product
+          // (hi | lo) bf16 pair of the result: the operand of the next product (zero in the padding past N; the
+          // columns past this tile's width belong to the next tile)
           __nv_bfloat16* hp = p.split + static_cast<int64_t>(row) * p.ld_split + col0;
+          const int split_lim = min(p.split_half, n0 + p.bn);
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-            if (col0 + 8 * j < p.split_half) {
+            if (col0 + 8 * j < split_lim) {
               uint32_t hi[4], lo[4];
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
@@ -424,16 +429,18 @@ forward_split_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             }
           }
         }
-        // the fp32 result: this lane's 32 consecutive columns of its row
+        // the fp32 result: this lane's consecutive columns of its row
         float* cp = Cp + static_cast<int64_t>(row) * ldc + col0;
-        if (whole && ((reinterpret_cast<uintptr_t>(cp) & 15u) == 0)) {
+        const bool cp16 = (reinterpret_cast<uintptr_t>(cp) & 15u) == 0;
 #pragma unroll
-          for (int j = 0; j < 8; ++j)
+        for (int j = 0; j < 8; ++j) {
+          if (cp16 && col0 + 4 * j + 4 <= nlim) {
             *reinterpret_cast<uint4*>(cp + 4 * j) = make_uint4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
-        } else {
+          } else {
 #pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (col0 + j < p.N) cp[j] = __uint_as_float(acc[j]);
+            for (int e = 0; e < 4; ++e)
+              if (col0 + 4 * j + e < nlim) cp[4 * j + e] = __uint_as_float(acc[4 * j + e]);
+          }
         }
       }
       tc_fence_before();
@@ -990,15 +997,16 @@ inline unsigned grid1d(int64_t items, int per_block) {
   return static_cast<unsigned>(std::max<int64_t>(1, std::min<int64_t>(g, static_cast<int64_t>(sm_count()) * 16)));
 }
 
-// Tile width (a multiple of 32, at most BN) for a product with tilesM row blocks and N columns on `sms` SMs.  The
+// Tile width (a multiple of `step` columns, at most `widest`) for a product with tilesM row blocks and N columns on
+// `sms` SMs.  The
 // persistent kernel runs ceil(tiles / sms) rounds of tiles; measured, a tile costs about max(width, 128) + 16
 // column-equivalents (below 128 columns a k-block is bound by the latency of its operand loads, not by the MMA).
 // Narrower tiles fill the SMs of small products, where 256-wide ones leave many idle or need a nearly empty
 // second round; ties go to the wider tile.
-inline int pick_tile_width(int sms, int64_t tilesM, int64_t N, int widest) {
+inline int pick_tile_width(int sms, int64_t tilesM, int64_t N, int widest, int step = 32) {
   int best = widest;
   int64_t best_cost = INT64_MAX;
-  for (int bn = widest; bn >= 128; bn -= 32) {
+  for (int bn = widest; bn >= 128; bn -= step) {
     const int64_t tiles = tilesM * ((N + bn - 1) / bn);
     const int64_t cost = ((tiles + sms - 1) / sms) * (bn + 16);
     if (cost < best_cost) { best_cost = cost; best = bn; }
@@ -1014,7 +1022,7 @@ template <int EPI>
 int split_product(sfb_ctx* ctx, int64_t off, int64_t n, __nv_bfloat16* A, __nv_bfloat16* B, int64_t N, int64_t Cp,
                   float* C, int64_t ldc, TcParams p, int64_t c_split_stride = 0, int* parts_out = nullptr) {
   const TcState* st = static_cast<const TcState*>(ctx->tc);
-  const int bn = pick_tile_width(st->sms, (n + BM - 1) / BM, N, FS_BN);
+  const int bn = pick_tile_width(st->sms, (n + BM - 1) / BM, N, FS_BN, 16);
   CUtensorMap ma, mb;
   if (!make_map(st, &ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, A, 2 * Cp, off + n, 2 * Cp * 2, BK, BM) ||
       !make_map(st, &mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, B, 2 * Cp, N, 2 * Cp * 2, BK, bn))
