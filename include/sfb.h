@@ -70,6 +70,8 @@ enum sfb_error {
 #define SFB_STATUS_LABEL_RANGE 0x1u
 #define SFB_STATUS_TIMEOUT     0x2u
 #define SFB_STATUS_SAMPLE_RANGE 0x4u   /* SDCA: a sample id outside [0, sdca_n) was skipped */
+#define SFB_STATUS_INDEX_RANGE 0x8u    /* sparse samples: a column index outside [0, cols), or row pointers that do not
+                                          describe the stated number of entries; the entry or the sample was skipped */
 
 typedef struct sfb_config {
   int32_t model;          /* enum sfb_model                                                            */
@@ -91,6 +93,8 @@ typedef struct sfb_config {
                              entries divided by 1 + eta*w.  Fused into the update pass; for SC it comes before
                              the column rescaling.  Not for SFB_L2MLR (its regulariser lives in the dual).     */
   float   prox_weight;    /* the weight w of that regulariser (>= 0)                                  */
+  int64_t csr_nnz_max;    /* MLR: room, in non-zeros per step over all K samples, for samples given in
+                             compressed-sparse-row form (sfb_compute_factors_csr); 0: none                */
   void*   stream;         /* cudaStream_t                                                              */
 } sfb_config;
 
@@ -134,6 +138,34 @@ int sfb_init(const sfb_config* cfg, float* W_dev, void* workspace_dev, size_t wo
  * its own): after such a write call sfb_refresh_operands, or the next forward product runs on the stale copy. */
 int sfb_compute_factors(sfb_ctx* ctx, int32_t worker, const float* X_dev, const float* Y_dev,
                         const int32_t* labels_dev);
+
+/* ---- sparse sufficient factors (MLR) --------------------------------------------------------------------------------
+ * Section 6: the features of the paper's data sets are sparse; the factor v_i = a_i of such a sample is its (index,
+ * value) pairs (Section 3: what a worker broadcasts).  sfb_compute_factors_csr is sfb_compute_factors for samples in
+ * compressed-sparse-row form: sample i of the call holds the entries indices_dev[indptr_dev[i] .. indptr_dev[i+1]) /
+ * values_dev[same range], column indices int32 in [0, cols), distinct within a sample, in any order; indptr_dev has
+ * B + 1 (worker >= 0) or K + 1 (worker = -1) int64 entries, and nnz = indptr[last] - indptr[0] is stated by the caller
+ * (the library does not read device memory on the host).  The entries of all workers of a step must fit
+ * cfg.csr_nnz_max (SFB_ERR_SHAPE otherwise; SFB_ERR_UNSUPPORTED when it is 0 or the model is not SFB_MLR).  A worker
+ * commits once per step in this form (SFB_ERR_STATE on a second call).  A column index out of range, or row pointers
+ * that are not ascending within [indptr[0], indptr[0] + nnz], set SFB_STATUS_INDEX_RANGE and the entry (the sample) is
+ * left out.  All arrays are copied or consumed before the call returns control of them to the stream order: they may
+ * be reused once later work on the stream may overwrite them.
+ *
+ * u is computed as for dense samples (the logits need every column of W, so the forward product is the dense one over
+ * the scattered samples).  When every worker of the step committed in this form, sfb_gather_factors builds the
+ * column-major form of the K samples (entries of a column in ascending sample order, so the result does not depend on
+ * scheduling) and sfb_apply_update sums, per entry of W, only the samples that have a non-zero in that column:
+ *     W[j][d] <- prox( W[j][d] - eta * sum_{i : x_id != 0} u_ij x_id ),
+ * one pass over W as in the dense update, the derived operand copies of W rewritten with it.  sfb_stats.gather_bytes
+ * then counts K*rows*element size for the u and 8 bytes per non-zero for the v.  A mini-batch too large for the
+ * kernel's on-chip factor slab (K above about 1200 in the fp32 modes, 2400 in bf16 mode) takes the dense update. */
+int sfb_compute_factors_csr(sfb_ctx* ctx, int32_t worker, const int64_t* indptr_dev, const int32_t* indices_dev,
+                            const float* values_dev, int64_t nnz, const int32_t* labels_dev);
+
+/* sfb_compute_factors_csr(worker = -1) -> sfb_gather_factors -> sfb_apply_update. */
+int sfb_step_csr(sfb_ctx* ctx, const int64_t* indptr_dev, const int32_t* indices_dev, const float* values_dev,
+                 int64_t nnz, const int32_t* labels_dev);
 
 /* ---- l2-regularised MLR by stochastic dual coordinate ascent (model SFB_L2MLR) ------------------------------------
  * Section 2.1 "Stochastic DCA": with the dual matrix U = [u_1 .. u_N], Z = 1/N U A^T and W = grad h^*(Z) = Z / lam, a

@@ -14,14 +14,15 @@ from .build import LIB, build
 MLR, DML, SC, L2MLR = 0, 1, 2, 3
 PREC_BF16, PREC_FP32, PREC_TF32X3, PREC_FP32_FFMA = 0, 1, 2, 3
 PROX_NONE, PROX_L1, PROX_L2SQ = 0, 1, 2
-STATUS_LABEL_RANGE, STATUS_TIMEOUT, STATUS_SAMPLE_RANGE = 0x1, 0x2, 0x4
+STATUS_LABEL_RANGE, STATUS_TIMEOUT, STATUS_SAMPLE_RANGE, STATUS_INDEX_RANGE = 0x1, 0x2, 0x4, 0x8
 
 EXPORTS = ("sfb_workspace_bytes", "sfb_init", "sfb_compute_factors", "sfb_gather_factors", "sfb_apply_update",
            "sfb_step", "sfb_step_host", "sfb_dense_sync_step", "sfb_get_factors", "sfb_get_stats",
            "sfb_get_status", "sfb_strerror", "sfb_last_cuda_error", "sfb_destroy", "sfb_prox_columns_noalloc",
            "sfb_selftest_wait_timeout", "sfb_set_row_shard", "sfb_forward_partials", "sfb_finish_factors",
            "sfb_replay_update", "sfb_refresh_operands", "sfb_sdca_set_dual", "sfb_sdca_compute_factors",
-           "sfb_sdca_step", "sfb_set_factors", "sfb_set_eta", "sfb_get_operand_copy")
+           "sfb_sdca_step", "sfb_set_factors", "sfb_set_eta", "sfb_get_operand_copy", "sfb_compute_factors_csr",
+           "sfb_step_csr")
 NOALLOC_MAX_COLS = 16384
 
 
@@ -31,7 +32,7 @@ class sfb_config(ctypes.Structure):
                 ("eta", ctypes.c_float), ("dml_margin", ctypes.c_float), ("sc_lambda", ctypes.c_float),
                 ("sc_ista_iters", ctypes.c_int32), ("sc_lipschitz", ctypes.c_float), ("sc_prox", ctypes.c_int32),
                 ("sdca_lambda", ctypes.c_float), ("sdca_n", ctypes.c_int64), ("prox_kind", ctypes.c_int32),
-                ("prox_weight", ctypes.c_float), ("stream", ctypes.c_void_p)]
+                ("prox_weight", ctypes.c_float), ("csr_nnz_max", ctypes.c_int64), ("stream", ctypes.c_void_p)]
 
 
 class sfb_stats(ctypes.Structure):
@@ -92,6 +93,8 @@ def lib() -> ctypes.CDLL:
         L.sfb_set_factors.argtypes = [vp, i32, vp, vp]
         L.sfb_set_eta.argtypes = [vp, ctypes.c_float]
         L.sfb_get_operand_copy.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(i32), ctypes.POINTER(i64)]
+        L.sfb_compute_factors_csr.argtypes = [vp, i32, vp, vp, vp, i64, vp]
+        L.sfb_step_csr.argtypes = [vp, vp, vp, vp, i64, vp]
         for name in EXPORTS:
             if name != "sfb_strerror":
                 getattr(L, name).restype = ctypes.c_int
@@ -105,9 +108,9 @@ def strerror(code: int) -> str:
 
 def make_config(model, rows, cols, workers, batch, eta, precision=PREC_FP32, dml_margin=1.0, sc_lambda=0.1,
                 sc_ista_iters=20, sc_lipschitz=0.0, sc_prox=0, stream=0, sdca_lambda=0.0, sdca_n=0, prox_kind=0,
-                prox_weight=0.0) -> sfb_config:
+                prox_weight=0.0, csr_nnz_max=0) -> sfb_config:
     return sfb_config(model, precision, rows, cols, workers, batch, eta, dml_margin, sc_lambda, sc_ista_iters,
-                      sc_lipschitz, sc_prox, sdca_lambda, sdca_n, prox_kind, prox_weight, stream)
+                      sc_lipschitz, sc_prox, sdca_lambda, sdca_n, prox_kind, prox_weight, csr_nnz_max, stream)
 
 
 def sfb_workspace_bytes(cfg: sfb_config) -> int:
@@ -189,6 +192,14 @@ class Context:
 
     def sfb_step(self, X, Y=None, labels=None):
         self._ck(lib().sfb_step(self._h, _ptr(X), _ptr(Y), _ptr(labels)), "sfb_step")
+
+    def sfb_compute_factors_csr(self, worker, indptr, indices, values, nnz, labels):
+        """indptr int64 [B+1 or K+1], indices int32, values fp32, labels int32: CUDA tensors; nnz = entries of the call."""
+        self._ck(lib().sfb_compute_factors_csr(self._h, worker, _ptr(indptr), _ptr(indices), _ptr(values), nnz,
+                                               _ptr(labels)), "sfb_compute_factors_csr")
+
+    def sfb_step_csr(self, indptr, indices, values, nnz, labels):
+        self._ck(lib().sfb_step_csr(self._h, _ptr(indptr), _ptr(indices), _ptr(values), nnz, _ptr(labels)), "sfb_step_csr")
 
     def sfb_step_host(self, X, Y=None, labels=None):
         """X, Y, labels: host tensors / numpy arrays (pinned recommended).  Returns (mean loss, status word)."""

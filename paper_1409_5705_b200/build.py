@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsfb.so")
-SOURCES = ["sfb_api.cu", "sfb_simt.cu", "sfb_factors.cu", "sfb_tc.cu", "sfb_update.cu", "sfb_selftest.cu"]
+SOURCES = ["sfb_api.cu", "sfb_simt.cu", "sfb_factors.cu", "sfb_tc.cu", "sfb_update.cu", "sfb_sparse.cu", "sfb_selftest.cu"]
 
 
 def _nvcc() -> str:

@@ -53,6 +53,7 @@ Layout make_layout(const sfb_config& cfg) {
   } else {
     tc_extend_layout(c, L, off);
   }
+  if (c.csr_nnz_max > 0 && c.model == SFB_MLR) sparse_extend_layout(c, L, off);
   L.total = off;
   return L;
 }
@@ -88,6 +89,7 @@ static int check_config(const sfb_config* c) {
   if (c->sc_prox < 0 || c->sc_prox > 1) return SFB_ERR_ARG;
   if (c->prox_kind < 0 || c->prox_kind > 2 || !(c->prox_weight >= 0.f)) return SFB_ERR_ARG;
   if (c->model == SFB_L2MLR && c->prox_kind != 0) return SFB_ERR_UNSUPPORTED;
+  if (c->csr_nnz_max < 0 || c->csr_nnz_max + c->cols > (1LL << 31) - 64) return SFB_ERR_SHAPE;
   return SFB_OK;
 }
 
@@ -137,6 +139,9 @@ extern "C" int sfb_init(const sfb_config* cfg, float* W_dev, void* workspace_dev
   ctx->K = static_cast<int64_t>(cfg->workers) * cfg->batch;
   ctx->in_dim = cfg->model == SFB_SC ? cfg->rows : cfg->cols;
   ctx->committed = 0;
+  ctx->sparse_mask = 0;
+  ctx->csr_fill = 0;
+  ctx->sparse_v = false;
   ctx->gathered = false;
   ctx->row_offset = 0;
   ctx->global_rows = cfg->rows;
@@ -215,6 +220,7 @@ static int factors_fp32(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, co
 
 static int update_fp32(sfb_ctx* ctx) {
   const sfb_config& c = ctx->cfg;
+  if (ctx->sparse_v) return sparse_update(ctx);
   EpiArgs e{};
   e.C = ctx->W; e.ldc = c.cols; e.alpha = -ctx->step;
   e.prox_kind = ctx->prox_kind; e.prox_a = ctx->prox_a;
@@ -242,6 +248,8 @@ extern "C" int sfb_compute_factors(sfb_ctx* ctx, int32_t worker, const float* X_
   const int64_t off = worker < 0 ? 0 : static_cast<int64_t>(worker) * c.batch;
   const int64_t n = worker < 0 ? ctx->K : c.batch;
   if (ctx->committed == 0) {
+    ctx->sparse_mask = 0;
+    ctx->csr_fill = 0;
     CK(cudaEventRecord(ctx->ev[0], ctx->stream));
     // the coder's step size comes from the W every worker sees at the start of the step (BSP)
     if (c.model == SFB_SC && !(c.sc_lipschitz > 0.f))
@@ -257,8 +265,57 @@ extern "C" int sfb_compute_factors(sfb_ctx* ctx, int32_t worker, const float* X_
   if (rc) return rc;
   const uint64_t all = c.workers == 64 ? ~0ull : ((1ull << c.workers) - 1);
   ctx->committed |= worker < 0 ? all : (1ull << worker);
+  ctx->sparse_mask &= ~(worker < 0 ? all : (1ull << worker));       // these samples are dense
   ctx->gathered = false;
   return SFB_OK;
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Samples in compressed-sparse-row form (MLR): scattered for the dense forward product, and kept as triples for the
+// column-major form that the update reads
+// ---------------------------------------------------------------------------------------------------------
+extern "C" int sfb_compute_factors_csr(sfb_ctx* ctx, int32_t worker, const int64_t* indptr_dev, const int32_t* indices_dev,
+                                       const float* values_dev, int64_t nnz, const int32_t* labels_dev) {
+  if (!ctx || !indptr_dev || !labels_dev || nnz < 0) return SFB_ERR_ARG;
+  if (nnz > 0 && (!indices_dev || !values_dev)) return SFB_ERR_ARG;
+  const sfb_config& c = ctx->cfg;
+  if (c.model != SFB_MLR || ctx->sdca || c.csr_nnz_max <= 0) return SFB_ERR_UNSUPPORTED;
+  if (worker < -1 || worker >= c.workers) return SFB_ERR_SHAPE;
+  if (ctx->partials_ready) return SFB_ERR_STATE;
+  const uint64_t all = c.workers == 64 ? ~0ull : ((1ull << c.workers) - 1);
+  const uint64_t bits = worker < 0 ? all : (1ull << worker);
+  if (ctx->committed == 0) {
+    ctx->sparse_mask = 0;
+    ctx->csr_fill = 0;
+  }
+  if (ctx->sparse_mask & bits) return SFB_ERR_STATE;                // its triples are already in the step's list
+  if (ctx->csr_fill + nnz > c.csr_nnz_max) return SFB_ERR_SHAPE;
+  const int64_t off = worker < 0 ? 0 : static_cast<int64_t>(worker) * c.batch;
+  const int64_t n = worker < 0 ? ctx->K : c.batch;
+  if (ctx->committed == 0) CK(cudaEventRecord(ctx->ev[0], ctx->stream));
+  int rc = sparse_stage(ctx, off, n, indptr_dev, indices_dev, values_dev, nnz);
+  if (rc) return rc;
+  const float* X = ctx->at<float>(ctx->lay.stageX) + off * c.cols;
+  rc = ctx->tf32 ? tc32_factors(ctx, off, n, X, labels_dev, nullptr, 0.f)
+       : c.precision == SFB_PREC_FP32 ? factors_fp32(ctx, off, n, X, nullptr, labels_dev)
+                                      : tc_factors(ctx, off, n, X, nullptr, labels_dev);
+  if (rc) return rc;
+  ctx->csr_fill += nnz;
+  ctx->sparse_mask |= bits;
+  ctx->committed |= bits;
+  ctx->gathered = false;
+  return SFB_OK;
+}
+
+extern "C" int sfb_step_csr(sfb_ctx* ctx, const int64_t* indptr_dev, const int32_t* indices_dev, const float* values_dev,
+                            int64_t nnz, const int32_t* labels_dev) {
+  if (!ctx) return SFB_ERR_ARG;
+  ctx->committed = 0;
+  int rc = sfb_compute_factors_csr(ctx, -1, indptr_dev, indices_dev, values_dev, nnz, labels_dev);
+  if (rc) return rc;
+  rc = sfb_gather_factors(ctx);
+  if (rc) return rc;
+  return sfb_apply_update(ctx);
 }
 
 // ---------------------------------------------------------------------------------------------------------
@@ -370,7 +427,12 @@ extern "C" int sfb_gather_factors(sfb_ctx* ctx) {
   CK(cudaEventRecord(ctx->ev[1], ctx->stream));
   // Every worker wrote its pairs at row offset p*B of the shared buffers, so the gathered operands are
   // complete; what remains is the per-step read-out over all K pairs.
-  if (c.precision == SFB_PREC_BF16 || ctx->tf32) {
+  // all K samples sparse: the v become their column-major form (and the dense update operands are not needed)
+  ctx->sparse_v = c.model == SFB_MLR && c.csr_nnz_max > 0 && ctx->sparse_mask == all && sparse_update_fits(ctx);
+  if (ctx->sparse_v) {
+    int rc = sparse_build_csc(ctx);
+    if (rc) return rc;
+  } else if (c.precision == SFB_PREC_BF16 || ctx->tf32) {
     int rc = ctx->tf32 ? tc32_gather(ctx) : tc_gather(ctx);
     if (rc) return rc;
   }
@@ -379,7 +441,9 @@ extern "C" int sfb_gather_factors(sfb_ctx* ctx) {
                &ctx->at<Scalars>(ctx->lay.scalars)->loss_mean));
   // bytes per gathered value: fp32, bf16, or a (hi, lo) pair of bf16 for the split operands of DML and SC
   const double esz = (c.precision == SFB_PREC_FP32 || c.model != SFB_MLR) ? 4.0 : 2.0;
-  const double pair = static_cast<double>(c.rows + c.cols) * esz;
+  // sparse v: 8 bytes (index, value) per non-zero instead of cols values per sample
+  const double pair = ctx->sparse_v ? static_cast<double>(c.rows) * esz + 8.0 * static_cast<double>(ctx->csr_fill) / ctx->K
+                                    : static_cast<double>(c.rows + c.cols) * esz;
   ctx->stats.gather_bytes += static_cast<double>(ctx->K) * pair;
   ctx->stats.gather_bytes_p2p += static_cast<double>(c.workers) * (c.workers - 1) * c.batch * pair;
   ctx->stats.dense_sync_bytes += static_cast<double>(c.workers) * c.rows * c.cols * 4.0;

@@ -30,6 +30,8 @@ struct Layout {
   // bf16 mode, DML and SC: (hi | lo) bf16 operands of the split products
   size_t Ws, WTs, As, Rs;             // W by rows, W transposed, the A operand (v or the codes), the residual
   size_t U2;                          // DML: second partial of z when the forward product splits its contraction
+  // sparse factors (MLR, csr_nnz_max > 0): the step's (sample, column, value) triples and their column-major form
+  size_t coo_i, coo_c, coo_x, csc_cnt, csc_cur, csc_ptr, csc_tmp, csc_ent;
   int64_t ldu;                        // row pitch of the fp32 U buffer (rows rounded up to 4 in bf16 mode)
   int64_t colsp, rowsp;               // cols, rows rounded up to 64
   int64_t Kp;                         // K rounded up to the contraction block of the update product
@@ -79,6 +81,9 @@ struct sfb_ctx {
   int32_t prox_kind;                  // entry-wise prox of the update pass and its parameter (threshold or factor)
   float prox_a;
   uint64_t committed;                 // bit p set: worker p has written its factors since the last update
+  uint64_t sparse_mask;               // bit p set: worker p's samples of this step came in compressed-sparse-row form
+  int64_t csr_fill;                   // triples staged so far in this step
+  bool sparse_v;                      // the gathered v are in column-major sparse form: the update sums only the non-zeros
   bool gathered;
   int last_cuda;
   cudaEvent_t ev[4];
@@ -149,5 +154,15 @@ cudaError_t estimate_lipschitz(cudaStream_t s, const float* W, int64_t rows, int
 cudaError_t set_lipschitz(cudaStream_t s, Scalars* sc, float L);
 cudaError_t axpy(cudaStream_t s, float* y, const float* x, float alpha, int64_t n);  // y += alpha*x
 cudaError_t prox_entries(cudaStream_t s, float* w, int64_t n, int kind, float a);      // w <- prox(w), entry-wise
+
+// ---------------------------------------------------------------------------------------------------------
+// Sparse sufficient factors (MLR): staging of compressed-sparse-row samples, their column-major form, the update
+// ---------------------------------------------------------------------------------------------------------
+void sparse_extend_layout(const sfb_config& c, Layout& L, size_t& off);
+bool sparse_update_fits(const sfb_ctx* ctx);          // the factor slab of K samples fits the shared memory of a block
+int sparse_stage(sfb_ctx* ctx, int64_t off, int64_t n, const int64_t* indptr, const int32_t* idx, const float* val,
+                 int64_t nnz);
+int sparse_build_csc(sfb_ctx* ctx);
+int sparse_update(sfb_ctx* ctx);
 
 }  // namespace sfb

@@ -1,0 +1,413 @@
+// Sparse sufficient factors of multiclass logistic regression (Section 6: the features of the paper's data sets are
+// sparse; Section 3: a factor v_i = a_i with few non-zeros is sent as its (index, value) pairs).
+//
+// The samples arrive in compressed-sparse-row form.  Their logits still need every column of W (the union of the
+// non-zero columns of a mini-batch covers the matrix), so the forward product stays the dense tensor-core product
+// over the scattered samples.  What the zeros remove is the work of the update:
+//     W[j][d] <- prox( W[j][d] - eta * sum_{i : x_id != 0} u_ij x_id )
+// has as many terms per entry as column d has non-zeros in the mini-batch (K * density) instead of K.  The kernel here
+// streams W once, as the dense update does, and sums only those terms, from the column-major (CSC) form of the
+// mini-batch that the gather step builds.
+#include <cuda_bf16.h>
+
+#include <algorithm>
+
+#include "sfb_internal.h"
+
+namespace sfb {
+
+namespace {
+
+constexpr unsigned kFull = 0xffffffffu;
+constexpr int kSuWarps = 16;                       // warps per block of the update kernel
+constexpr int kSuThreads = kSuWarps * 32;
+constexpr int kSuStage = 32 * 33;                  // floats of one warp's transpose buffer
+constexpr int kSmemOptIn = 232448 - 1024;          // dynamic shared memory asked for: what a block may opt into, less the static part
+
+inline unsigned grid1d(int64_t n, int block, int cap = 148 * 16) {
+  return static_cast<unsigned>(std::max<int64_t>(1, std::min<int64_t>((n + block - 1) / block, cap)));
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Staging of a worker's CSR block: the dense fp32 samples for the forward product, and (sample, column, value)
+// triples appended to the step's list for the column-major form.  One warp per sample.
+// ---------------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) csr_stage_kernel(const int64_t* __restrict__ indptr, const int32_t* __restrict__ idx,
+                                                        const float* __restrict__ val, int64_t n, int64_t nnz, int64_t cols,
+                                                        int64_t off, float* __restrict__ Xd, int32_t* __restrict__ coo_i,
+                                                        int32_t* __restrict__ coo_c, float* __restrict__ coo_x,
+                                                        uint32_t* __restrict__ status) {
+  const int64_t i = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (i >= n) return;
+  const int64_t base = indptr[0];
+  const int64_t b = indptr[i] - base, e = indptr[i + 1] - base;
+  if (b < 0 || e < b || e > nnz) {                 // row pointers that do not describe nnz entries: sample left empty
+    if (lane == 0) atomicOr(status, SFB_STATUS_INDEX_RANGE);
+    return;
+  }
+  for (int64_t t = b + lane; t < e; t += 32) {
+    const int32_t c = idx[base + t];
+    const float x = val[base + t];
+    if (c < 0 || c >= cols) {                      // entry skipped (its slot keeps the "no entry" mark)
+      atomicOr(status, SFB_STATUS_INDEX_RANGE);
+      continue;
+    }
+    Xd[(off + i) * cols + c] = x;
+    coo_i[t] = static_cast<int32_t>(off + i);
+    coo_c[t] = c;
+    coo_x[t] = x;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Column-major form of the step's K samples: a counting sort of the triples by column, then every column's
+// entries in ascending sample order (so that the sums of the update have one order, whatever order the atomics
+// of the fill took).  Column d owns ent[ptr[d] .. ptr[d+1]); its length is rounded up to an even number with a
+// (sample K, value 0) entry, which points at an all-zero row of the factor slab.
+// ---------------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) csc_count_kernel(const int32_t* __restrict__ coo_c, int64_t nnz, int32_t* __restrict__ cnt) {
+  const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+  for (int64_t t = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; t < nnz; t += stride) {
+    const int32_t c = coo_c[t];
+    if (c >= 0) atomicAdd(&cnt[c], 1);
+  }
+}
+
+__global__ void __launch_bounds__(1024) csc_scan_kernel(const int32_t* __restrict__ cnt, int64_t cols, int32_t* __restrict__ ptr) {
+  __shared__ int32_t part[1024];
+  const int t = threadIdx.x;
+  const int64_t chunk = (cols + 1023) / 1024;
+  const int64_t lo = t * chunk < cols ? t * chunk : cols, hi = lo + chunk < cols ? lo + chunk : cols;
+  int32_t s = 0;
+  for (int64_t d = lo; d < hi; ++d) s += (cnt[d] + 1) & ~1;
+  part[t] = s;
+  __syncthreads();
+  for (int o = 1; o < 1024; o <<= 1) {             // inclusive scan of the 1024 chunk sums
+    const int32_t v = t >= o ? part[t - o] : 0;
+    __syncthreads();
+    part[t] += v;
+    __syncthreads();
+  }
+  int32_t run = t > 0 ? part[t - 1] : 0;
+  for (int64_t d = lo; d < hi; ++d) {
+    ptr[d] = run;
+    run += (cnt[d] + 1) & ~1;
+  }
+  if (t == 1023) ptr[cols] = part[1023];
+}
+
+__global__ void __launch_bounds__(256) csc_fill_kernel(const int32_t* __restrict__ coo_i, const int32_t* __restrict__ coo_c,
+                                                       const float* __restrict__ coo_x, int64_t nnz,
+                                                       const int32_t* __restrict__ ptr, int32_t* __restrict__ cur,
+                                                       int2* __restrict__ tmp) {
+  const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+  for (int64_t t = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; t < nnz; t += stride) {
+    const int32_t c = coo_c[t];
+    if (c < 0) continue;
+    const int32_t pos = ptr[c] + atomicAdd(&cur[c], 1);
+    tmp[pos] = make_int2(coo_i[t], __float_as_int(coo_x[t]));
+  }
+}
+
+// One block per column (grid-stride): rank of every entry among the column's entries by sample index.
+__global__ void __launch_bounds__(128) csc_sort_kernel(const int2* __restrict__ tmp, const int32_t* __restrict__ ptr,
+                                                       const int32_t* __restrict__ cnt, int64_t cols, int32_t K,
+                                                       int2* __restrict__ ent) {
+  for (int64_t d = blockIdx.x; d < cols; d += gridDim.x) {
+    const int32_t n = cnt[d], b = ptr[d];
+    for (int32_t e = threadIdx.x; e < n; e += blockDim.x) {
+      const int2 me = tmp[b + e];
+      int32_t rank = 0;
+      for (int32_t f = 0; f < n; ++f) {
+        const int32_t o = tmp[b + f].x;
+        rank += (o < me.x || (o == me.x && f < e)) ? 1 : 0;
+      }
+      ent[b + rank] = me;
+    }
+    if (threadIdx.x == 0 && (n & 1)) ent[b + n] = make_int2(K, 0);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// The update.  A block owns 32 rows of W at a time and keeps their factor slab u[i][row] (all K samples) in shared
+// memory; its warps take 32-column blocks of those rows.  Within a block of 32 x 32 entries a lane first is a ROW:
+// for each of the 32 columns it sums x_id * u[i][row] over the column's entries (the entries are read by all lanes at
+// once, the slab row by row without bank conflicts).  The 32 x 32 sums are then transposed through shared memory so
+// that a lane is a COLUMN and each row's 32 entries of W leave as one 128-byte piece.
+//   USRC 0: factors fp32, sample-major [K x ldu] (fp32 modes);  1: bf16, transposed [rows x ldut] (bf16 mode, whose
+//           label entries are applied separately in fp32).
+//   SHADOW 0: none;  1: bf16 operand copy of W, a 64-byte row piece rewritten only if one of its roundings changed;
+//           2: the (big | small) tf32 copy.
+// ---------------------------------------------------------------------------------------------------------
+struct SuParams {
+  float* W;
+  int64_t rows, cols;
+  const int32_t* ptr;
+  const int2* ent;
+  const float* U;
+  int64_t ldu;
+  const __nv_bfloat16* UT;
+  int64_t ldut;
+  int32_t K;
+  float alpha;
+  int32_t prox_kind;
+  float prox_a;
+  __nv_bfloat16* shadow;
+  int64_t shadow_ld;
+  float* shadow32;
+  int64_t shadow32_ld, shadow_half;
+  unsigned long long* copy_counters;
+};
+
+template <int USRC>
+struct Slab {
+  static constexpr int kPitch = USRC == 0 ? 33 * 4 : 34 * 2;      // bytes per sample: 32 rows, padded to an odd word count
+  static __device__ __forceinline__ float load(const uint8_t* us, int32_t i, int lane) {
+    if (USRC == 0) return *reinterpret_cast<const float*>(us + i * kPitch + lane * 4);
+    return __uint_as_float(static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(us + i * kPitch + lane * 2)) << 16);
+  }
+};
+
+__device__ __forceinline__ float tf32_round(float x) {
+  uint32_t u;
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(u) : "f"(x));
+  return __uint_as_float(u);
+}
+
+template <int USRC, int SHADOW>
+__global__ void __launch_bounds__(kSuThreads, 1) sparse_update_kernel(const SuParams p) {
+  extern __shared__ __align__(16) uint8_t su_smem[];
+  __shared__ int next_cb;
+  using S = Slab<USRC>;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  uint8_t* us = su_smem;
+  const int slab_bytes = ((p.K + 1) * S::kPitch + 15) & ~15;
+  float* stg = reinterpret_cast<float*>(su_smem + slab_bytes) + warp * kSuStage;
+  const int nrb = static_cast<int>((p.rows + 31) / 32), ncb = static_cast<int>((p.cols + 31) / 32);
+  // sample K of the slab is all zero: the padding entries of odd columns point there
+  for (int t = threadIdx.x; t < S::kPitch / 2; t += kSuThreads) reinterpret_cast<uint16_t*>(us + p.K * S::kPitch)[t] = 0;
+  unsigned long long pieces = 0, written = 0;
+
+  for (int rb = blockIdx.x; rb < nrb; rb += gridDim.x) {
+    const int64_t r0 = static_cast<int64_t>(rb) * 32;
+    __syncthreads();                                   // every warp is done with the previous slab
+    if (USRC == 0) {
+      const bool rv = r0 + lane < p.rows;
+      for (int i = warp; i < p.K; i += kSuWarps)
+        *reinterpret_cast<float*>(us + i * S::kPitch + lane * 4) = rv ? p.U[static_cast<int64_t>(i) * p.ldu + r0 + lane] : 0.f;
+    } else {
+      for (int r = warp; r < 32; r += kSuWarps) {
+        const bool rv = r0 + r < p.rows;
+        const uint16_t* src = reinterpret_cast<const uint16_t*>(p.UT) + (r0 + r) * p.ldut;
+        for (int i = lane; i < p.K; i += 32)
+          *reinterpret_cast<uint16_t*>(us + i * S::kPitch + r * 2) = rv ? src[i] : static_cast<uint16_t>(0);
+      }
+    }
+    if (threadIdx.x == 0) next_cb = 0;
+    __syncthreads();
+
+    for (;;) {
+      int cb = 0;
+      if (lane == 0) cb = atomicAdd(&next_cb, 1);       // which warp takes which block does not change any result
+      cb = __shfl_sync(kFull, cb, 0);
+      if (cb >= ncb) break;
+      const int64_t d = static_cast<int64_t>(cb) * 32 + lane;
+      const bool dv = d < p.cols;
+      // as a column: the 32 rows of W at column d, asked for before the sums so that they arrive meanwhile
+      float wv[32];
+#pragma unroll
+      for (int r = 0; r < 32; ++r) wv[r] = (dv && r0 + r < p.rows) ? p.W[(r0 + r) * p.cols + d] : 0.f;
+      const int32_t pb = p.ptr[dv ? d : p.cols], pe = p.ptr[dv ? d + 1 : p.cols];
+      // as a row: sums over the entries of each of the 32 columns
+      float acc[32];
+#pragma unroll
+      for (int c = 0; c < 32; ++c) {
+        int32_t e = __shfl_sync(kFull, pb, c);
+        const int32_t e1 = __shfl_sync(kFull, pe, c);
+        float a = 0.f;
+        for (; e + 8 <= e1; e += 8) {
+          const int4 t0 = __ldg(reinterpret_cast<const int4*>(p.ent + e));
+          const int4 t1 = __ldg(reinterpret_cast<const int4*>(p.ent + e + 2));
+          const int4 t2 = __ldg(reinterpret_cast<const int4*>(p.ent + e + 4));
+          const int4 t3 = __ldg(reinterpret_cast<const int4*>(p.ent + e + 6));
+          const float u0 = S::load(us, t0.x, lane), u1 = S::load(us, t0.z, lane);
+          const float u2 = S::load(us, t1.x, lane), u3 = S::load(us, t1.z, lane);
+          const float u4 = S::load(us, t2.x, lane), u5 = S::load(us, t2.z, lane);
+          const float u6 = S::load(us, t3.x, lane), u7 = S::load(us, t3.z, lane);
+          a = fmaf(__int_as_float(t0.y), u0, a); a = fmaf(__int_as_float(t0.w), u1, a);
+          a = fmaf(__int_as_float(t1.y), u2, a); a = fmaf(__int_as_float(t1.w), u3, a);
+          a = fmaf(__int_as_float(t2.y), u4, a); a = fmaf(__int_as_float(t2.w), u5, a);
+          a = fmaf(__int_as_float(t3.y), u6, a); a = fmaf(__int_as_float(t3.w), u7, a);
+        }
+        for (; e < e1; e += 2) {
+          const int4 t0 = __ldg(reinterpret_cast<const int4*>(p.ent + e));
+          const float u0 = S::load(us, t0.x, lane), u1 = S::load(us, t0.z, lane);
+          a = fmaf(__int_as_float(t0.y), u0, a); a = fmaf(__int_as_float(t0.w), u1, a);
+        }
+        acc[c] = a;
+      }
+#pragma unroll
+      for (int c = 0; c < 32; ++c) stg[c * 33 + lane] = acc[c];
+      __syncwarp();
+#pragma unroll
+      for (int r = 0; r < 32; ++r) {
+        const bool ok = dv && r0 + r < p.rows;
+        const float wo = wv[r];
+        const float wn = prox_entry(fmaf(p.alpha, stg[lane * 33 + r], wo), p.prox_kind, p.prox_a);
+        if (ok) p.W[(r0 + r) * p.cols + d] = wn;
+        if (SHADOW == 1) {
+          const __nv_bfloat16 bo = __float2bfloat16_rn(wo), bn = __float2bfloat16_rn(wn);
+          const bool differs = ok && __bfloat16_as_ushort(bo) != __bfloat16_as_ushort(bn);
+          const bool any = __any_sync(kFull, differs);
+          if (r0 + r < p.rows) {
+            ++pieces;
+            if (any) {
+              ++written;
+              if (ok) p.shadow[(r0 + r) * p.shadow_ld + d] = bn;
+            }
+          }
+        }
+        if (SHADOW == 2 && ok) {
+          const float big = tf32_round(wn);
+          float* sp = p.shadow32 + (r0 + r) * p.shadow32_ld + d;
+          sp[0] = big;
+          sp[p.shadow_half] = tf32_round(wn - big);
+        }
+      }
+      __syncwarp();                                    // the transpose buffer is free again
+    }
+  }
+  if (SHADOW == 1 && p.copy_counters && lane == 0) {
+    atomicAdd(p.copy_counters, pieces);
+    atomicAdd(p.copy_counters + 1, written);
+  }
+}
+
+template <int USRC, int SHADOW>
+cudaError_t launch_sparse_update(cudaStream_t s, const SuParams& p, int smem) {
+  static std::atomic<uint64_t> prepared{0};            // one bit per device ordinal
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const uint64_t bit = 1ull << (dev & 63);
+  if (!(prepared.load(std::memory_order_acquire) & bit)) {
+    e = cudaFuncSetAttribute(sparse_update_kernel<USRC, SHADOW>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemOptIn);
+    if (e != cudaSuccess) return e;
+    prepared.fetch_or(bit, std::memory_order_release);
+  }
+  const int nrb = static_cast<int>((p.rows + 31) / 32);
+  sparse_update_kernel<USRC, SHADOW><<<std::min(nrb, sm_count()), kSuThreads, smem, s>>>(p);
+  count_launch();
+  return cudaGetLastError();
+}
+
+int slab_smem(int64_t K, bool bf16) {
+  const int64_t pitch = bf16 ? 34 * 2 : 33 * 4;
+  const int64_t bytes = (((K + 1) * pitch + 15) & ~int64_t(15)) + static_cast<int64_t>(kSuWarps) * kSuStage * 4;
+  return bytes <= kSmemOptIn ? static_cast<int>(bytes) : -1;
+}
+
+}  // namespace
+
+#define CKS(call)                                       \
+  do {                                                  \
+    cudaError_t e__ = (call);                           \
+    if (e__ != cudaSuccess) {                           \
+      ctx->last_cuda = static_cast<int>(e__);           \
+      return SFB_ERR_CUDA;                              \
+    }                                                   \
+  } while (0)
+
+void sparse_extend_layout(const sfb_config& c, Layout& L, size_t& off) {
+  auto take = [&](size_t bytes) { size_t o = off; off += (bytes + kAlign - 1) / kAlign * kAlign; return o; };
+  const size_t nnz = static_cast<size_t>(c.csr_nnz_max), cols = static_cast<size_t>(c.cols);
+  L.coo_i = take(nnz * 4);
+  L.coo_c = take(nnz * 4);
+  L.coo_x = take(nnz * 4);
+  L.csc_cnt = take((cols + 1) * 4);
+  L.csc_cur = take((cols + 1) * 4);
+  L.csc_ptr = take((cols + 1) * 4);
+  L.csc_tmp = take((nnz + cols) * 8);
+  L.csc_ent = take((nnz + cols + 8) * 8);
+}
+
+bool sparse_update_fits(const sfb_ctx* ctx) {
+  return slab_smem(ctx->K, ctx->cfg.precision == SFB_PREC_BF16) > 0;
+}
+
+int sparse_stage(sfb_ctx* ctx, int64_t off, int64_t n, const int64_t* indptr, const int32_t* idx, const float* val,
+                 int64_t nnz) {
+  const Layout& L = ctx->lay;
+  const int64_t cols = ctx->cfg.cols;
+  cudaStream_t s = ctx->stream;
+  float* Xd = ctx->at<float>(L.stageX);
+  CKS(cudaMemsetAsync(Xd + off * cols, 0, static_cast<size_t>(n) * cols * 4, s));
+  if (nnz > 0) CKS(cudaMemsetAsync(ctx->at<int32_t>(L.coo_c) + ctx->csr_fill, 0xff, static_cast<size_t>(nnz) * 4, s));   // "no entry"
+  csr_stage_kernel<<<static_cast<unsigned>((n * 32 + 255) / 256), 256, 0, s>>>(
+      indptr, idx, val, n, nnz, cols, off, Xd, ctx->at<int32_t>(L.coo_i) + ctx->csr_fill,
+      ctx->at<int32_t>(L.coo_c) + ctx->csr_fill, ctx->at<float>(L.coo_x) + ctx->csr_fill, ctx->at<uint32_t>(L.status));
+  count_launch();
+  CKS(cudaGetLastError());
+  return SFB_OK;
+}
+
+int sparse_build_csc(sfb_ctx* ctx) {
+  const Layout& L = ctx->lay;
+  const int64_t cols = ctx->cfg.cols, nnz = ctx->csr_fill;
+  cudaStream_t s = ctx->stream;
+  int32_t* cnt = ctx->at<int32_t>(L.csc_cnt);
+  int32_t* cur = ctx->at<int32_t>(L.csc_cur);
+  int32_t* ptr = ctx->at<int32_t>(L.csc_ptr);
+  CKS(cudaMemsetAsync(cnt, 0, static_cast<size_t>(cols + 1) * 4, s));
+  CKS(cudaMemsetAsync(cur, 0, static_cast<size_t>(cols + 1) * 4, s));
+  if (nnz > 0) {
+    csc_count_kernel<<<grid1d(nnz, 256), 256, 0, s>>>(ctx->at<int32_t>(L.coo_c), nnz, cnt);
+    count_launch();
+  }
+  csc_scan_kernel<<<1, 1024, 0, s>>>(cnt, cols, ptr);
+  count_launch();
+  if (nnz > 0) {
+    csc_fill_kernel<<<grid1d(nnz, 256), 256, 0, s>>>(ctx->at<int32_t>(L.coo_i), ctx->at<int32_t>(L.coo_c), ctx->at<float>(L.coo_x),
+                                                     nnz, ptr, cur, ctx->at<int2>(L.csc_tmp));
+    count_launch();
+    csc_sort_kernel<<<grid1d(cols, 1, 148 * 16), 128, 0, s>>>(ctx->at<int2>(L.csc_tmp), ptr, cnt, cols,
+                                                              static_cast<int32_t>(ctx->K), ctx->at<int2>(L.csc_ent));
+    count_launch();
+  }
+  CKS(cudaGetLastError());
+  return SFB_OK;
+}
+
+// W <- prox(W - step * U^T V) with V in the column-major form built by sparse_build_csc.
+int sparse_update(sfb_ctx* ctx) {
+  const sfb_config& c = ctx->cfg;
+  const Layout& L = ctx->lay;
+  const bool bf16 = c.precision == SFB_PREC_BF16;
+  const int smem = slab_smem(ctx->K, bf16);
+  if (smem < 0) return SFB_ERR_SHAPE;
+  SuParams p{};
+  p.W = ctx->W; p.rows = c.rows; p.cols = c.cols;
+  p.ptr = ctx->at<int32_t>(L.csc_ptr);
+  p.ent = ctx->at<int2>(L.csc_ent);
+  p.K = static_cast<int32_t>(ctx->K);
+  p.alpha = -ctx->step;
+  p.prox_kind = ctx->prox_kind; p.prox_a = ctx->prox_a;
+  if (bf16) {
+    p.UT = ctx->at<__nv_bfloat16>(L.UT); p.ldut = L.Kp;
+    p.shadow = ctx->at<__nv_bfloat16>(L.Wb); p.shadow_ld = L.colsb;
+    p.copy_counters = &ctx->at<Scalars>(L.scalars)->copy_pieces;
+    CKS((launch_sparse_update<1, 1>(ctx->stream, p, smem)));
+  } else {
+    p.U = ctx->at<float>(L.U); p.ldu = c.rows;
+    if (ctx->tf32) {
+      p.shadow32 = ctx->at<float>(L.Ws); p.shadow32_ld = 2 * L.colsp; p.shadow_half = L.colsp;
+      CKS((launch_sparse_update<0, 2>(ctx->stream, p, smem)));
+    } else {
+      CKS((launch_sparse_update<0, 0>(ctx->stream, p, smem)));
+    }
+  }
+  return SFB_OK;
+}
+
+}  // namespace sfb

@@ -461,6 +461,7 @@ int tc_update_init(sfb_ctx* ctx, TcState* st) {
 // [cols x 2 Kp] with Kp the pair count rounded up to 32;  U^T V = Ub Vb + Ub Vs + Us Vb  (Us Vs, 2^-22 of the product,
 // is dropped).  The label entries are part of U here: no separate label-row pass, no bf16 copy of W.
 int tc32_update(sfb_ctx* ctx) {
+  if (ctx->sparse_v) return sparse_update(ctx);         // writes the (big | small) copy as well
   const sfb_config& c = ctx->cfg;
   const TcState* st = static_cast<const TcState*>(ctx->tc);
   const Layout& L = ctx->lay;
@@ -541,6 +542,10 @@ int tc_update(sfb_ctx* ctx) {
       label_rows_kernel<<<lgrid, 256, 0, ctx->stream>>>(
           ctx->W, c.rows, c.cols, ctx->at<float>(L.Xf), ctx->at<int32_t>(L.labels), ctx->at<float>(L.coef),
           static_cast<int>(ctx->K), ctx->step, ctx->at<__nv_bfloat16>(L.Wb), L.colsb);   // keeps the copy = bf16(W)
+    } else if (ctx->sparse_v) {
+      const int rc = sparse_update(ctx);                                                // the same sum over the non-zeros of V
+      if (rc) return rc;
+      continue;
     } else {
       update_pair_kernel<1><<<grid, kThreads, kSmem, ctx->stream>>>(ma, mb, mc, p);     // W += -eta * P^T V
     }

@@ -244,3 +244,52 @@ def ssp_delays(seed: int, clocks: int, workers: int, staleness: int) -> np.ndarr
     for p in range(workers):
         d[:, p, p] = 0
     return d
+
+
+# ----------------------------------------------------------------------------------------------------------
+# Sparse features (Section "Experiments": the paper's data sets have sparse features).  tf-idf-like samples in
+# compressed-sparse-row form: the number of non-zeros of a sample is Poisson around nnz_mean (at least 1), its columns
+# are drawn without replacement with Pr(column of popularity rank r) proportional to (r+1)^-zipf_s (the popularity
+# order is a seeded permutation of the columns), its values are log-normal and the sample is scaled to unit length.
+# ----------------------------------------------------------------------------------------------------------
+_S_SPARSE = 10
+
+
+@dataclass
+class SparseSamples:
+    indptr: np.ndarray     # int64 [n + 1]
+    indices: np.ndarray    # int32 [nnz], ascending within a sample
+    values: np.ndarray     # fp32 [nnz]
+
+    @property
+    def nnz(self) -> int:
+        return int(self.indptr[-1] - self.indptr[0])
+
+
+def sparse_samples(seed: int, step: int, n: int, cols: int, nnz_mean: float, zipf_s: float = 1.0) -> SparseSamples:
+    g = _gen(seed, _S_SPARSE, step)
+    order = _gen(seed, _S_SPARSE, 1 << 30).permutation(cols)
+    w = np.arange(1, cols + 1, dtype=np.float64) ** (-zipf_s)
+    prob = np.empty(cols, dtype=np.float64)
+    prob[order] = w / w.sum()
+    counts = np.clip(g.poisson(nnz_mean, size=n), 1, cols).astype(np.int64)
+    indptr = np.zeros(n + 1, dtype=np.int64)
+    np.cumsum(counts, out=indptr[1:])
+    indices = np.empty(int(indptr[-1]), dtype=np.int32)
+    values = np.empty(int(indptr[-1]), dtype=np.float32)
+    for i in range(n):
+        c = np.sort(g.choice(cols, size=int(counts[i]), replace=False, p=prob))
+        v = np.exp(0.5 * g.standard_normal(int(counts[i])))
+        v /= math.sqrt(float(np.dot(v, v)))
+        indices[indptr[i]:indptr[i + 1]] = c
+        values[indptr[i]:indptr[i + 1]] = v
+    return SparseSamples(indptr=indptr, indices=indices, values=values)
+
+
+def densify(sp: SparseSamples, cols: int) -> np.ndarray:
+    """The same samples as a dense fp32 [n x cols] array (zeros elsewhere)."""
+    n = len(sp.indptr) - 1
+    X = np.zeros((n, cols), dtype=np.float32)
+    rows = np.repeat(np.arange(n), np.diff(sp.indptr))
+    X[rows, sp.indices] = sp.values
+    return X
