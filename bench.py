@@ -463,6 +463,9 @@ def main():
     ap.add_argument("--phase", default="", choices=["", "update"],
                     help="update: after the timed steps, loop the fused update alone for --phase-seconds")
     ap.add_argument("--phase-seconds", type=float, default=2.0)
+    ap.add_argument("--sparse-nnz", type=float, default=0.0,
+                    help="MLR: samples in compressed-sparse-row form with about this many non-zeros each (tf-idf-like, "
+                         "Zipf column popularity); the update then sums only the non-zeros of each column")
     ap.add_argument("--shard", default="", choices=["", "rows"],
                     help="rows: partition W by rows over the ranks instead of running replicas")
     args = ap.parse_args()
@@ -509,8 +512,21 @@ def main():
     if full_forward_oracle:
         W_host = W.cpu().numpy()
     nb = 4
+    sparse = args.sparse_nnz > 0
+    if sparse and wl.model != I.MLR:
+        raise SystemExit("--sparse-nnz is for the MLR workloads")
     true_dict = I.sc_true_dictionary(wl) if wl.model == I.SC else None
     batches = [I.step_inputs(wl, rank * 1000 + t, true_dict) for t in range(nb)]
+    nnz_max = 0
+    if sparse:
+        # the same labels, the features replaced by sparse ones; the dense arrays are not used
+        sps = [I.sparse_samples(wl.seed, rank * 1000 + t, wl.K, wl.cols, args.sparse_nnz) for t in range(nb)]
+        nnz_max = max(sp.nnz for sp in sps)
+        hS = [(torch.from_numpy(sp.indptr).pin_memory(), torch.from_numpy(sp.indices).pin_memory(),
+               torch.from_numpy(sp.values).pin_memory(), sp.nnz) for sp in sps]
+        dS = [(a.to(dev), b.to(dev), c.to(dev), n) for a, b, c, n in hS]
+        for b in batches:
+            b.X = np.zeros((1, 4), dtype=np.float32)
     dX = [torch.from_numpy(b.X).to(dev) for b in batches]
     dY = [None if b.Y is None else torch.from_numpy(b.Y).to(dev) for b in batches]
     dL = [None if b.labels is None else torch.from_numpy(b.labels).to(dev) for b in batches]
@@ -520,7 +536,7 @@ def main():
 
     cfg = S.make_config(wl.model, wl.rows, wl.cols, wl.workers, wl.batch, wl.eta, prec, dml_margin=wl.dml_margin,
                         sc_lambda=wl.sc_lambda, sc_ista_iters=wl.sc_iters, sc_lipschitz=L,
-                        sc_prox=1 if wl.model == I.SC else 0)
+                        sc_prox=1 if wl.model == I.SC else 0, csr_nnz_max=nnz_max)
     ctx = S.Context(cfg, W)
     flusher = None
     if wl.rows * wl.cols * 4 <= 2 * 126e6:
@@ -537,7 +553,10 @@ def main():
             flusher.zero_()
         if ev is not None:
             ev[0].record()
-        ctx.sfb_compute_factors(-1, dX[k], dY[k], dL[k])
+        if sparse:
+            ctx.sfb_compute_factors_csr(-1, dS[k][0], dS[k][1], dS[k][2], dS[k][3], dL[k])
+        else:
+            ctx.sfb_compute_factors(-1, dX[k], dY[k], dL[k])
         if ev is not None:
             ev[1].record()
         ctx.sfb_gather_factors()
@@ -599,15 +618,25 @@ def main():
                        "roofline": update_roofline(wl, prec == S.PREC_BF16, ms_loop, peaks, ck,
                                                    tf32=runs_tf32(wl, args.precision))}
 
-    # ---- end to end: host minibatch -> sfb_step_host -> loss back on the host, every step
+    # ---- end to end: host minibatch -> sfb_step_host -> loss back on the host, every step (sparse samples: the three
+    # arrays and the labels copied from pinned memory, sfb_step_csr, the loss read back through sfb_get_stats)
+    def host_step(i):
+        k = i % nb
+        if not sparse:
+            return ctx.sfb_step_host(hX[k], hY[k], hL[k])[0]
+        ip, ix, vl, n = hS[k]
+        ctx.sfb_step_csr(ip.to(dev, non_blocking=True), ix.to(dev, non_blocking=True), vl.to(dev, non_blocking=True), n,
+                         hL[k].to(dev, non_blocking=True))
+        return ctx.sfb_get_stats().last_loss
+
     for i in range(3):
-        ctx.sfb_step_host(hX[i % nb], hY[i % nb], hL[i % nb])
+        host_step(i)
     barrier()
     e2e_steps = args.steps
     t0 = time.perf_counter()
     loss = 0.0
     for i in range(e2e_steps):
-        loss, _ = ctx.sfb_step_host(hX[i % nb], hY[i % nb], hL[i % nb])
+        loss = host_step(i)
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
 
@@ -621,13 +650,27 @@ def main():
     value = aggregate_value(world, K, args.steps, total_ms)
     e2e_value = aggregate_value(world, K, e2e_steps, e2e_ms)
     h2d = K * wl.in_dim * 4 + (K * wl.cols * 4 if wl.model == I.DML else 0) + (K * 4 if wl.model != I.SC else 0)
+    if sparse:
+        h2d = int(sum(8 * (K + 1) + 8 * n for _, _, _, n in hS) / nb) + K * 4
 
     # ---- roofline of the dominant kernel (the fused update), timed inside the long step: sustained tensor figure
     roof = update_roofline(wl, prec == S.PREC_BF16, ms_u, peaks, clocks, tf32=runs_tf32(wl, args.precision),
                            copy_fraction=min(1.0, copy_stats["rewritten_per_step"] / (wl.rows * math.ceil(wl.cols / 32)))
                            if copy_stats else 1.0)
+    if sparse:
+        # the sparse update is one read-modify-write pass over W plus the factors: bound by HBM
+        nnz = sum(n for _, _, _, n in hS) / nb
+        usz = 2 if prec == S.PREC_BF16 else 4
+        algo = 8.0 * wl.rows * wl.cols + usz * K * wl.rows + 8.0 * nnz
+        peak = peaks["hbm_gbs"]
+        roof = {"bound": "hbm", "achieved": algo / (ms_u * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
+                "frac": algo / (ms_u * 1e-3) / 1e9 / peak, "traffic": None, "peak_source": peaks["source"],
+                "kernel": "sparse_update_kernel (+ label_rows_kernel in bf16 mode)", "ms": ms_u,
+                "algorithmic_bytes": algo, "fma_per_entry_of_W": nnz / wl.cols,
+                "note": "W read and written once in fp32, the factors u read once, 8 bytes per non-zero of v; "
+                        "the operand copy of W is rewritten where its rounding changed (not counted)"}
     roof_fwd, roof_step = (None, None)
-    if prec == S.PREC_BF16 and wl.model == I.MLR:
+    if prec == S.PREC_BF16 and wl.model == I.MLR and not sparse:
         roof_fwd, roof_step = forward_and_step_rooflines(wl, ms_f, total_ms / args.steps, roof["roof_ms"], peaks)
 
     cpu = None
@@ -645,17 +688,22 @@ def main():
     if prec == S.PREC_BF16 and wl.model != I.MLR:
         esz = 4
     one_copy = K * (wl.rows + wl.cols) * esz
+    cfg_line = workload_config(wl, dtype_name(wl, args.precision))
+    if sparse:
+        one_copy = K * wl.rows * esz + 8 * sum(n for _, _, _, n in hS) / nb
+        cfg_line["features"] = (f"compressed sparse rows, about {args.sparse_nnz:g} non-zeros per sample "
+                                f"(Poisson), Zipf(1) column popularity, log-normal values, unit-length samples")
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": dtype_name(wl, args.precision),
-            "data": "synthetic", "config": workload_config(wl, dtype_name(wl, args.precision)),
+            "data": "synthetic", "config": cfg_line,
             "roofline": roof, "roofline_forward": roof_fwd, "roofline_step": roof_step, "cpu_baseline": cpu,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 8,
                     "ms_per_step": e2e_ms / e2e_steps, "last_loss": loss},
             "gpu_launches": int(launches), "clocks": clocks,
             "phases_ms": {"factors": ms_f, "gather": ms_g, "update": ms_u},
             "bytes": {"sf_gather_one_copy": one_copy,
-                      "sf_broadcast_p2p": wl.workers * (wl.workers - 1) * wl.batch * (wl.rows + wl.cols) * esz,
+                      "sf_broadcast_p2p": (wl.workers - 1) * one_copy,
                       "dense_sync": wl.workers * wl.rows * wl.cols * 4,
                       "dense_over_sf": wl.workers * wl.rows * wl.cols * 4 / one_copy},
             "operand_copy": copy_stats, "status_word": status}

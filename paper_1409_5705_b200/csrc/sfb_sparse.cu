@@ -21,7 +21,9 @@ namespace {
 constexpr unsigned kFull = 0xffffffffu;
 constexpr int kSuWarps = 16;                       // warps per block of the update kernel
 constexpr int kSuThreads = kSuWarps * 32;
-constexpr int kSuStage = 32 * 33;                  // floats of one warp's transpose buffer
+constexpr int kSuStage = 32 * 33;                  // floats of one warp's 32 x 32 buffer of sums
+constexpr int kSuChunk = 176;                      // entries (8 bytes each) of a column block staged at a time, per warp
+constexpr int kSuWarpBytes = kSuStage * 4 + kSuChunk * 8;
 constexpr int kSmemOptIn = 232448 - 1024;          // dynamic shared memory asked for: what a block may opt into, less the static part
 
 inline unsigned grid1d(int64_t n, int block, int cap = 148 * 16) {
@@ -160,12 +162,40 @@ struct SuParams {
   unsigned long long* copy_counters;
 };
 
+// Shared-memory reads of the inner loop through 32-bit shared-space addresses (one integer multiply-add per address).
+__device__ __forceinline__ uint32_t shared_addr(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ float lds_f32(uint32_t a) {
+  float v;
+  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint32_t lds_u16(uint32_t a) {
+  uint16_t v;
+  asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ void sts_f32(uint32_t a, float v) {
+  asm volatile("st.shared.f32 [%0], %1;" ::"r"(a), "f"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+__device__ __forceinline__ int4 lds_v4(uint32_t a) {
+  int4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+  return v;
+}
+
 template <int USRC>
 struct Slab {
   static constexpr int kPitch = USRC == 0 ? 33 * 4 : 34 * 2;      // bytes per sample: 32 rows, padded to an odd word count
-  static __device__ __forceinline__ float load(const uint8_t* us, int32_t i, int lane) {
-    if (USRC == 0) return *reinterpret_cast<const float*>(us + i * kPitch + lane * 4);
-    return __uint_as_float(static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(us + i * kPitch + lane * 2)) << 16);
+  // base: shared address of this lane's row in sample 0
+  static __device__ __forceinline__ float load(uint32_t base, int32_t i) {
+    if (USRC == 0) return lds_f32(base + i * kPitch);
+    return __uint_as_float(lds_u16(base + i * kPitch) << 16);
   }
 };
 
@@ -175,7 +205,7 @@ __device__ __forceinline__ float tf32_round(float x) {
   return __uint_as_float(u);
 }
 
-template <int USRC, int SHADOW>
+template <int USRC, int SHADOW, bool PROX>
 __global__ void __launch_bounds__(kSuThreads, 1) sparse_update_kernel(const SuParams p) {
   extern __shared__ __align__(16) uint8_t su_smem[];
   __shared__ int next_cb;
@@ -183,23 +213,32 @@ __global__ void __launch_bounds__(kSuThreads, 1) sparse_update_kernel(const SuPa
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   uint8_t* us = su_smem;
   const int slab_bytes = ((p.K + 1) * S::kPitch + 15) & ~15;
-  float* stg = reinterpret_cast<float*>(su_smem + slab_bytes) + warp * kSuStage;
+  float* stg = reinterpret_cast<float*>(su_smem + slab_bytes + warp * kSuWarpBytes);
+  int2* ebuf = reinterpret_cast<int2*>(stg + kSuStage);
+  const uint32_t ebuf_s = shared_addr(ebuf);
+  const uint32_t stg_s = shared_addr(stg) + lane * 4;                      // this lane's row of column 0 of the sums
+  const uint32_t us_s = shared_addr(us) + lane * (USRC == 0 ? 4 : 2);     // this lane's row of sample 0
   const int nrb = static_cast<int>((p.rows + 31) / 32), ncb = static_cast<int>((p.cols + 31) / 32);
+  // second role of a lane, for the pass over W: 8 lanes x 4 columns cover a row's 32 columns, 4 rows per step
+  const int sub = lane >> 3, jj = lane & 7;
   // sample K of the slab is all zero: the padding entries of odd columns point there
   for (int t = threadIdx.x; t < S::kPitch / 2; t += kSuThreads) reinterpret_cast<uint16_t*>(us + p.K * S::kPitch)[t] = 0;
   unsigned long long pieces = 0, written = 0;
 
   for (int rb = blockIdx.x; rb < nrb; rb += gridDim.x) {
     const int64_t r0 = static_cast<int64_t>(rb) * 32;
+    const int nrows = p.rows - r0 < 32 ? static_cast<int>(p.rows - r0) : 32;
     __syncthreads();                                   // every warp is done with the previous slab
     if (USRC == 0) {
-      const bool rv = r0 + lane < p.rows;
+      const bool rv = lane < nrows;
+#pragma unroll 8
       for (int i = warp; i < p.K; i += kSuWarps)
         *reinterpret_cast<float*>(us + i * S::kPitch + lane * 4) = rv ? p.U[static_cast<int64_t>(i) * p.ldu + r0 + lane] : 0.f;
     } else {
       for (int r = warp; r < 32; r += kSuWarps) {
-        const bool rv = r0 + r < p.rows;
+        const bool rv = r < nrows;
         const uint16_t* src = reinterpret_cast<const uint16_t*>(p.UT) + (r0 + r) * p.ldut;
+#pragma unroll 8
         for (int i = lane; i < p.K; i += 32)
           *reinterpret_cast<uint16_t*>(us + i * S::kPitch + r * 2) = rv ? src[i] : static_cast<uint16_t>(0);
       }
@@ -212,99 +251,141 @@ __global__ void __launch_bounds__(kSuThreads, 1) sparse_update_kernel(const SuPa
       if (lane == 0) cb = atomicAdd(&next_cb, 1);       // which warp takes which block does not change any result
       cb = __shfl_sync(kFull, cb, 0);
       if (cb >= ncb) break;
-      const int64_t d = static_cast<int64_t>(cb) * 32 + lane;
-      const bool dv = d < p.cols;
-      // as a column: the 32 rows of W at column d, asked for before the sums so that they arrive meanwhile
-      float wv[32];
+      // the block's 32 x 32 entries of W, asked for before the sums so that they arrive meanwhile
+      const int64_t dq = static_cast<int64_t>(cb) * 32 + 4 * jj;        // cols is a multiple of 4: a quad is in or out
+      const bool qv = dq < p.cols;
+      float4 wv[8];
 #pragma unroll
-      for (int r = 0; r < 32; ++r) wv[r] = (dv && r0 + r < p.rows) ? p.W[(r0 + r) * p.cols + d] : 0.f;
-      const int32_t pb = p.ptr[dv ? d : p.cols], pe = p.ptr[dv ? d + 1 : p.cols];
-      // as a row: sums over the entries of each of the 32 columns
-      float acc[32];
-#pragma unroll
-      for (int c = 0; c < 32; ++c) {
-        int32_t e = __shfl_sync(kFull, pb, c);
-        const int32_t e1 = __shfl_sync(kFull, pe, c);
-        float a = 0.f;
-        for (; e + 8 <= e1; e += 8) {
-          const int4 t0 = __ldg(reinterpret_cast<const int4*>(p.ent + e));
-          const int4 t1 = __ldg(reinterpret_cast<const int4*>(p.ent + e + 2));
-          const int4 t2 = __ldg(reinterpret_cast<const int4*>(p.ent + e + 4));
-          const int4 t3 = __ldg(reinterpret_cast<const int4*>(p.ent + e + 6));
-          const float u0 = S::load(us, t0.x, lane), u1 = S::load(us, t0.z, lane);
-          const float u2 = S::load(us, t1.x, lane), u3 = S::load(us, t1.z, lane);
-          const float u4 = S::load(us, t2.x, lane), u5 = S::load(us, t2.z, lane);
-          const float u6 = S::load(us, t3.x, lane), u7 = S::load(us, t3.z, lane);
-          a = fmaf(__int_as_float(t0.y), u0, a); a = fmaf(__int_as_float(t0.w), u1, a);
-          a = fmaf(__int_as_float(t1.y), u2, a); a = fmaf(__int_as_float(t1.w), u3, a);
-          a = fmaf(__int_as_float(t2.y), u4, a); a = fmaf(__int_as_float(t2.w), u5, a);
-          a = fmaf(__int_as_float(t3.y), u6, a); a = fmaf(__int_as_float(t3.w), u7, a);
-        }
-        for (; e < e1; e += 2) {
-          const int4 t0 = __ldg(reinterpret_cast<const int4*>(p.ent + e));
-          const float u0 = S::load(us, t0.x, lane), u1 = S::load(us, t0.z, lane);
-          a = fmaf(__int_as_float(t0.y), u0, a); a = fmaf(__int_as_float(t0.w), u1, a);
-        }
-        acc[c] = a;
+      for (int it = 0; it < 8; ++it) {
+        const int r = 4 * it + sub;
+        wv[it] = (qv && r < nrows) ? *reinterpret_cast<const float4*>(p.W + (r0 + r) * p.cols + dq)
+                                   : make_float4(0.f, 0.f, 0.f, 0.f);
       }
+      // first role of a lane: a ROW.  The sum over the entries of each of the 32 columns goes to the warp's 32 x 32
+      // buffer (column-major with an odd pitch: conflict-free both ways).  The entries of the block are contiguous
+      // (column after column); a window of kSuChunk of them is staged in a second small buffer and moved on when a
+      // column runs past its end (one trip to L2 per window).  The column loop is deliberately not unrolled: sixteen
+      // warps at sixteen places of a long unrolled body starve on instruction fetch.
+      const int64_t d = static_cast<int64_t>(cb) * 32 + lane;
+      const int32_t pb = p.ptr[d < p.cols ? d : p.cols], pe = p.ptr[d + 1 < p.cols ? d + 1 : p.cols];
+      const int32_t len = pe - pb;
+      const int32_t E1 = __shfl_sync(kFull, pe, 31);
+      int32_t b = __shfl_sync(kFull, pb, 0);                       // running entry index
+      int32_t wlo = 0, whi = 0;                                    // staged window of entries [wlo, whi)
+      uint32_t sacc = stg_s;
+#pragma unroll 1
+      for (int c = 0; c < 32; ++c, sacc += 33 * 4) {
+        int32_t left = __shfl_sync(kFull, len, c);
+        float a = 0.f;
+        while (left > 0) {
+          if (b >= whi) {
+            __syncwarp();                                          // every lane is done with the old window
+            wlo = b;
+            whi = b + kSuChunk < E1 ? b + kSuChunk : E1;
+            for (int32_t t = wlo + 2 * lane; t < whi; t += 64)
+              *reinterpret_cast<int4*>(ebuf + (t - wlo)) = __ldg(reinterpret_cast<const int4*>(p.ent + t));
+            __syncwarp();
+          }
+          int32_t n = left < whi - b ? left : whi - b;
+          uint32_t q = ebuf_s + static_cast<uint32_t>(b - wlo) * 8u;
+          b += n;
+          left -= n;
+          for (; n >= 8; n -= 8, q += 64) {
+            const int4 t0 = lds_v4(q), t1 = lds_v4(q + 16), t2 = lds_v4(q + 32), t3 = lds_v4(q + 48);
+            const float u0 = S::load(us_s, t0.x), u1 = S::load(us_s, t0.z);
+            const float u2 = S::load(us_s, t1.x), u3 = S::load(us_s, t1.z);
+            const float u4 = S::load(us_s, t2.x), u5 = S::load(us_s, t2.z);
+            const float u6 = S::load(us_s, t3.x), u7 = S::load(us_s, t3.z);
+            a = fmaf(__int_as_float(t0.y), u0, a); a = fmaf(__int_as_float(t0.w), u1, a);
+            a = fmaf(__int_as_float(t1.y), u2, a); a = fmaf(__int_as_float(t1.w), u3, a);
+            a = fmaf(__int_as_float(t2.y), u4, a); a = fmaf(__int_as_float(t2.w), u5, a);
+            a = fmaf(__int_as_float(t3.y), u6, a); a = fmaf(__int_as_float(t3.w), u7, a);
+          }
+          if (n >= 4) {
+            const int4 t0 = lds_v4(q), t1 = lds_v4(q + 16);
+            const float u0 = S::load(us_s, t0.x), u1 = S::load(us_s, t0.z);
+            const float u2 = S::load(us_s, t1.x), u3 = S::load(us_s, t1.z);
+            a = fmaf(__int_as_float(t0.y), u0, a); a = fmaf(__int_as_float(t0.w), u1, a);
+            a = fmaf(__int_as_float(t1.y), u2, a); a = fmaf(__int_as_float(t1.w), u3, a);
+            n -= 4; q += 32;
+          }
+          if (n >= 2) {
+            const int4 t0 = lds_v4(q);
+            const float u0 = S::load(us_s, t0.x), u1 = S::load(us_s, t0.z);
+            a = fmaf(__int_as_float(t0.y), u0, a); a = fmaf(__int_as_float(t0.w), u1, a);
+          }
+        }
+        sts_f32(sacc, a);
+      }
+      __syncwarp();                                    // all sums are in the buffer
+      // second role: the pass over W, 4 rows of 32 columns per step, every lane a quad of columns
+      if (SHADOW == 1 && lane == 0) pieces += nrows;
 #pragma unroll
-      for (int c = 0; c < 32; ++c) stg[c * 33 + lane] = acc[c];
-      __syncwarp();
-#pragma unroll
-      for (int r = 0; r < 32; ++r) {
-        const bool ok = dv && r0 + r < p.rows;
-        const float wo = wv[r];
-        const float wn = prox_entry(fmaf(p.alpha, stg[lane * 33 + r], wo), p.prox_kind, p.prox_a);
-        if (ok) p.W[(r0 + r) * p.cols + d] = wn;
+      for (int it = 0; it < 8; ++it) {
+        const int r = 4 * it + sub;
+        const bool ok = qv && r < nrows;
+        const float4 wo = wv[it];
+        const float* sp = stg + (4 * jj) * 33 + r;
+        float4 wn = make_float4(fmaf(p.alpha, sp[0], wo.x), fmaf(p.alpha, sp[33], wo.y), fmaf(p.alpha, sp[66], wo.z),
+                                fmaf(p.alpha, sp[99], wo.w));
+        if (PROX) {
+          wn.x = prox_entry(wn.x, p.prox_kind, p.prox_a); wn.y = prox_entry(wn.y, p.prox_kind, p.prox_a);
+          wn.z = prox_entry(wn.z, p.prox_kind, p.prox_a); wn.w = prox_entry(wn.w, p.prox_kind, p.prox_a);
+        }
+        if (ok) *reinterpret_cast<float4*>(p.W + (r0 + r) * p.cols + dq) = wn;
         if (SHADOW == 1) {
-          const __nv_bfloat16 bo = __float2bfloat16_rn(wo), bn = __float2bfloat16_rn(wn);
-          const bool differs = ok && __bfloat16_as_ushort(bo) != __bfloat16_as_ushort(bn);
-          const bool any = __any_sync(kFull, differs);
-          if (r0 + r < p.rows) {
-            ++pieces;
-            if (any) {
-              ++written;
-              if (ok) p.shadow[(r0 + r) * p.shadow_ld + d] = bn;
-            }
+          const uint32_t o01 = pack_bf16x2(wo.x, wo.y), o23 = pack_bf16x2(wo.z, wo.w);
+          const uint32_t n01 = pack_bf16x2(wn.x, wn.y), n23 = pack_bf16x2(wn.z, wn.w);
+          const unsigned bal = __ballot_sync(kFull, ok && (o01 != n01 || o23 != n23));
+          if ((bal >> (8 * sub)) & 0xffu) {             // this row's 64-byte piece changes: rewrite it
+            if (jj == 0) ++written;
+            if (ok) *reinterpret_cast<uint2*>(p.shadow + (r0 + r) * p.shadow_ld + dq) = make_uint2(n01, n23);
           }
         }
         if (SHADOW == 2 && ok) {
-          const float big = tf32_round(wn);
-          float* sp = p.shadow32 + (r0 + r) * p.shadow32_ld + d;
-          sp[0] = big;
-          sp[p.shadow_half] = tf32_round(wn - big);
+          const float4 big = make_float4(tf32_round(wn.x), tf32_round(wn.y), tf32_round(wn.z), tf32_round(wn.w));
+          float* s32 = p.shadow32 + (r0 + r) * p.shadow32_ld + dq;
+          *reinterpret_cast<float4*>(s32) = big;
+          *reinterpret_cast<float4*>(s32 + p.shadow_half) =
+              make_float4(tf32_round(wn.x - big.x), tf32_round(wn.y - big.y), tf32_round(wn.z - big.z), tf32_round(wn.w - big.w));
         }
       }
-      __syncwarp();                                    // the transpose buffer is free again
+      __syncwarp();                                    // the buffer of sums is free again
     }
   }
-  if (SHADOW == 1 && p.copy_counters && lane == 0) {
-    atomicAdd(p.copy_counters, pieces);
-    atomicAdd(p.copy_counters + 1, written);
+  if (SHADOW == 1 && p.copy_counters) {
+    if (lane == 0) atomicAdd(p.copy_counters, pieces);
+    if (jj == 0 && written) atomicAdd(p.copy_counters + 1, written);
   }
 }
 
-template <int USRC, int SHADOW>
-cudaError_t launch_sparse_update(cudaStream_t s, const SuParams& p, int smem) {
+template <int USRC, int SHADOW, bool PROX>
+cudaError_t launch_sparse_update_k(cudaStream_t s, const SuParams& p, int smem) {
   static std::atomic<uint64_t> prepared{0};            // one bit per device ordinal
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   const uint64_t bit = 1ull << (dev & 63);
   if (!(prepared.load(std::memory_order_acquire) & bit)) {
-    e = cudaFuncSetAttribute(sparse_update_kernel<USRC, SHADOW>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemOptIn);
+    e = cudaFuncSetAttribute(sparse_update_kernel<USRC, SHADOW, PROX>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemOptIn);
     if (e != cudaSuccess) return e;
     prepared.fetch_or(bit, std::memory_order_release);
   }
   const int nrb = static_cast<int>((p.rows + 31) / 32);
-  sparse_update_kernel<USRC, SHADOW><<<std::min(nrb, sm_count()), kSuThreads, smem, s>>>(p);
+  sparse_update_kernel<USRC, SHADOW, PROX><<<std::min(nrb, sm_count()), kSuThreads, smem, s>>>(p);
   count_launch();
   return cudaGetLastError();
 }
 
+template <int USRC, int SHADOW>
+cudaError_t launch_sparse_update(cudaStream_t s, const SuParams& p, int smem) {
+  return p.prox_kind != 0 ? launch_sparse_update_k<USRC, SHADOW, true>(s, p, smem)
+                          : launch_sparse_update_k<USRC, SHADOW, false>(s, p, smem);
+}
+
 int slab_smem(int64_t K, bool bf16) {
   const int64_t pitch = bf16 ? 34 * 2 : 33 * 4;
-  const int64_t bytes = (((K + 1) * pitch + 15) & ~int64_t(15)) + static_cast<int64_t>(kSuWarps) * kSuStage * 4;
+  const int64_t bytes = (((K + 1) * pitch + 15) & ~int64_t(15)) + static_cast<int64_t>(kSuWarps) * kSuWarpBytes;
   return bytes <= kSmemOptIn ? static_cast<int>(bytes) : -1;
 }
 
