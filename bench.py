@@ -466,6 +466,8 @@ def main():
     ap.add_argument("--sparse-nnz", type=float, default=0.0,
                     help="MLR: samples in compressed-sparse-row form with about this many non-zeros each (tf-idf-like, "
                          "Zipf column popularity); the update then sums only the non-zeros of each column")
+    ap.add_argument("--sparse-update", default="auto", choices=["auto", "sparse", "dense"],
+                    help="with --sparse-nnz: which update the step takes (auto: the library's cost model)")
     ap.add_argument("--shard", default="", choices=["", "rows"],
                     help="rows: partition W by rows over the ranks instead of running replicas")
     args = ap.parse_args()
@@ -536,7 +538,8 @@ def main():
 
     cfg = S.make_config(wl.model, wl.rows, wl.cols, wl.workers, wl.batch, wl.eta, prec, dml_margin=wl.dml_margin,
                         sc_lambda=wl.sc_lambda, sc_ista_iters=wl.sc_iters, sc_lipschitz=L,
-                        sc_prox=1 if wl.model == I.SC else 0, csr_nnz_max=nnz_max)
+                        sc_prox=1 if wl.model == I.SC else 0, csr_nnz_max=nnz_max,
+                        csr_update={"auto": 0, "sparse": 1, "dense": 2}[args.sparse_update])
     ctx = S.Context(cfg, W)
     flusher = None
     if wl.rows * wl.cols * 4 <= 2 * 126e6:
@@ -657,7 +660,8 @@ def main():
     roof = update_roofline(wl, prec == S.PREC_BF16, ms_u, peaks, clocks, tf32=runs_tf32(wl, args.precision),
                            copy_fraction=min(1.0, copy_stats["rewritten_per_step"] / (wl.rows * math.ceil(wl.cols / 32)))
                            if copy_stats else 1.0)
-    if sparse:
+    sparse_ran = sparse and st1.sparse_updates > st0.sparse_updates
+    if sparse_ran:
         # the sparse update is one read-modify-write pass over W plus the factors: bound by HBM
         nnz = sum(n for _, _, _, n in hS) / nb
         usz = 2 if prec == S.PREC_BF16 else 4
@@ -693,6 +697,7 @@ def main():
         one_copy = K * wl.rows * esz + 8 * sum(n for _, _, _, n in hS) / nb
         cfg_line["features"] = (f"compressed sparse rows, about {args.sparse_nnz:g} non-zeros per sample "
                                 f"(Poisson), Zipf(1) column popularity, log-normal values, unit-length samples")
+        cfg_line["update"] = ("sparse" if sparse_ran else "dense") + f" ({args.sparse_update})"
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": dtype_name(wl, args.precision),

@@ -95,6 +95,9 @@ typedef struct sfb_config {
   float   prox_weight;    /* the weight w of that regulariser (>= 0)                                  */
   int64_t csr_nnz_max;    /* MLR: room, in non-zeros per step over all K samples, for samples given in
                              compressed-sparse-row form (sfb_compute_factors_csr); 0: none                */
+  int32_t csr_update;     /* which update a step of sparse samples takes: 0 the cheaper one by the library's
+                             cost model (non-zeros per column against K) | 1 the sparse one whenever its
+                             factor slab fits | 2 always the dense one                                    */
   void*   stream;         /* cudaStream_t                                                              */
 } sfb_config;
 
@@ -113,6 +116,7 @@ typedef struct sfb_stats {
                                  passes went over since sfb_init, and                                          */
   int64_t copy_written;       /* how many of them they rewrote (a piece whose 32 bf16 roundings did not change
                                  already holds bf16 of the new values and is left alone)                      */
+  int64_t sparse_updates;     /* steps whose update summed only the non-zeros of sparse samples                */
 } sfb_stats;
 
 /* Bytes of device workspace a context with this config needs.  Host-only; no CUDA call. */
@@ -159,7 +163,10 @@ int sfb_compute_factors(sfb_ctx* ctx, int32_t worker, const float* X_dev, const 
  *     W[j][d] <- prox( W[j][d] - eta * sum_{i : x_id != 0} u_ij x_id ),
  * one pass over W as in the dense update, the derived operand copies of W rewritten with it.  sfb_stats.gather_bytes
  * then counts K*rows*element size for the u and 8 bytes per non-zero for the v.  A mini-batch too large for the
- * kernel's on-chip factor slab (K above about 1200 in the fp32 modes, 2400 in bf16 mode) takes the dense update. */
+ * kernel's on-chip factor slab (K above about 1200 in the fp32 modes, 2400 in bf16 mode) takes the dense update, and
+ * so does, unless cfg.csr_update says otherwise, one whose columns hold so many non-zeros that the tensor-core update
+ * over the scattered samples is the faster of the two (in bf16 mode from about 2 non-zeros per column at K = 1024; in
+ * the fp32 modes from about 30). */
 int sfb_compute_factors_csr(sfb_ctx* ctx, int32_t worker, const int64_t* indptr_dev, const int32_t* indices_dev,
                             const float* values_dev, int64_t nnz, const int32_t* labels_dev);
 

@@ -14,6 +14,7 @@ from .build import LIB, build
 MLR, DML, SC, L2MLR = 0, 1, 2, 3
 PREC_BF16, PREC_FP32, PREC_TF32X3, PREC_FP32_FFMA = 0, 1, 2, 3
 PROX_NONE, PROX_L1, PROX_L2SQ = 0, 1, 2
+CSR_UPDATE_AUTO, CSR_UPDATE_SPARSE, CSR_UPDATE_DENSE = 0, 1, 2
 STATUS_LABEL_RANGE, STATUS_TIMEOUT, STATUS_SAMPLE_RANGE, STATUS_INDEX_RANGE = 0x1, 0x2, 0x4, 0x8
 
 EXPORTS = ("sfb_workspace_bytes", "sfb_init", "sfb_compute_factors", "sfb_gather_factors", "sfb_apply_update",
@@ -32,7 +33,7 @@ class sfb_config(ctypes.Structure):
                 ("eta", ctypes.c_float), ("dml_margin", ctypes.c_float), ("sc_lambda", ctypes.c_float),
                 ("sc_ista_iters", ctypes.c_int32), ("sc_lipschitz", ctypes.c_float), ("sc_prox", ctypes.c_int32),
                 ("sdca_lambda", ctypes.c_float), ("sdca_n", ctypes.c_int64), ("prox_kind", ctypes.c_int32),
-                ("prox_weight", ctypes.c_float), ("csr_nnz_max", ctypes.c_int64), ("stream", ctypes.c_void_p)]
+                ("prox_weight", ctypes.c_float), ("csr_nnz_max", ctypes.c_int64), ("csr_update", ctypes.c_int32), ("stream", ctypes.c_void_p)]
 
 
 class sfb_stats(ctypes.Structure):
@@ -41,7 +42,7 @@ class sfb_stats(ctypes.Structure):
                 ("dense_sync_bytes", ctypes.c_double), ("ms_factors", ctypes.c_float),
                 ("ms_gather", ctypes.c_float), ("ms_update", ctypes.c_float), ("last_loss", ctypes.c_float),
                 ("sc_lipschitz", ctypes.c_float), ("kernel_launches", ctypes.c_int64),
-                ("copy_pieces", ctypes.c_int64), ("copy_written", ctypes.c_int64)]
+                ("copy_pieces", ctypes.c_int64), ("copy_written", ctypes.c_int64), ("sparse_updates", ctypes.c_int64)]
 
 
 class SfbError(RuntimeError):
@@ -108,9 +109,9 @@ def strerror(code: int) -> str:
 
 def make_config(model, rows, cols, workers, batch, eta, precision=PREC_FP32, dml_margin=1.0, sc_lambda=0.1,
                 sc_ista_iters=20, sc_lipschitz=0.0, sc_prox=0, stream=0, sdca_lambda=0.0, sdca_n=0, prox_kind=0,
-                prox_weight=0.0, csr_nnz_max=0) -> sfb_config:
+                prox_weight=0.0, csr_nnz_max=0, csr_update=0) -> sfb_config:
     return sfb_config(model, precision, rows, cols, workers, batch, eta, dml_margin, sc_lambda, sc_ista_iters,
-                      sc_lipschitz, sc_prox, sdca_lambda, sdca_n, prox_kind, prox_weight, csr_nnz_max, stream)
+                      sc_lipschitz, sc_prox, sdca_lambda, sdca_n, prox_kind, prox_weight, csr_nnz_max, csr_update, stream)
 
 
 def sfb_workspace_bytes(cfg: sfb_config) -> int:

@@ -90,6 +90,7 @@ static int check_config(const sfb_config* c) {
   if (c->prox_kind < 0 || c->prox_kind > 2 || !(c->prox_weight >= 0.f)) return SFB_ERR_ARG;
   if (c->model == SFB_L2MLR && c->prox_kind != 0) return SFB_ERR_UNSUPPORTED;
   if (c->csr_nnz_max < 0 || c->csr_nnz_max + c->cols > (1LL << 31) - 64) return SFB_ERR_SHAPE;
+  if (c->csr_update < 0 || c->csr_update > 2) return SFB_ERR_ARG;
   return SFB_OK;
 }
 
@@ -428,7 +429,7 @@ extern "C" int sfb_gather_factors(sfb_ctx* ctx) {
   // Every worker wrote its pairs at row offset p*B of the shared buffers, so the gathered operands are
   // complete; what remains is the per-step read-out over all K pairs.
   // all K samples sparse: the v become their column-major form (and the dense update operands are not needed)
-  ctx->sparse_v = c.model == SFB_MLR && c.csr_nnz_max > 0 && ctx->sparse_mask == all && sparse_update_fits(ctx);
+  ctx->sparse_v = c.model == SFB_MLR && c.csr_nnz_max > 0 && ctx->sparse_mask == all && sparse_update_wanted(ctx);
   if (ctx->sparse_v) {
     int rc = sparse_build_csc(ctx);
     if (rc) return rc;
@@ -473,6 +474,7 @@ extern "C" int sfb_apply_update(sfb_ctx* ctx) {
   ctx->gathered = false;
   ctx->stats.steps += 1;
   ctx->stats.samples += ctx->K;
+  if (ctx->sparse_v) ctx->stats.sparse_updates += 1;
   return SFB_OK;
 }
 

@@ -159,7 +159,9 @@ cudaError_t prox_entries(cudaStream_t s, float* w, int64_t n, int kind, float a)
 // Sparse sufficient factors (MLR): staging of compressed-sparse-row samples, their column-major form, the update
 // ---------------------------------------------------------------------------------------------------------
 void sparse_extend_layout(const sfb_config& c, Layout& L, size_t& off);
-bool sparse_update_fits(const sfb_ctx* ctx);          // the factor slab of K samples fits the shared memory of a block
+// The step's sparse samples take the sparse update: its factor slab of K samples fits the shared memory of a block and,
+// unless the config forces either, the cost model prefers it to the tensor-core update over the scattered samples.
+bool sparse_update_wanted(const sfb_ctx* ctx);
 int sparse_stage(sfb_ctx* ctx, int64_t off, int64_t n, const int64_t* indptr, const int32_t* idx, const float* val,
                  int64_t nnz);
 int sparse_build_csc(sfb_ctx* ctx);

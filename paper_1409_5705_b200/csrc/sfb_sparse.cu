@@ -413,8 +413,19 @@ void sparse_extend_layout(const sfb_config& c, Layout& L, size_t& off) {
   L.csc_ent = take((nnz + cols + 8) * 8);
 }
 
-bool sparse_update_fits(const sfb_ctx* ctx) {
-  return slab_smem(ctx->K, ctx->cfg.precision == SFB_PREC_BF16) > 0;
+// Cost model, in time per entry of W relative to the dense update of K = 1024 pairs in bf16 (measured at 325,000 x
+// 10,000 on one B200: 8.5 ms): the sparse update costs a fixed 0.83 for its pass over W (1.57 in the tensor-core fp32
+// mode, whose 8-byte operand copy it also writes) plus 0.089 per non-zero of an average column; the dense update
+// costs K/1024 in bf16 mode, 4.4 K/1024 with tf32 pairs, and far more on the FMA kernels.
+bool sparse_update_wanted(const sfb_ctx* ctx) {
+  const sfb_config& c = ctx->cfg;
+  const bool bf16 = c.precision == SFB_PREC_BF16;
+  if (c.csr_update == 2 || slab_smem(ctx->K, bf16) < 0) return false;
+  if (c.csr_update == 1 || (!bf16 && !ctx->tf32)) return true;
+  const double per_col = static_cast<double>(ctx->csr_fill) / static_cast<double>(c.cols);
+  const double k = static_cast<double>(ctx->K) / 1024.0;
+  const double sparse = (bf16 ? 0.83 : 1.57) + 0.089 * per_col;
+  return sparse < (bf16 ? 1.0 : 4.4) * k;
 }
 
 int sparse_stage(sfb_ctx* ctx, int64_t off, int64_t n, const int64_t* indptr, const int32_t* idx, const float* val,

@@ -29,6 +29,7 @@ def _inputs(wl, step, nnz_mean):
 
 
 def _config(wl, prec, nnz_max, **kw):
+    kw.setdefault("csr_update", S.CSR_UPDATE_SPARSE)        # these shapes are small: the cost model would go dense
     return S.make_config(wl.model, wl.rows, wl.cols, wl.workers, wl.batch, wl.eta, prec, csr_nnz_max=nnz_max, **kw)
 
 
