@@ -141,3 +141,52 @@ def test_mlr_large_sampled_rows(prec):
     assert entries_ok(Wg[last], ref[last], W0r[last], TOL[prec])
     zy = np.einsum("kd,kd->k", inp.X.astype(np.float64), W0[inp.labels].astype(np.float64))
     assert abs(loss - float((lse - zy).mean())) < 1e-3
+
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_mlr_large_sparse_samples_sampled_rows(prec):
+    """The paper-scale shape with sparse samples (about 100 non-zeros each) through the sparse update, against the
+    oracle on the same samples written out densely."""
+    wl = I.WORKLOADS["mlr_large"]
+    W0 = I.initial_W(wl, threads=16)
+    labels = I.step_inputs(wl, 0).labels
+    sp = I.sparse_samples(wl.seed, 0, wl.K, wl.cols, 100.0)
+    X = I.densify(sp, wl.cols)
+    W = torch.empty((wl.rows, wl.cols), dtype=torch.float32, device="cuda")
+    chunk = 32768
+    for r0 in range(0, wl.rows, chunk):
+        W[r0:r0 + chunk].copy_(torch.from_numpy(W0[r0:r0 + chunk]))
+    cfg = S.make_config(wl.model, wl.rows, wl.cols, wl.workers, wl.batch, wl.eta, prec, csr_nnz_max=sp.nnz,
+                        csr_update=S.CSR_UPDATE_SPARSE)
+    ctx = S.Context(cfg, W)
+    ctx.sfb_step_csr(to_dev(sp.indptr, torch), to_dev(sp.indices, torch), to_dev(sp.values, torch), sp.nnz,
+                     to_dev(labels, torch))
+    assert ctx.sfb_get_status() == 0
+    st = ctx.sfb_get_stats()
+    assert st.sparse_updates == 1
+    rng = np.random.default_rng(11)
+    label_rows = np.unique(labels)
+    rows = np.unique(np.concatenate([label_rows, rng.integers(0, wl.rows, 4096), np.arange(wl.rows - 136, wl.rows)]))
+    Wg = W[torch.from_numpy(rows).cuda()].cpu().numpy()
+    if prec == S.PREC_BF16:                      # the operand copy follows the sparse update exactly
+        copy = ctx.operand_copy_as_tensor()
+        sel = torch.from_numpy(rows[::16]).cuda()
+        assert torch.equal(copy[sel][:, :wl.cols].float(), W[sel].to(torch.bfloat16).float())
+    ctx.close()
+    del W
+    torch.cuda.empty_cache()
+    lse = O.mlr_log_partition(W0, X)
+    ref = O.mlr_updated_rows(W0[rows], rows, X, labels, lse, wl.eta)
+    W0r = W0[rows]
+    err = rel_err(Wg, ref, W0r)
+    print(f"mlr_large sparse: rel err on {len(rows)} rows {err:.3e} (tol {TOL[prec]})")
+    assert err <= TOL[prec]
+    # entry-wise, the bound following the entry's own update (updates of sparse samples span orders of magnitude)
+    upd = np.abs(ref - W0r)
+    rms = float(np.sqrt((upd * upd).mean()))
+    half_ulp = 0.5 * np.spacing(np.abs(ref).astype(np.float32)).astype(np.float64)
+    is_label = np.isin(rows, label_rows)
+    ok = np.abs(Wg.astype(np.float64) - ref) - half_ulp <= 8 * TOL[prec] * (upd + rms)
+    assert ok[~is_label].all()
+    assert abs(st.last_loss - float((lse - np.einsum("kd,kd->k", X.astype(np.float64),
+                                                      W0[labels].astype(np.float64))).mean())) < 1e-3
