@@ -340,6 +340,8 @@ extern "C" int sfb_forward_partials(sfb_ctx* ctx, const float* X_dev, const int3
   if (!al16(partials_dev)) return SFB_ERR_ALIGN;
   const sfb_config& c = ctx->cfg;
   ctx->committed = 0;
+  ctx->sparse_mask = 0;
+  ctx->csr_fill = 0;
   ctx->gathered = false;
   CK(cudaEventRecord(ctx->ev[0], ctx->stream));
   if (c.precision == SFB_PREC_BF16 || ctx->tf32) {
@@ -404,6 +406,7 @@ extern "C" int sfb_set_factors(sfb_ctx* ctx, int32_t worker, const float* U_dev,
                        static_cast<size_t>(c.batch), cudaMemcpyDeviceToDevice, ctx->stream));
   CK(cudaMemcpyAsync(V, V_dev, static_cast<size_t>(c.batch) * c.cols * 4, cudaMemcpyDeviceToDevice, ctx->stream));
   ctx->committed |= 1ull << worker;
+  ctx->sparse_mask &= ~(1ull << worker);             // received factors are dense
   ctx->gathered = false;
   return SFB_OK;
 }
@@ -471,6 +474,8 @@ extern "C" int sfb_apply_update(sfb_ctx* ctx) {
   if (rc) return rc;
   CK(cudaEventRecord(ctx->ev[3], ctx->stream));
   ctx->committed = 0;
+  ctx->sparse_mask = 0;               // the next step starts with no sparse samples staged
+  ctx->csr_fill = 0;
   ctx->gathered = false;
   ctx->stats.steps += 1;
   ctx->stats.samples += ctx->K;

@@ -179,3 +179,30 @@ def test_bad_indices_are_flagged_and_skipped_and_limits_are_errors():
         ctx.sfb_step_csr(*_dev(sp, labels)[:3], sp.nnz, to_dev(labels, torch))
     assert e.value.code == -10
     ctx.close()
+
+
+@pytest.mark.parametrize("prec", [pytest.param(S.PREC_TF32X3, id="tf32x3"), pytest.param(S.PREC_BF16, id="bf16")])
+def test_sparse_and_dense_steps_alternate_on_one_context(prec):
+    """sparse, dense, sparse on the same context: no state of a sparse step leaks into the next step, and the operand
+    copy of W that the forward products read stays current through both kinds of update."""
+    wl = WL_TILES
+    W0 = I.initial_W(wl)
+    W = to_dev(W0, torch)
+    ctx = S.Context(_config(wl, prec, 30 * wl.K), W)
+    start = W0.astype(np.float64)
+    for step, kind in enumerate(["sparse", "dense", "sparse"]):
+        sp, labels = _inputs(wl, step, 10.0)
+        X = I.densify(sp, wl.cols)
+        if kind == "sparse":
+            ctx.sfb_step_csr(*_dev(sp, labels)[:3], sp.nnz, to_dev(labels, torch))
+        else:
+            ctx.sfb_step(to_dev(X, torch), None, to_dev(labels, torch))
+        assert ctx.sfb_get_status() == 0
+        Wg = W.cpu().numpy()
+        ref = O.sfb_step(I.MLR, start, X, None, labels, workers=wl.workers, eta=wl.eta)
+        err = rel_err(Wg, ref, start)
+        print(f"{kind} step {step}: err {err:.3e}")
+        assert err <= TOL[prec]
+        start = Wg.astype(np.float64)
+    assert ctx.sfb_get_stats().sparse_updates == 2
+    ctx.close()
