@@ -183,7 +183,7 @@ extern "C" int sfb_destroy(sfb_ctx* ctx) {
 // fp32-operand path
 // ---------------------------------------------------------------------------------------------------------
 static int factors_fp32(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float* Y,
-                        const int32_t* labels) {
+                        const int32_t* labels, bool sparse_fwd = false) {
   const sfb_config& c = ctx->cfg;
   const int64_t rows = c.rows, cols = c.cols;
   float* V = ctx->at<float>(ctx->lay.V) + off * cols;
@@ -195,8 +195,13 @@ static int factors_fp32(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, co
   if (c.model == SFB_MLR || c.model == SFB_DML) {
     CK(pack_copy(s, V, X, c.model == SFB_DML ? Y : nullptr, n * cols));                 // v = x | x - y
     e.C = U; e.ldc = rows;
-    CK(sgemm(s, true, true, EPI_STORE, n, rows, cols, V, cols, ctx->W, cols, e));       // z_i = W v_i
-    ctx->stats.flops += 2.0 * n * rows * cols;
+    if (sparse_fwd) {                                                                   // z_i = W v_i over the non-zeros of v_i
+      const int rc = sparse_forward(ctx, off, n, ctx->at<float>(ctx->lay.U), rows);
+      if (rc) return rc;
+    } else {
+      CK(sgemm(s, true, true, EPI_STORE, n, rows, cols, V, cols, ctx->W, cols, e));     // z_i = W v_i
+      ctx->stats.flops += 2.0 * n * rows * cols;
+    }
     if (c.model == SFB_MLR)
       CK(mlr_softmax_rows(s, U, n, rows, labels, ctx->at<float>(ctx->lay.loss) + off, status));
     else
@@ -298,7 +303,7 @@ extern "C" int sfb_compute_factors_csr(sfb_ctx* ctx, int32_t worker, const int64
   if (rc) return rc;
   const float* X = ctx->at<float>(ctx->lay.stageX) + off * c.cols;
   rc = ctx->tf32 ? tc32_factors(ctx, off, n, X, labels_dev, nullptr, 0.f)
-       : c.precision == SFB_PREC_FP32 ? factors_fp32(ctx, off, n, X, nullptr, labels_dev)
+       : c.precision == SFB_PREC_FP32 ? factors_fp32(ctx, off, n, X, nullptr, labels_dev, sparse_forward_rows(ctx, n) > 0)
                                       : tc_factors(ctx, off, n, X, nullptr, labels_dev);
   if (rc) return rc;
   ctx->csr_fill += nnz;

@@ -31,7 +31,7 @@ struct Layout {
   size_t Ws, WTs, As, Rs;             // W by rows, W transposed, the A operand (v or the codes), the residual
   size_t U2;                          // DML: second partial of z when the forward product splits its contraction
   // sparse factors (MLR, csr_nnz_max > 0): the step's (sample, column, value) triples and their column-major form
-  size_t coo_i, coo_c, coo_x, csc_cnt, csc_cur, csc_ptr, csc_tmp, csc_ent;
+  size_t coo_i, coo_c, coo_x, coo_cx, row_beg, row_end, csc_cnt, csc_cur, csc_ptr, csc_tmp, csc_ent;
   int64_t ldu;                        // row pitch of the fp32 U buffer (rows rounded up to 4 in bf16 mode)
   int64_t colsp, rowsp;               // cols, rows rounded up to 64
   int64_t Kp;                         // K rounded up to the contraction block of the update product
@@ -83,6 +83,7 @@ struct sfb_ctx {
   uint64_t committed;                 // bit p set: worker p has written its factors since the last update
   uint64_t sparse_mask;               // bit p set: worker p's samples of this step came in compressed-sparse-row form
   int64_t csr_fill;                   // triples staged so far in this step
+  int64_t last_stage_nnz;             // entries of the last staged block of samples
   bool sparse_v;                      // the gathered v are in column-major sparse form: the update sums only the non-zeros
   bool gathered;
   int last_cuda;
@@ -164,6 +165,9 @@ void sparse_extend_layout(const sfb_config& c, Layout& L, size_t& off);
 bool sparse_update_wanted(const sfb_ctx* ctx);
 int sparse_stage(sfb_ctx* ctx, int64_t off, int64_t n, const int64_t* indptr, const int32_t* idx, const float* val,
                  int64_t nnz);
+// fp32 FMA mode: rows of W per block of the row-wise forward over sparse samples (0: the rows do not fit), and that product
+int sparse_forward_rows(const sfb_ctx* ctx, int64_t n);
+int sparse_forward(sfb_ctx* ctx, int64_t off, int64_t n, float* Z, int64_t ldz);
 int sparse_build_csc(sfb_ctx* ctx);
 int sparse_update(sfb_ctx* ctx);
 

@@ -30,6 +30,33 @@ inline unsigned grid1d(int64_t n, int block, int cap = 148 * 16) {
   return static_cast<unsigned>(std::max<int64_t>(1, std::min<int64_t>((n + block - 1) / block, cap)));
 }
 
+// Shared-memory reads of the inner loop through 32-bit shared-space addresses (one integer multiply-add per address).
+__device__ __forceinline__ uint32_t shared_addr(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ float lds_f32(uint32_t a) {
+  float v;
+  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint32_t lds_u16(uint32_t a) {
+  uint16_t v;
+  asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ void sts_f32(uint32_t a, float v) {
+  asm volatile("st.shared.f32 [%0], %1;" ::"r"(a), "f"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+__device__ __forceinline__ int4 lds_v4(uint32_t a) {
+  int4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+  return v;
+}
+
 // ---------------------------------------------------------------------------------------------------------
 // Staging of a worker's CSR block: the dense fp32 samples for the forward product, and (sample, column, value)
 // triples appended to the step's list for the column-major form.  One warp per sample.
@@ -38,23 +65,33 @@ __global__ void __launch_bounds__(256) csr_stage_kernel(const int64_t* __restric
                                                         const float* __restrict__ val, int64_t n, int64_t nnz, int64_t cols,
                                                         int64_t off, float* __restrict__ Xd, int32_t* __restrict__ coo_i,
                                                         int32_t* __restrict__ coo_c, float* __restrict__ coo_x,
-                                                        uint32_t* __restrict__ status) {
+                                                        int2* __restrict__ coo_cx, int32_t fill, int32_t* __restrict__ row_beg,
+                                                        int32_t* __restrict__ row_end, uint32_t* __restrict__ status) {
   const int64_t i = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (i >= n) return;
   const int64_t base = indptr[0];
   const int64_t b = indptr[i] - base, e = indptr[i + 1] - base;
   if (b < 0 || e < b || e > nnz) {                 // row pointers that do not describe nnz entries: sample left empty
-    if (lane == 0) atomicOr(status, SFB_STATUS_INDEX_RANGE);
+    if (lane == 0) {
+      atomicOr(status, SFB_STATUS_INDEX_RANGE);
+      row_beg[off + i] = row_end[off + i] = fill;
+    }
     return;
+  }
+  if (lane == 0) {                                 // the sample's range in the step's list (for the row-wise forward)
+    row_beg[off + i] = fill + static_cast<int32_t>(b);
+    row_end[off + i] = fill + static_cast<int32_t>(e);
   }
   for (int64_t t = b + lane; t < e; t += 32) {
     const int32_t c = idx[base + t];
     const float x = val[base + t];
     if (c < 0 || c >= cols) {                      // entry skipped (its slot keeps the "no entry" mark)
       atomicOr(status, SFB_STATUS_INDEX_RANGE);
+      coo_cx[t] = make_int2(0, 0);                 // value 0 at column 0: adds nothing to a logit
       continue;
     }
+    coo_cx[t] = make_int2(c, __float_as_int(x));
     Xd[(off + i) * cols + c] = x;
     coo_i[t] = static_cast<int32_t>(off + i);
     coo_c[t] = c;
@@ -132,6 +169,118 @@ __global__ void __launch_bounds__(128) csc_sort_kernel(const int2* __restrict__ 
 }
 
 // ---------------------------------------------------------------------------------------------------------
+// Row-wise forward product for sparse samples in the fp32 FMA mode:  z_ij = sum_t x_it W[j][c_it]  (Section 2.1: the
+// logits W a_i), the sparse counterpart of the FFMA product (the tensor-core modes keep their dense product over the
+// scattered samples, which is faster than any gather).  A block holds RB whole rows of W in shared memory; a warp takes
+// one sample at a time with its lanes as RB rows x 32/RB entries: each lane multiplies every (32/RB)-th entry of the
+// sample with its row's value at that column, the partial sums of a row are added by shuffles.  The entries of a
+// sample come through a small per-warp buffer in shared memory, filled by asynchronous copies two samples ahead.  Sums
+// are in a fixed order.
+// ---------------------------------------------------------------------------------------------------------
+constexpr int kSfWarps = 16;
+constexpr int kSfThreads = kSfWarps * 32;
+constexpr int kSfChunk = 128;                        // entries of a sample staged at once (a warp's buffer: 1 KB)
+constexpr int kSfBufs = 3;                           // the samples one and two ahead are in flight
+
+__device__ __forceinline__ void cp_async_8(uint32_t dst, const void* src, bool valid) {
+  const uint32_t n = valid ? 8u : 0u;                // 0: nothing is read, the 8 bytes are filled with zeros
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ int2 lds_v2(uint32_t a) {
+  int2 v;
+  asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
+  return v;
+}
+
+// The first kSfChunk entries [b, e) of a sample into a warp's buffer, zeros after the last one.
+__device__ __forceinline__ void stage_entries(uint32_t buf, const int2* __restrict__ cx, int32_t b, int32_t e, int lane) {
+#pragma unroll
+  for (int k = 0; k < kSfChunk / 32; ++k) {
+    const int32_t t = b + k * 32 + lane;
+    cp_async_8(buf + static_cast<uint32_t>(k * 32 + lane) * 8u, cx + (t < e ? t : b), t < e);
+  }
+  cp_async_commit();
+}
+
+template <int RB>
+__global__ void __launch_bounds__(kSfThreads, 1) sparse_forward_kernel(const float* __restrict__ W, int64_t rows, int64_t cols,
+                                                                       int32_t pitch, const int32_t* __restrict__ row_beg,
+                                                                       const int32_t* __restrict__ row_end,
+                                                                       const int2* __restrict__ cx, int64_t off, int32_t n,
+                                                                       float* __restrict__ Z, int64_t ldz) {
+  extern __shared__ __align__(16) uint8_t sf_smem[];
+  constexpr int EP = 32 / RB;                        // entries of a sample worked on at once
+  float* ws = reinterpret_cast<float*>(sf_smem);     // RB rows of W, row pitch `pitch` floats
+  int2* ranges = reinterpret_cast<int2*>(ws + static_cast<size_t>(RB) * pitch);   // (begin, end) of the n samples
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r = lane % RB, e = lane / RB;
+  const uint32_t ebuf = shared_addr(ranges + n) + static_cast<uint32_t>(warp) * (kSfBufs * kSfChunk * 8);
+  for (int s = threadIdx.x; s < n; s += kSfThreads) ranges[s] = make_int2(row_beg[off + s], row_end[off + s]);
+  const uint32_t wrow = shared_addr(ws) + static_cast<uint32_t>(r) * pitch * 4u;
+  const int64_t nblk = (rows + RB - 1) / RB;
+  const int quads = static_cast<int>(cols / 4);
+
+  for (int64_t blk = blockIdx.x; blk < nblk; blk += gridDim.x) {
+    const int64_t j0 = blk * RB;
+    __syncthreads();                                 // every warp is done with the previous rows (and ranges is filled)
+    for (int q = threadIdx.x; q < RB * quads; q += kSfThreads) {
+      const int rr = q / quads, cc = (q - rr * quads) * 4;
+      const float4 v = j0 + rr < rows ? *reinterpret_cast<const float4*>(W + (j0 + rr) * cols + cc)
+                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+      *reinterpret_cast<float4*>(ws + static_cast<size_t>(rr) * pitch + cc) = v;
+    }
+    __syncthreads();
+
+    // samples warp, warp + 16, ...: buffer (it % 3) holds the entries of the it-th of them
+    int2 rg = warp < n ? ranges[warp] : make_int2(0, 0);
+    stage_entries(ebuf, cx, rg.x, rg.y, lane);
+    {
+      const int2 r1 = warp + kSfWarps < n ? ranges[warp + kSfWarps] : make_int2(0, 0);
+      stage_entries(ebuf + kSfChunk * 8, cx, r1.x, r1.y, lane);
+    }
+    int it = 0;
+    for (int s = warp; s < n; s += kSfWarps, ++it) {
+      {
+        const int2 r2 = s + 2 * kSfWarps < n ? ranges[s + 2 * kSfWarps] : make_int2(0, 0);
+        stage_entries(ebuf + static_cast<uint32_t>((it + 2) % kSfBufs) * (kSfChunk * 8), cx, r2.x, r2.y, lane);
+      }
+      cp_async_wait<2>();                            // all but the two newest groups: this sample's entries are in
+      __syncwarp();
+      const uint32_t q0 = ebuf + static_cast<uint32_t>(it % kSfBufs) * (kSfChunk * 8) + static_cast<uint32_t>(e) * 8u;
+      const int32_t len = rg.y - rg.x;
+      const int32_t cnt = len < kSfChunk ? len : kSfChunk;
+      float acc = 0.f;
+      uint32_t q = q0;
+      int32_t m = 0;
+      for (; m + 4 * EP <= cnt; m += 4 * EP, q += 4 * EP * 8) {
+        const int2 a0 = lds_v2(q), a1 = lds_v2(q + EP * 8), a2 = lds_v2(q + 2 * EP * 8), a3 = lds_v2(q + 3 * EP * 8);
+        const float w0 = lds_f32(wrow + static_cast<uint32_t>(a0.x) * 4u), w1 = lds_f32(wrow + static_cast<uint32_t>(a1.x) * 4u);
+        const float w2 = lds_f32(wrow + static_cast<uint32_t>(a2.x) * 4u), w3 = lds_f32(wrow + static_cast<uint32_t>(a3.x) * 4u);
+        acc = fmaf(__int_as_float(a0.y), w0, acc); acc = fmaf(__int_as_float(a1.y), w1, acc);
+        acc = fmaf(__int_as_float(a2.y), w2, acc); acc = fmaf(__int_as_float(a3.y), w3, acc);
+      }
+      for (; m < cnt; m += EP, q += EP * 8) {       // the rest: groups of EP entries, zeros after the last entry
+        const int2 a0 = lds_v2(q);
+        acc = fmaf(__int_as_float(a0.y), lds_f32(wrow + static_cast<uint32_t>(a0.x) * 4u), acc);
+      }
+      for (int32_t t = rg.x + kSfChunk + e; t < rg.y; t += EP) {     // a sample of more than kSfChunk entries: the rest
+        const int2 a0 = __ldg(cx + t);
+        acc = fmaf(__int_as_float(a0.y), lds_f32(wrow + static_cast<uint32_t>(a0.x) * 4u), acc);
+      }
+#pragma unroll
+      for (int o = RB; o < 32; o <<= 1) acc += __shfl_xor_sync(kFull, acc, o);
+      if (e == 0 && j0 + r < rows) Z[(off + s) * ldz + j0 + r] = acc;
+      __syncwarp();                                  // the buffer may be refilled two iterations from now
+      rg = s + kSfWarps < n ? ranges[s + kSfWarps] : make_int2(0, 0);
+    }
+    cp_async_wait<0>();
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------
 // The update.  A block owns 32 rows of W at a time and keeps their factor slab u[i][row] (all K samples) in shared
 // memory; its warps take 32-column blocks of those rows.  Within a block of 32 x 32 entries a lane first is a ROW:
 // for each of the 32 columns it sums x_id * u[i][row] over the column's entries (the entries are read by all lanes at
@@ -161,33 +310,6 @@ struct SuParams {
   int64_t shadow32_ld, shadow_half;
   unsigned long long* copy_counters;
 };
-
-// Shared-memory reads of the inner loop through 32-bit shared-space addresses (one integer multiply-add per address).
-__device__ __forceinline__ uint32_t shared_addr(const void* p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ float lds_f32(uint32_t a) {
-  float v;
-  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(a));
-  return v;
-}
-__device__ __forceinline__ uint32_t lds_u16(uint32_t a) {
-  uint16_t v;
-  asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a));
-  return v;
-}
-__device__ __forceinline__ void sts_f32(uint32_t a, float v) {
-  asm volatile("st.shared.f32 [%0], %1;" ::"r"(a), "f"(v) : "memory");
-}
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<const uint32_t*>(&v);
-}
-__device__ __forceinline__ int4 lds_v4(uint32_t a) {
-  int4 v;
-  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
-  return v;
-}
 
 template <int USRC>
 struct Slab {
@@ -406,6 +528,9 @@ void sparse_extend_layout(const sfb_config& c, Layout& L, size_t& off) {
   L.coo_i = take(nnz * 4);
   L.coo_c = take(nnz * 4);
   L.coo_x = take(nnz * 4);
+  L.coo_cx = take((nnz + 128) * 8);
+  L.row_beg = take(static_cast<size_t>(c.workers) * c.batch * 4);
+  L.row_end = take(static_cast<size_t>(c.workers) * c.batch * 4);
   L.csc_cnt = take((cols + 1) * 4);
   L.csc_cur = take((cols + 1) * 4);
   L.csc_ptr = take((cols + 1) * 4);
@@ -438,9 +563,68 @@ int sparse_stage(sfb_ctx* ctx, int64_t off, int64_t n, const int64_t* indptr, co
   if (nnz > 0) CKS(cudaMemsetAsync(ctx->at<int32_t>(L.coo_c) + ctx->csr_fill, 0xff, static_cast<size_t>(nnz) * 4, s));   // "no entry"
   csr_stage_kernel<<<static_cast<unsigned>((n * 32 + 255) / 256), 256, 0, s>>>(
       indptr, idx, val, n, nnz, cols, off, Xd, ctx->at<int32_t>(L.coo_i) + ctx->csr_fill,
-      ctx->at<int32_t>(L.coo_c) + ctx->csr_fill, ctx->at<float>(L.coo_x) + ctx->csr_fill, ctx->at<uint32_t>(L.status));
+      ctx->at<int32_t>(L.coo_c) + ctx->csr_fill, ctx->at<float>(L.coo_x) + ctx->csr_fill,
+      ctx->at<int2>(L.coo_cx) + ctx->csr_fill, static_cast<int32_t>(ctx->csr_fill), ctx->at<int32_t>(L.row_beg),
+      ctx->at<int32_t>(L.row_end), ctx->at<uint32_t>(L.status));
   count_launch();
   CKS(cudaGetLastError());
+  ctx->last_stage_nnz = nnz;
+  return SFB_OK;
+}
+
+namespace {
+
+template <int RB>
+cudaError_t launch_sparse_forward(sfb_ctx* ctx, int64_t off, int64_t n, float* Z, int64_t ldz, int pitch, int smem) {
+  static std::atomic<uint64_t> prepared{0};            // one bit per device ordinal
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const uint64_t bit = 1ull << (dev & 63);
+  if (!(prepared.load(std::memory_order_acquire) & bit)) {
+    e = cudaFuncSetAttribute(sparse_forward_kernel<RB>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemOptIn);
+    if (e != cudaSuccess) return e;
+    prepared.fetch_or(bit, std::memory_order_release);
+  }
+  const Layout& L = ctx->lay;
+  const sfb_config& c = ctx->cfg;
+  const int64_t nblk = (c.rows + RB - 1) / RB;
+  sparse_forward_kernel<RB><<<static_cast<unsigned>(std::min<int64_t>(nblk, sm_count())), kSfThreads, smem, ctx->stream>>>(
+      ctx->W, c.rows, c.cols, pitch, ctx->at<int32_t>(L.row_beg), ctx->at<int32_t>(L.row_end), ctx->at<int2>(L.coo_cx), off,
+      static_cast<int32_t>(n), Z, ldz);
+  count_launch();
+  return cudaGetLastError();
+}
+
+// Row pitch (floats) of the rows of W in shared memory: at least cols, and congruent to 32/RB modulo 32 so that the RB
+// rows of one column fall into different banks.
+int forward_pitch(int64_t cols, int rb) {
+  const int64_t want = rb == 1 ? 0 : 32 / rb;
+  int64_t p = (cols + 31) / 32 * 32 + want;
+  return static_cast<int>(p);
+}
+
+}  // namespace
+
+// Rows of W a block of the row-wise forward can hold (4, 2 or 1), or 0 when even one row does not fit.
+int sparse_forward_rows(const sfb_ctx* ctx, int64_t n) {
+  for (int rb = 4; rb >= 1; rb >>= 1) {
+    const int64_t bytes = static_cast<int64_t>(rb) * forward_pitch(ctx->cfg.cols, rb) * 4 + n * 8 + kSfWarps * kSfBufs * kSfChunk * 8;
+    if (bytes <= kSmemOptIn) return rb;
+  }
+  return 0;
+}
+
+// Z[off .. off+n) = X W^T for the n staged sparse samples at pair offset off (fp32, row pitch ldz).
+int sparse_forward(sfb_ctx* ctx, int64_t off, int64_t n, float* Z, int64_t ldz) {
+  const int rb = sparse_forward_rows(ctx, n);
+  if (rb == 0) return SFB_ERR_SHAPE;
+  const int pitch = forward_pitch(ctx->cfg.cols, rb);
+  const int smem = static_cast<int>(static_cast<int64_t>(rb) * pitch * 4 + n * 8 + kSfWarps * kSfBufs * kSfChunk * 8);
+  if (rb == 4) CKS(launch_sparse_forward<4>(ctx, off, n, Z, ldz, pitch, smem));
+  else if (rb == 2) CKS(launch_sparse_forward<2>(ctx, off, n, Z, ldz, pitch, smem));
+  else CKS(launch_sparse_forward<1>(ctx, off, n, Z, ldz, pitch, smem));
+  ctx->stats.flops += 2.0 * static_cast<double>(ctx->cfg.rows) * static_cast<double>(ctx->last_stage_nnz);
   return SFB_OK;
 }
 
