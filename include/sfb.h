@@ -156,8 +156,10 @@ int sfb_compute_factors(sfb_ctx* ctx, int32_t worker, const float* X_dev, const 
  * left out.  All arrays are copied or consumed before the call returns control of them to the stream order: they may
  * be reused once later work on the stream may overwrite them.
  *
- * u is computed as for dense samples (the logits need every column of W, so the forward product is the dense one over
- * the scattered samples).  When every worker of the step committed in this form, sfb_gather_factors builds the
+ * u is computed as for dense samples.  The logits need every column of W (the non-zero columns of a mini-batch cover
+ * it), so in the tensor-core modes the forward product is the dense one over the scattered samples; in the fp32 FMA
+ * mode it is a row-wise product over the non-zeros (z_ij = sum_t x_it W[j][c_it], rows of W held on chip, cols up to
+ * about 55,000; the dense FMA product beyond).  When every worker of the step committed in this form, sfb_gather_factors builds the
  * column-major form of the K samples (entries of a column in ascending sample order, so the result does not depend on
  * scheduling) and sfb_apply_update sums, per entry of W, only the samples that have a non-zero in that column:
  *     W[j][d] <- prox( W[j][d] - eta * sum_{i : x_id != 0} u_ij x_id ),

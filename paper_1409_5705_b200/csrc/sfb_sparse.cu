@@ -2,8 +2,9 @@
 // sparse; Section 3: a factor v_i = a_i with few non-zeros is sent as its (index, value) pairs).
 //
 // The samples arrive in compressed-sparse-row form.  Their logits still need every column of W (the union of the
-// non-zero columns of a mini-batch covers the matrix), so the forward product stays the dense tensor-core product
-// over the scattered samples.  What the zeros remove is the work of the update:
+// non-zero columns of a mini-batch covers the matrix): the tensor-core modes keep the dense forward product over the
+// scattered samples, the fp32 FMA mode has a row-wise product over the non-zeros (sparse_forward_kernel).  What the
+// zeros remove is the work of the update:
 //     W[j][d] <- prox( W[j][d] - eta * sum_{i : x_id != 0} u_ij x_id )
 // has as many terms per entry as column d has non-zeros in the mini-batch (K * density) instead of K.  The kernel here
 // streams W once, as the dense update does, and sums only those terms, from the column-major (CSC) form of the
