@@ -6,6 +6,9 @@ its own updates it always sees.  s = 0 is bulk-synchronous execution.  Section 5
 replica W_p^c with the reference sequence W^c that applies every update in clock order, and shows that their distance
 vanishes for a decreasing step size.
 
+Asynchronous parallel execution (the third model named there) puts no bound on the delay: staleness = None
+accepts any non-negative delays.
+
 Emulated here exactly as stated, in fp64 numpy: P replicas; at clock c each worker first applies the factor sets
 whose delivery is due, then computes the factors of its minibatch against ITS replica, applies them to its own
 replica at once with the step eta_c, and posts them to every other worker q with the delivery clock
@@ -14,8 +17,8 @@ produced it.  Readings: a worker applies deliveries in (clock, sender) order; th
 clock in sender order at the end of that clock.
 
 Pins (tests/test_ssp_pins.py): s = 0 reproduces the bulk-synchronous step of oracle.sfb_oracle clock by clock; the SSP
-guarantee holds by bookkeeping at every clock; after all deliveries every replica equals the reference; with
-eta_c = eta_0 / (c + 1) the largest distance to the reference decays.
+guarantee holds by bookkeeping at every clock; after all deliveries every replica equals the reference (also without a
+bound on the delays); with eta_c = eta_0 / (c + 1) the largest distance to the reference decays.
 """
 from __future__ import annotations
 
@@ -48,7 +51,7 @@ def emulate(model, W0, batches, etas, delays, staleness, margin=1.0, lam=0.1, L=
             produced.append((U, V))
             for q in range(P):
                 if q != p:
-                    assert 0 <= delays[c][p][q] <= staleness
+                    assert 0 <= delays[c][p][q] and (staleness is None or delays[c][p][q] <= staleness)
                     inbox[q].append((c + 1 + int(delays[c][p][q]), c, p, U, V))
         for p in range(P):
             ref = O.rank_k_update(ref, produced[p][0], produced[p][1], etas[c])

@@ -246,6 +246,15 @@ def ssp_delays(seed: int, clocks: int, workers: int, staleness: int) -> np.ndarr
     return d
 
 
+def asp_delays(seed: int, clocks: int, workers: int, mean: float) -> np.ndarray:
+    """Delays without a bound (asynchronous parallel execution): geometric with the given mean, 0 on the diagonal."""
+    g = _gen(seed, _S_DELAY, 1)
+    d = g.geometric(1.0 / (1.0 + mean), size=(clocks, workers, workers)).astype(np.int64) - 1
+    for p in range(workers):
+        d[:, p, p] = 0
+    return d
+
+
 # ----------------------------------------------------------------------------------------------------------
 # Sparse features (Section "Experiments": the paper's data sets have sparse features).  tf-idf-like samples in
 # compressed-sparse-row form: the number of non-zeros of a sample is Poisson around nnz_mean (at least 1), its columns

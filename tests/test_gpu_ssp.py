@@ -15,7 +15,7 @@ pytestmark = pytest.mark.gpu
 torch = pytest.importorskip("torch")
 
 
-def _run(model_name, prec, s, clocks, tol):
+def _run(model_name, prec, s, clocks, tol, asp_mean=0.0):
     P, B = 3, 8
     if model_name == "mlr":
         wl = I.scaled(I.WORKLOADS["mlr_mid"], "mlr_ssp", rows=45, cols=36, workers=P, batch=B, eta=0.2, w_std=0.3,
@@ -24,9 +24,15 @@ def _run(model_name, prec, s, clocks, tol):
         wl = I.scaled(I.WORKLOADS["dml"], "dml_ssp", rows=24, cols=40, workers=P, batch=B, eta=2e-3)
     W0 = I.initial_W(wl)
     etas = [wl.eta / (c + 1) for c in range(clocks)]
-    for c in range(clocks - (s + 1), clocks):
+    if asp_mean > 0.0:                                        # asynchronous: no bound on the delays (s is None)
+        delays = I.asp_delays(7, clocks, P, asp_mean)
+        tail = int(delays.max()) + 1
+        delays[clocks - tail:] = 0
+    else:
+        delays = I.ssp_delays(7, clocks, P, s)
+        tail = s + 1
+    for c in range(clocks - tail, clocks):
         etas[c] = 0.0                                         # let the deliveries under way arrive
-    delays = I.ssp_delays(7, clocks, P, s)
     batches_h = []
     for c in range(clocks):
         inp = I.step_inputs(wl, c)
@@ -59,6 +65,10 @@ def _run(model_name, prec, s, clocks, tol):
 def test_mlr_fp32_bulk_synchronous_and_stale():
     _run("mlr", S.PREC_FP32, 0, 8, 2e-5)
     _run("mlr", S.PREC_FP32, 2, 12, 2e-5)
+
+
+def test_mlr_fp32_asynchronous():
+    _run("mlr", S.PREC_FP32, None, 24, 2e-5, asp_mean=2.0)
 
 
 def test_dml_split_bf16_stale():

@@ -56,6 +56,24 @@ def test_staleness_guarantee_and_eventual_agreement():
         np.testing.assert_allclose(Wp[-1][p], ref[-1], atol=1e-12)              # same sets, only their order differs
 
 
+def test_asynchronous_execution_agrees_once_every_set_has_arrived():
+    """No bound on the delays (Section 4.1, asynchronous parallel): once every factor set has reached every worker all
+    replicas hold W_0 plus the same sets, so they equal the reference whatever the order of arrival."""
+    wl, W0, batches = _setup(clocks=30)
+    clocks, P = len(batches), wl.workers
+    delays = I.asp_delays(5, clocks, P, 2.5)
+    assert delays.max() >= 6                                   # really beyond any small staleness bound
+    tail = int(delays.max()) + 1
+    etas = [0.2] * (clocks - tail) + [0.0] * tail              # nothing new while the deliveries under way arrive
+    delays[clocks - tail:] = 0
+    Wp, ref, seen = E.emulate(O.MLR, W0, batches, etas, delays, None)
+    late = max(c - c0 for c in range(clocks) for p in range(P) for c0 in range(c)
+               if any((c0, q) not in seen[c][p] for q in range(P)))
+    assert late >= 4                                           # some worker ran four or more clocks behind another
+    for p in range(P):
+        np.testing.assert_allclose(Wp[-1][p], ref[-1], atol=1e-12)
+
+
 def test_distance_to_the_reference_decays_with_a_decreasing_step_size():
     wl, W0, batches = _setup(clocks=60, seed=1)
     clocks, P, s = len(batches), wl.workers, 3
