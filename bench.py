@@ -468,6 +468,9 @@ def main():
                          "Zipf column popularity); the update then sums only the non-zeros of each column")
     ap.add_argument("--sparse-update", default="auto", choices=["auto", "sparse", "dense"],
                     help="with --sparse-nnz: which update the step takes (auto: the library's cost model)")
+    ap.add_argument("--context-library-update", action="store_true",
+                    help="MLR bf16: also time the library way to the same fused update (one cuBLAS GEMM through torch.addmm, "
+                         "bf16 operands, fp32 W read and written with beta = 1), as context beside the roofline")
     ap.add_argument("--shard", default="", choices=["", "rows"],
                     help="rows: partition W by rows over the ranks instead of running replicas")
     args = ap.parse_args()
@@ -643,6 +646,37 @@ def main():
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
 
+    # ---- context, not a target: the same read-modify-write of W as one library GEMM (no bf16 copy of W, no fp32 label
+    # entries); it runs last because it overwrites W with updates of the last step's factors
+    library_update = None
+    if args.context_library_update and rank == 0 and prec == S.PREC_BF16 and wl.model == I.MLR and not sparse:
+        Uq, Vq, dt_, lo_, ldu_, ldv_ = ctx.sfb_get_factors()
+        ws0 = ctx.workspace.data_ptr()
+        UT = ctx.workspace[Uq - ws0:Uq - ws0 + wl.rows * ldu_ * 2].view(torch.bfloat16).view(wl.rows, ldu_)[:, :wl.K]
+        VT = ctx.workspace[Vq - ws0:Vq - ws0 + wl.cols * ldv_ * 2].view(torch.bfloat16).view(wl.cols, ldv_)[:, :wl.K]
+        def library_loop(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                torch.addmm(W, UT, VT.t(), out_dtype=torch.float32, beta=1.0, alpha=-wl.eta, out=W)
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / reps
+
+        library_loop(3)
+        time.sleep(1.0)                                  # let the clocks recover from the runs before
+        ms_burst = library_loop(10)
+        sampler3, sfile3 = clocks_sampler(local)
+        w0 = time.time()
+        reps = max(20, int(args.phase_seconds * 1e3 / ms_burst))
+        ms_long = library_loop(reps)
+        ck3 = clocks_summary(sampler3, sfile3, w0, time.time())
+        library_update = {"call": "torch.addmm(W, U^T, V, out_dtype=float32, beta=1, alpha=-eta, out=W): one cuBLAS GEMM",
+                          "ms_first_10_launches": ms_burst, "ms": ms_long, "launches": reps, "clocks": ck3,
+                          "ms_x_sm_mhz": ms_long * ck3["sm_mhz"] if ck3.get("sm_mhz") else None,
+                          "note": "context only: W read and written in fp32 like the update kernel, but no bf16 operand copy "
+                                  "of W and no fp32 label rows; launches back to back for --phase-seconds"}
+
     total_ms, e2e_ms, ms_f, ms_g, ms_u = max_over_ranks([total_ms, e2e_s * 1e3, ms_f, ms_g, ms_u], dev, world)
     if rank != 0:
         if world > 1:
@@ -714,6 +748,8 @@ def main():
             "operand_copy": copy_stats, "status_word": status}
     if update_loop is not None:
         line["update_loop"] = update_loop
+    if library_update is not None:
+        line["library_update"] = library_update
     print(json.dumps(line), flush=True)
     ctx.close()
     if world > 1:

@@ -38,22 +38,35 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
+// The same with a suspend-time hint: the thread may stay suspended in the wait for up to about `ns` nanoseconds and is
+// woken when the phase completes, so a long wait is a handful of instructions instead of a hot polling loop.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint64_t* bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t"
+      ".reg .pred P;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, P;\n\t"
+      "}\n"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(ns) : "memory");
+  return ok != 0;
+}
 
-// Polls until the phase with this parity has completed.  Gives up (returns false) after kMaxWaitCycles SM clock
+// Waits until the phase with this parity has completed.  Gives up (returns false) after kMaxWaitCycles SM clock
 // cycles (about two seconds) or kMaxPolls polls, whichever comes first, or as soon as *abort is set by another
-// role of the CTA.  The clock is the SM's own cycle counter, which costs a few cycles to read.
+// role of the CTA.  Every poll may suspend the thread for up to kWaitHintNs; the clock is the SM's own cycle counter,
+// read after every unsuccessful poll (cheap beside the suspension).
 constexpr uint32_t kMaxPolls = 1u << 26;
 constexpr long long kMaxWaitCycles = 4000000000ll;
+constexpr uint32_t kWaitHintNs = 2000;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort,
                                           long long max_cycles = kMaxWaitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t i = 0; i < kMaxPolls; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 255u) == 255u) {
-      if (*abort) return false;
-      if (clock64() - t0 > max_cycles) break;
-    }
+    if (mbar_try_wait_hint(bar, parity, kWaitHintNs)) return true;
+    if (*abort) return false;
+    if (clock64() - t0 > max_cycles) break;
   }
   *abort = 1;
   return false;
