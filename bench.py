@@ -226,10 +226,11 @@ def run_reference(args, wl, rank):
 # profiles/ncu_update_pair_kernel_mlr_large_dram.md (dram__bytes_read.sum + dram__bytes_write.sum of one launch of the
 # full-size bench).  The bf16 copy of W is rewritten only where its rounding changed, so the traffic depends on the data
 # and does not scale with the rows: the figure applies to this workload only.  "kernel_unchanged_since" names the
-# commit of csrc/sfb_update.cu the counters were taken at: when the kernel is edited this entry has to be re-captured
+# commit of the kernel's sources (csrc/sfb_update.cu, csrc/sfb_ptx.cuh) the counters were taken at: when the kernel is edited
+# this entry has to be re-captured
 # or set to None.
-NCU_UPDATE_TRAFFIC = {"rows": 325000, "cols": 10000, "K": 1024, "bytes": 15.90e9 + 13.85e9,
-                      "kernel_unchanged_since": "318561f"}
+NCU_UPDATE_TRAFFIC = {"rows": 325000, "cols": 10000, "K": 1024, "bytes": 15.29e9 + 13.85e9,
+                      "kernel_unchanged_since": "d08beef"}
 
 
 def ncu_traffic_per_launch(wl, prec):
