@@ -206,3 +206,62 @@ def test_sparse_and_dense_steps_alternate_on_one_context(prec):
         start = Wg.astype(np.float64)
     assert ctx.sfb_get_stats().sparse_updates == 2
     ctx.close()
+
+
+def _manual_samples(rows_of_entries, cols):
+    """CSR arrays from a list of per-sample [(column, value), ...] lists."""
+    indptr = np.zeros(len(rows_of_entries) + 1, dtype=np.int64)
+    idx, val = [], []
+    for i, ents in enumerate(rows_of_entries):
+        indptr[i + 1] = indptr[i] + len(ents)
+        idx += [c for c, _ in ents]
+        val += [v for _, v in ents]
+    return I.SparseSamples(indptr, np.asarray(idx, dtype=np.int32), np.asarray(val, dtype=np.float32))
+
+
+@pytest.mark.parametrize("prec", [pytest.param(S.PREC_FP32_FFMA, id="ffma"), pytest.param(S.PREC_BF16, id="bf16")])
+def test_degenerate_sparse_batches(prec):
+    """Empty samples, one sample with every column (more than one staging chunk of the row-wise forward and a column
+    block longer than the update's entry window), columns no sample touches, unsorted indices, and a batch with no
+    entry at all."""
+    wl = I.scaled(I.WORKLOADS["mlr_mid"], "mlr_sparse_edge", rows=70, cols=300, workers=2, batch=5, eta=0.1, w_std=0.1,
+                  x_scale="unit")
+    rng = np.random.default_rng(3)
+    full = [(int(c), float(v)) for c, v in zip(rng.permutation(wl.cols), rng.standard_normal(wl.cols) * 0.1)]
+    few = [(299, 0.5), (0, -0.25), (17, 1.0)]                                  # unsorted, first and last column
+    samples = [[], full, few, [], [(5, 2.0)], full[:200], [], [(5, -1.0), (6, 1.0)], few[::-1], []]
+    sp = _manual_samples(samples, wl.cols)
+    labels = I.zipf_labels(wl.seed, 5, 0, wl.K, wl.rows, 0.0)
+    W0 = I.initial_W(wl)
+    W = to_dev(W0, torch)
+    ctx = S.Context(_config(wl, prec, sp.nnz + 8), W)
+    ctx.sfb_step_csr(*_dev(sp, labels)[:3], sp.nnz, to_dev(labels, torch))
+    assert ctx.sfb_get_status() == 0
+    ref = O.sfb_step(I.MLR, W0, I.densify(sp, wl.cols), None, labels, workers=wl.workers, eta=wl.eta)
+    assert rel_err(W.cpu().numpy(), ref, W0) <= TOL[prec]
+    # a batch without a single entry: u = softmax(0) - onehot, v = 0, W unchanged
+    before = W.clone()
+    empty = _manual_samples([[] for _ in range(wl.K)], wl.cols)
+    ip = to_dev(empty.indptr, torch)
+    dummy_i = torch.zeros(1, dtype=torch.int32, device="cuda")
+    dummy_v = torch.zeros(1, dtype=torch.float32, device="cuda")
+    ctx.sfb_step_csr(ip, dummy_i, dummy_v, 0, to_dev(labels, torch))
+    assert ctx.sfb_get_status() == 0
+    assert torch.equal(W, before)
+    assert ctx.sfb_get_stats().sparse_updates == 2
+    ctx.close()
+
+
+def test_a_batch_too_large_for_the_factor_slab_takes_the_dense_update():
+    wl = I.scaled(I.WORKLOADS["mlr_mid"], "mlr_sparse_bigk", rows=64, cols=64, workers=4, batch=640, eta=0.05, w_std=0.1,
+                  x_scale="unit")                                                 # K = 2560: beyond the slab in either mode
+    sp, labels = _inputs(wl, 0, 4.0)
+    W0 = I.initial_W(wl)
+    W = to_dev(W0, torch)
+    ctx = S.Context(_config(wl, S.PREC_FP32_FFMA, sp.nnz), W)
+    ctx.sfb_step_csr(*_dev(sp, labels)[:3], sp.nnz, to_dev(labels, torch))
+    assert ctx.sfb_get_status() == 0
+    assert ctx.sfb_get_stats().sparse_updates == 0
+    ref = O.sfb_step(I.MLR, W0, I.densify(sp, wl.cols), None, labels, workers=wl.workers, eta=wl.eta)
+    assert rel_err(W.cpu().numpy(), ref, W0) <= 1e-5
+    ctx.close()
