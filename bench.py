@@ -469,6 +469,9 @@ def main():
                          "Zipf column popularity); the update then sums only the non-zeros of each column")
     ap.add_argument("--sparse-update", default="auto", choices=["auto", "sparse", "dense"],
                     help="with --sparse-nnz: which update the step takes (auto: the library's cost model)")
+    ap.add_argument("--graph", action="store_true",
+                    help="launch each step as one CUDA graph (captured once per rotating minibatch from the same library "
+                         "calls): for the launch-bound small workloads; value and ms_per_step are then the replays'")
     ap.add_argument("--context-library-update", action="store_true",
                     help="MLR bf16: also time the library way to the same fused update (one cuBLAS GEMM through torch.addmm, "
                          "bf16 operands, fp32 W read and written with beta = 1), as context beside the roofline")
@@ -544,6 +547,8 @@ def main():
                         sc_lambda=wl.sc_lambda, sc_ista_iters=wl.sc_iters, sc_lipschitz=L,
                         sc_prox=1 if wl.model == I.SC else 0, csr_nnz_max=nnz_max,
                         csr_update={"auto": 0, "sparse": 1, "dense": 2}[args.sparse_update])
+    if args.graph:
+        torch.cuda.set_stream(torch.cuda.Stream(dev))      # a step can only be captured on a stream of its own
     ctx = S.Context(cfg, W)
     flusher = None
     if wl.rows * wl.cols * 4 <= 2 * 126e6:
@@ -554,16 +559,19 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    def factors_call(k):
+        if sparse:
+            ctx.sfb_compute_factors_csr(-1, dS[k][0], dS[k][1], dS[k][2], dS[k][3], dL[k])
+        else:
+            ctx.sfb_compute_factors(-1, dX[k], dY[k], dL[k])
+
     def phased_step(i, ev=None):
         k = i % nb
         if flusher is not None:
             flusher.zero_()
         if ev is not None:
             ev[0].record()
-        if sparse:
-            ctx.sfb_compute_factors_csr(-1, dS[k][0], dS[k][1], dS[k][2], dS[k][3], dL[k])
-        else:
-            ctx.sfb_compute_factors(-1, dX[k], dY[k], dL[k])
+        factors_call(k)
         if ev is not None:
             ev[1].record()
         ctx.sfb_gather_factors()
@@ -591,6 +599,10 @@ def main():
     barrier()
     clocks = clocks_summary(sampler, sfile, wall0, time.time()) if rank == 0 else None
     total_ms = t_start.elapsed_time(t_end)
+    ms_incl_flush = total_ms / args.steps
+    if flusher is not None:
+        # the L2 flush runs between the steps; the value counts the steps' own device intervals
+        total_ms = sum(e[0].elapsed_time(e[3]) for e in evs)
     st1 = ctx.sfb_get_stats()
     launches = st1.kernel_launches - launches0
     copy_stats = {"row_pieces_per_step": (st1.copy_pieces - st0.copy_pieces) / args.steps,
@@ -601,6 +613,37 @@ def main():
     ms_f = sum(e[0].elapsed_time(e[1]) for e in evs) / args.steps
     ms_g = sum(e[1].elapsed_time(e[2]) for e in evs) / args.steps
     ms_u = sum(e[2].elapsed_time(e[3]) for e in evs) / args.steps
+
+    # ---- the same steps, each launched as one CUDA graph (captured from the same library calls on the context's stream)
+    graph_info = None
+    if args.graph:
+        l0 = ctx.sfb_get_stats().kernel_launches
+        graphs = []
+        for k in range(nb):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=ctx.stream):
+                factors_call(k)
+                ctx.sfb_gather_factors()
+                ctx.sfb_apply_update()
+            graphs.append(g)
+        per_step_launches = (ctx.sfb_get_stats().kernel_launches - l0) / nb
+        for i in range(3):
+            graphs[i % nb].replay()
+        gev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
+        barrier()
+        for i in range(args.steps):
+            if flusher is not None:
+                flusher.zero_()
+            gev[i][0].record()
+            graphs[i % nb].replay()
+            gev[i][1].record()
+        barrier()
+        g_ms = sum(e[0].elapsed_time(e[1]) for e in gev) if flusher is not None else gev[0][0].elapsed_time(gev[-1][1])
+        graph_info = {"ms_per_step": g_ms / args.steps, "eager_ms_per_step": total_ms / args.steps,
+                      "kernels_per_graph": per_step_launches, "graphs": nb}
+        status |= ctx.sfb_get_status()
+        total_ms = g_ms
+        launches = int(per_step_launches * args.steps)
 
     # ---- the fused update alone, back to back (same factors applied again and again): separates the kernel from the
     # rest of the step; ms x median SM MHz is the clock-independent figure
@@ -747,6 +790,13 @@ def main():
                       "dense_sync": wl.workers * wl.rows * wl.cols * 4,
                       "dense_over_sf": wl.workers * wl.rows * wl.cols * 4 / one_copy},
             "operand_copy": copy_stats, "status_word": status}
+    if flusher is not None:
+        line["ms_per_step_incl_l2_flush"] = ms_incl_flush
+        line["config"]["l2"] = "l2_flushed_between_steps (the flush is outside the timed intervals)"
+    if graph_info is not None:
+        line["graph"] = graph_info
+        line["config"]["launch"] = "one CUDA graph per step"
+
     if update_loop is not None:
         line["update_loop"] = update_loop
     if library_update is not None:

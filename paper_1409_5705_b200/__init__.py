@@ -239,6 +239,18 @@ class Context:
             return view(U, K, ldu)[:, :rows].float(), view(V, K, ldv)[:, :cols].float()
         return view(U, rows, ldu)[:, :K].t().float(), view(V, cols, ldv)[:, :K].t().float()
 
+    def capture(self, calls):
+        """Captures the library calls made by ``calls()`` on this context's stream into one CUDA graph and returns it
+        (``.replay()`` launches them again on the same buffers).  The context must have been created on a stream of
+        its own (not the default stream), and every kind of call in ``calls`` must have run once before, so that
+        one-off set-up (kernel attributes) is not part of the capture.  Plumbing only: torch records what the library
+        launches."""
+        import torch
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=self.stream):
+            calls()
+        return g
+
     def operand_copy_as_tensor(self):
         """The library's operand copy of W as a torch view into the workspace: bf16 [rows, ld] (MLR, bf16 mode) or
         fp32 [rows, ld] with the (big | small) tf32 halves side by side (tensor-core fp32 mode)."""
