@@ -36,7 +36,7 @@ typedef struct sfb_ctx sfb_ctx;
  * ascent (Section 2.1 "Stochastic DCA"; the fourth model of Section 6).  See sfb_sdca_compute_factors. */
 enum sfb_model { SFB_MLR = 0, SFB_DML = 1, SFB_SC = 2, SFB_L2MLR = 3 };
 
-/* Operand precision of the matrix products.  The master copy of W is fp32 in both modes.
+/* Operand precision of the matrix products.  The master copy of W is fp32 in every mode.
  * SFB_PREC_BF16: tensor-core products on bf16 operands with fp32 accumulation.  MLR: forward and update
  *                products on single bf16 operands (the label entry of u is kept in fp32).  DML, SC: u is a residual
  *                that cancels, so every product -- the forward W v, the products of the ISTA coder and the update --
@@ -159,9 +159,10 @@ int sfb_compute_factors(sfb_ctx* ctx, int32_t worker, const float* X_dev, const 
  * u is computed as for dense samples.  The logits need every column of W (the non-zero columns of a mini-batch cover
  * it), so in the tensor-core modes the forward product is the dense one over the scattered samples; in the fp32 FMA
  * mode it is a row-wise product over the non-zeros (z_ij = sum_t x_it W[j][c_it], rows of W held on chip, cols up to
- * about 55,000; the dense FMA product beyond).  When every worker of the step committed in this form, sfb_gather_factors builds the
- * column-major form of the K samples (entries of a column in ascending sample order, so the result does not depend on
- * scheduling) and sfb_apply_update sums, per entry of W, only the samples that have a non-zero in that column:
+ * about 55,000; the dense FMA product beyond).
+ * When every worker of the step committed in this form, sfb_gather_factors builds the column-major form of the K
+ * samples (entries of a column in ascending sample order, so the result does not depend on scheduling) and
+ * sfb_apply_update sums, per entry of W, only the samples that have a non-zero in that column:
  *     W[j][d] <- prox( W[j][d] - eta * sum_{i : x_id != 0} u_ij x_id ),
  * one pass over W as in the dense update, the derived operand copies of W rewritten with it.  sfb_stats.gather_bytes
  * then counts K*rows*element size for the u and 8 bytes per non-zero for the v.  A mini-batch too large for the
