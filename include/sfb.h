@@ -205,12 +205,19 @@ int sfb_sdca_compute_factors(sfb_ctx* ctx, int32_t worker, const float* X_dev, c
                              const int32_t* sample_ids_dev);
 int sfb_sdca_step(sfb_ctx* ctx, const float* X_dev, const int32_t* labels_dev, const int32_t* sample_ids_dev);
 
-/* The receiving side of the broadcast (Section 3: a worker applies the sufficient factors it has received from the
- * others): the B pairs U_dev [B x rows], V_dev [B x cols] (fp32, pair-major, dense rows), computed elsewhere -- by
- * another replica, under another consistency model (Section 4.1), on another machine -- take worker `worker`'s place
- * in the gathered buffers and the worker counts as committed.  Pairs come out of a context through sfb_get_factors.
- * Built for the layouts in which factors are fp32 pairs (SFB_PREC_FP32; DML and SC in either mode); SFB_ERR_UNSUPPORTED
- * for MLR in bf16 mode (its u is held as bf16 probabilities plus an fp32 label term) and for SFB_L2MLR. */
+/* The two sides of the broadcast (Section 3: every worker sends its sufficient factors to the others and applies the
+ * ones it receives).
+ * sfb_export_factors: the fp32 factors of worker `worker` as they are sent, U_out_dev [B x rows], V_out_dev [B x cols]
+ * (pair-major, dense rows).  Valid between that worker's sfb_compute_factors and the update (SFB_ERR_STATE otherwise).
+ * In bf16 mode MLR holds logits and log-partitions rather than u:  u_ij = exp(z_ij - lse_i) - [j = y_i]  is formed here
+ * in fp32.
+ * sfb_set_factors: B pairs U_dev, V_dev of the same form, computed elsewhere -- by another replica, under another
+ * consistency model (Section 4.1), on another machine -- take worker `worker`'s place in the gathered buffers and the
+ * worker counts as committed.  For MLR in bf16 mode a received u is split the way a local one is: the class of the
+ * sample is read off it (u = p - onehot(y) has its one negative, hence smallest, entry at y), that entry goes to W in
+ * fp32, the rest as bf16.
+ * Both: SFB_ERR_UNSUPPORTED for SFB_L2MLR. */
+int sfb_export_factors(sfb_ctx* ctx, int32_t worker, float* U_out_dev, float* V_out_dev);
 int sfb_set_factors(sfb_ctx* ctx, int32_t worker, const float* U_dev, const float* V_dev);
 
 /* Changes the step size eta of the following updates (step-size schedules, e.g. the decreasing eta_c of the

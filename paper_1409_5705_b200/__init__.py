@@ -23,7 +23,7 @@ EXPORTS = ("sfb_workspace_bytes", "sfb_init", "sfb_compute_factors", "sfb_gather
            "sfb_selftest_wait_timeout", "sfb_set_row_shard", "sfb_forward_partials", "sfb_finish_factors",
            "sfb_replay_update", "sfb_refresh_operands", "sfb_sdca_set_dual", "sfb_sdca_compute_factors",
            "sfb_sdca_step", "sfb_set_factors", "sfb_set_eta", "sfb_get_operand_copy", "sfb_compute_factors_csr",
-           "sfb_step_csr")
+           "sfb_step_csr", "sfb_export_factors")
 NOALLOC_MAX_COLS = 16384
 
 
@@ -92,6 +92,7 @@ def lib() -> ctypes.CDLL:
         L.sfb_sdca_compute_factors.argtypes = [vp, i32, vp, vp, vp]
         L.sfb_sdca_step.argtypes = [vp, vp, vp, vp]
         L.sfb_set_factors.argtypes = [vp, i32, vp, vp]
+        L.sfb_export_factors.argtypes = [vp, i32, vp, vp]
         L.sfb_set_eta.argtypes = [vp, ctypes.c_float]
         L.sfb_get_operand_copy.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(i32), ctypes.POINTER(i64)]
         L.sfb_compute_factors_csr.argtypes = [vp, i32, vp, vp, vp, i64, vp]
@@ -181,6 +182,10 @@ class Context:
         """U [B, rows], V [B, cols]: contiguous fp32 CUDA tensors of factors computed elsewhere."""
         self._ck(lib().sfb_set_factors(self._h, worker, _ptr(U), _ptr(V)), "sfb_set_factors")
 
+    def sfb_export_factors(self, worker, U_out, V_out):
+        """U_out [B, rows], V_out [B, cols]: contiguous fp32 CUDA tensors that receive the worker's factors as they are sent."""
+        self._ck(lib().sfb_export_factors(self._h, worker, _ptr(U_out), _ptr(V_out)), "sfb_export_factors")
+
     def sfb_set_eta(self, eta):
         self._ck(lib().sfb_set_eta(self._h, eta), "sfb_set_eta")
         self.cfg.eta = eta
@@ -200,7 +205,7 @@ class Context:
                                                _ptr(labels)), "sfb_compute_factors_csr")
 
     def sfb_step_csr(self, indptr, indices, values, nnz, labels):
-        self._ck(lib().sfb_step_csr(self._h, _ptr(indptr), _ptr(indices), _ptr(values), nnz, _ptr(labels)), "sfb_step_csr")
+        self._ck(lib().sfb_step_csr(self._h, _ptr(indptr), _ptr(indices), _ptr(values), nnz, _ptr(labels)), "sfb_step_csr", "sfb_export_factors")
 
     def sfb_step_host(self, X, Y=None, labels=None):
         """X, Y, labels: host tensors / numpy arrays (pinned recommended).  Returns (mean loss, status word)."""

@@ -14,7 +14,7 @@ from __future__ import annotations
 
 class StaleSynchronousWorkers:
     def __init__(self, contexts, reference_context=None):
-        """contexts[p]: a Context with workers = 1 over worker p's replica (fp32 factors: SFB_PREC_FP32, or DML / SC).
+        """contexts[p]: a Context with workers = 1 over worker p's replica (any precision).
         reference_context: optional context over a further copy of W that applies every set in clock order."""
         self.ctx = list(contexts)
         self.ref = reference_context
@@ -40,8 +40,9 @@ class StaleSynchronousWorkers:
             X, Y, labels = batches[p]
             ctx.sfb_set_eta(eta)
             ctx.sfb_compute_factors(0, X, Y, labels)
-            U, V = ctx.factors_as_tensors()
-            U, V = U.clone().contiguous(), V.clone().contiguous()   # the copy that is "sent"
+            U = X.new_empty((ctx.cfg.batch, ctx.cfg.rows))           # the copy that is "sent"
+            V = X.new_empty((ctx.cfg.batch, ctx.cfg.cols))
+            ctx.sfb_export_factors(0, U, V)
             ctx.sfb_gather_factors()
             ctx.sfb_apply_update()
             produced.append((U, V))

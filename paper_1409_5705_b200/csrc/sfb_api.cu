@@ -400,10 +400,18 @@ extern "C" int sfb_set_factors(sfb_ctx* ctx, int32_t worker, const float* U_dev,
   if (!ctx || !U_dev || !V_dev) return SFB_ERR_ARG;
   const sfb_config& c = ctx->cfg;
   if (worker < 0 || worker >= c.workers) return SFB_ERR_SHAPE;
-  if (ctx->sdca || (c.precision == SFB_PREC_BF16 && c.model == SFB_MLR)) return SFB_ERR_UNSUPPORTED;
+  if (ctx->sdca) return SFB_ERR_UNSUPPORTED;
   if (ctx->partials_ready) return SFB_ERR_STATE;
   if (ctx->committed == 0) CK(cudaEventRecord(ctx->ev[0], ctx->stream));
   const int64_t off = static_cast<int64_t>(worker) * c.batch;
+  if (c.precision == SFB_PREC_BF16 && c.model == SFB_MLR) {
+    const int rc = tc_import_factors(ctx, off, c.batch, U_dev, V_dev);
+    if (rc) return rc;
+    ctx->committed |= 1ull << worker;
+    ctx->sparse_mask &= ~(1ull << worker);
+    ctx->gathered = false;
+    return SFB_OK;
+  }
   const int64_t ldu = c.precision == SFB_PREC_FP32 ? c.rows : ctx->lay.ldu;
   float* U = ctx->at<float>(ctx->lay.U) + off * ldu;
   float* V = ctx->at<float>(ctx->lay.V) + off * c.cols;
@@ -413,6 +421,23 @@ extern "C" int sfb_set_factors(sfb_ctx* ctx, int32_t worker, const float* U_dev,
   ctx->committed |= 1ull << worker;
   ctx->sparse_mask &= ~(1ull << worker);             // received factors are dense
   ctx->gathered = false;
+  return SFB_OK;
+}
+
+extern "C" int sfb_export_factors(sfb_ctx* ctx, int32_t worker, float* U_out_dev, float* V_out_dev) {
+  if (!ctx || !U_out_dev || !V_out_dev) return SFB_ERR_ARG;
+  const sfb_config& c = ctx->cfg;
+  if (worker < 0 || worker >= c.workers) return SFB_ERR_SHAPE;
+  if (ctx->sdca) return SFB_ERR_UNSUPPORTED;
+  if (!(ctx->committed & (1ull << worker))) return SFB_ERR_STATE;
+  const int64_t off = static_cast<int64_t>(worker) * c.batch;
+  if (c.precision == SFB_PREC_BF16 && c.model == SFB_MLR) return tc_export_factors(ctx, off, c.batch, U_out_dev, V_out_dev);
+  const int64_t ldu = c.precision == SFB_PREC_FP32 ? c.rows : ctx->lay.ldu;
+  CK(cudaMemcpy2DAsync(U_out_dev, static_cast<size_t>(c.rows) * 4, ctx->at<float>(ctx->lay.U) + off * ldu,
+                       static_cast<size_t>(ldu) * 4, static_cast<size_t>(c.rows) * 4, static_cast<size_t>(c.batch),
+                       cudaMemcpyDeviceToDevice, ctx->stream));
+  CK(cudaMemcpyAsync(V_out_dev, ctx->at<float>(ctx->lay.V) + off * c.cols, static_cast<size_t>(c.batch) * c.cols * 4,
+                     cudaMemcpyDeviceToDevice, ctx->stream));
   return SFB_OK;
 }
 

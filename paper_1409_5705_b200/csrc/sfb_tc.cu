@@ -1295,6 +1295,95 @@ int tc_finish_factors(sfb_ctx* ctx, const float* parts, int shards) {
   return SFB_OK;
 }
 
+// What a worker sends (Section 3) in bf16 mode: u_ij = exp(z_ij - lse_i) - [j = y_i] in fp32 from the logits and the
+// log-partition it holds; one block row per sample.
+__global__ void __launch_bounds__(256) mlr_export_u_kernel(const float* __restrict__ Z, int64_t ldz, int64_t rows,
+                                                           const float* __restrict__ lse, const int32_t* __restrict__ labels,
+                                                           int64_t off, float* __restrict__ U_out) {
+  const int64_t i = blockIdx.y;
+  const float l = lse[off + i];
+  const int32_t y = labels[off + i];
+  const float* z = Z + (off + i) * ldz;
+  float* u = U_out + i * rows;
+  const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+  for (int64_t j = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; j < rows; j += stride)
+    u[j] = expf(z[j] - l) - (j == y ? 1.f : 0.f);
+}
+
+// A received u = p - onehot(y): its smallest entry is the (only negative) one at y.  Per sample: the class, the fp32
+// label coefficient 1 - p_y = -u_y and the loss -log p_y, as the local softmax pass leaves them.  One block per sample;
+// ties (none for a valid u) go to the smaller index.
+__global__ void __launch_bounds__(256) mlr_import_labels_kernel(const float* __restrict__ U_in, int64_t rows, int64_t off,
+                                                                int32_t* __restrict__ labels, float* __restrict__ coef,
+                                                                float* __restrict__ loss) {
+  __shared__ float sv[256];
+  __shared__ int32_t si[256];
+  const int64_t i = blockIdx.x;
+  const float* u = U_in + i * rows;
+  float best = INFINITY;
+  int32_t arg = 0;
+  for (int64_t j = threadIdx.x; j < rows; j += 256) {
+    const float v = u[j];
+    if (v < best) { best = v; arg = static_cast<int32_t>(j); }
+  }
+  sv[threadIdx.x] = best; si[threadIdx.x] = arg;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if (threadIdx.x < o) {
+      const float v = sv[threadIdx.x + o];
+      const int32_t a = si[threadIdx.x + o];
+      if (v < sv[threadIdx.x] || (v == sv[threadIdx.x] && a < si[threadIdx.x])) { sv[threadIdx.x] = v; si[threadIdx.x] = a; }
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const float c = fminf(fmaxf(-sv[0], 0.f), 1.f);
+    labels[off + i] = si[0];
+    coef[off + i] = c;
+    loss[off + i] = -logf(fmaxf(1.f - c, 1e-37f));
+  }
+}
+
+int tc_export_factors(sfb_ctx* ctx, int64_t off, int64_t n, float* U_out, float* V_out) {
+  const sfb_config& c = ctx->cfg;
+  const Layout& L = ctx->lay;
+  const int64_t ldz = round_up(c.rows, 32);
+  dim3 grid(static_cast<unsigned>(std::min<int64_t>((c.rows + 255) / 256, 64)), static_cast<unsigned>(n));
+  mlr_export_u_kernel<<<grid, 256, 0, ctx->stream>>>(ctx->at<float>(L.ZT), ldz, c.rows, ctx->at<float>(L.V),
+                                                     ctx->at<int32_t>(L.labels), off, U_out);
+  count_launch();
+  CKC(cudaGetLastError());
+  CKC(cudaMemcpyAsync(V_out, ctx->at<float>(L.Xf) + off * c.cols, static_cast<size_t>(n) * c.cols * 4, cudaMemcpyDeviceToDevice,
+                      ctx->stream));
+  return SFB_OK;
+}
+
+// Received fp32 factors take a worker's place in the bf16 layout: v into V^T (bf16) and the fp32 sample copy, u into U^T
+// (bf16, 0 at the class entry), the class entry into the fp32 label coefficients.
+int tc_import_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* U_in, const float* V_in) {
+  const sfb_config& c = ctx->cfg;
+  const Layout& L = ctx->lay;
+  const int64_t rows = c.rows, cols = c.cols;
+  const int64_t ldz = round_up(rows, 32);
+  cudaStream_t s = ctx->stream;
+  int32_t* labels = ctx->at<int32_t>(L.labels);
+  mlr_import_labels_kernel<<<static_cast<unsigned>(n), 256, 0, s>>>(U_in, rows, off, labels, ctx->at<float>(L.coef),
+                                                                   ctx->at<float>(L.loss));
+  count_launch();
+  float* Z = ctx->at<float>(L.ZT);
+  CKC(cudaMemcpy2DAsync(Z + off * ldz, static_cast<size_t>(ldz) * 4, U_in, static_cast<size_t>(rows) * 4,
+                        static_cast<size_t>(rows) * 4, static_cast<size_t>(n), cudaMemcpyDeviceToDevice, s));
+  dim3 pgrid(static_cast<unsigned>((cols + 63) / 64), static_cast<unsigned>((n + 63) / 64));
+  pack_mlr_kernel<<<pgrid, 256, 0, s>>>(V_in, n, cols, ctx->at<__nv_bfloat16>(L.Xb), L.colsb, ctx->at<__nv_bfloat16>(L.VT), L.Kp,
+                                        off, ctx->at<float>(L.Xf), labels + off, labels);
+  count_launch();
+  dim3 egrid(static_cast<unsigned>((rows + 63) / 64), static_cast<unsigned>((n + 63) / 64));
+  mlr_emit_ut_kernel<true><<<egrid, 256, 0, s>>>(Z, ldz, rows, nullptr, off, n, labels + off, ctx->at<__nv_bfloat16>(L.UT), L.Kp);
+  count_launch();
+  CKC(cudaGetLastError());
+  return SFB_OK;
+}
+
 // SDCA factors in bf16 mode: logits by the forward product, the dual changes in fp32 in place of the logits, then the
 // bf16 operand U^T = du (0 at the label entry, which goes to W in fp32 through coef, as for MLR).
 int tc_sdca_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const int32_t* labels, const int32_t* ids,

@@ -28,6 +28,9 @@ int tc_forward_partials(sfb_ctx* ctx, const float* X, const int32_t* labels, flo
 int tc_finish_factors(sfb_ctx* ctx, const float* parts, int shards);
 int tc_sdca_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const int32_t* labels, const int32_t* ids,
                     float inv_lam_n);
+// MLR, bf16 mode: a worker's factors in fp32 as they are sent, and received fp32 factors put into the bf16 layout.
+int tc_export_factors(sfb_ctx* ctx, int64_t off, int64_t n, float* U_out, float* V_out);
+int tc_import_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* U_in, const float* V_in);
 int tc_gather(sfb_ctx* ctx);
 int tc_update(sfb_ctx* ctx);
 int tc_get_factors(sfb_ctx* ctx, const void** U, const void** V, int32_t* dtype, int32_t* layout, int64_t* ldu,

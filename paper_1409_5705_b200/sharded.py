@@ -22,6 +22,8 @@ from __future__ import annotations
 
 from dataclasses import dataclass
 
+from . import MLR, PREC_BF16
+
 
 def row_shard_bounds(rows: int, shards: int, g: int) -> tuple[int, int]:
     """Rows [r0, r1) of shard g when ``rows`` rows are dealt to ``shards`` shards as evenly as possible (the first
@@ -92,7 +94,7 @@ def sharded_step(ctx, X_local, labels_local, partials, partials_all, X_all, labe
 def replica_step(ctx, my_workers, X_local, Y_local, labels_local, U_all, V_all, group=None, dist=None):
     """One step of the replica form on this rank.
 
-    ctx          a context over this rank's replica of W with ALL P workers in its config (fp32 factor layout)
+    ctx          a context over this rank's replica of W with ALL P workers in its config (any precision)
     my_workers   the worker indices this rank computes, ascending and contiguous; X_local [len*B, in_dim] etc. hold
                  their samples in that order
     U_all, V_all [K, rows], [K, cols] fp32: receive every worker's factors (worker-major)
@@ -103,20 +105,23 @@ def replica_step(ctx, my_workers, X_local, Y_local, labels_local, U_all, V_all, 
         sl = slice(k * B, (k + 1) * B)
         ctx.sfb_compute_factors(p, X_local[sl], None if Y_local is None else Y_local[sl],
                                 None if labels_local is None else labels_local[sl])
-    U, V = ctx.factors_as_tensors()
     lo, hi = my_workers[0] * B, (my_workers[-1] + 1) * B
-    U_own, V_own = U[lo:hi].contiguous(), V[lo:hi].contiguous()
+    # what this rank sends: its workers' factors in fp32, written straight into their places of the receive buffers
+    U_own, V_own = U_all[lo:hi], V_all[lo:hi]
+    for k, p in enumerate(my_workers):
+        ctx.sfb_export_factors(p, U_own[k * B:(k + 1) * B], V_own[k * B:(k + 1) * B])
     if dist is None:
-        U_all[lo:hi].copy_(U_own)
-        V_all[lo:hi].copy_(V_own)
         received = 0
     else:
-        dist.all_gather_into_tensor(U_all, U_own, group=group)
-        dist.all_gather_into_tensor(V_all, V_own, group=group)
+        dist.all_gather_into_tensor(U_all, U_own.clone(), group=group)
+        dist.all_gather_into_tensor(V_all, V_own.clone(), group=group)
         received = (U_all.numel() - U_own.numel() + V_all.numel() - V_own.numel()) * U_all.element_size()
     mine = set(my_workers)
+    # MLR in bf16 mode rounds a received u to its bf16 operand; a rank takes its own factors back the same way, so that
+    # every replica applies the same operands bit for bit and the replicas do not drift apart
+    reimport_own = getattr(ctx.cfg, "model", None) == MLR and getattr(ctx.cfg, "precision", None) == PREC_BF16
     for q in range(ctx.cfg.workers):
-        if q not in mine:
+        if q not in mine or reimport_own:
             ctx.sfb_set_factors(q, U_all[q * B:(q + 1) * B], V_all[q * B:(q + 1) * B])
     ctx.sfb_gather_factors()
     ctx.sfb_apply_update()

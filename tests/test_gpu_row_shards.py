@@ -153,14 +153,14 @@ def test_row_shard_call_order_and_argument_errors():
     cd.close()
 
 
-@pytest.mark.parametrize("name", ["mlr", "dml"])
+@pytest.mark.parametrize("name", ["mlr", "mlr_bf16", "dml"])
 def test_replica_form_two_ranks_on_one_gpu(name):
     """The paper's own form: two replicas of W, each computes the factors of half of the workers, the factors are
     exchanged (here: copied between the two contexts' buffers, as an all-gather would), both apply all K pairs.  Both
     replicas must end at the oracle's step."""
     from paper_1409_5705_b200.sharded import replica_step
-    if name == "mlr":
-        wl, prec = I.scaled(_workload(), "mlr_rep", workers=4, batch=20), S.PREC_FP32
+    if name.startswith("mlr"):
+        wl, prec = I.scaled(_workload(), "mlr_rep", workers=4, batch=20), S.PREC_BF16 if name == "mlr_bf16" else S.PREC_FP32
     else:
         wl, prec = I.scaled(I.WORKLOADS["dml"], "dml_rep", rows=150, cols=388, workers=4, batch=33, eta=1e-3), S.PREC_BF16
     W0 = I.initial_W(wl)
@@ -179,13 +179,16 @@ def test_replica_form_two_ranks_on_one_gpu(name):
         for p in own[g]:
             sl = slice(p * B, (p + 1) * B)
             ctx.sfb_compute_factors(p, X[sl], None if Y is None else Y[sl], lab[sl])
-        U, V = ctx.factors_as_tensors()
-        U_all[lo:hi].copy_(U[lo:hi])
-        V_all[lo:hi].copy_(V[lo:hi])
+        for p in own[g]:
+            ctx.sfb_export_factors(p, U_all[p * B:(p + 1) * B], V_all[p * B:(p + 1) * B])
+    if name == "mlr_bf16":
+        # what was sent is the fp32 u of Section 2.1, class entry included (the bf16 layout itself holds 0 there)
+        Uo, _ = O.mlr_factors(W0, inp.X, inp.labels)
+        assert np.abs(U_all.cpu().numpy() - Uo).max() <= 2e-3 * np.abs(Uo).max()
     # phase 2: every rank takes the others' factors and applies all K pairs
     for g, ctx in enumerate(ctxs):
         for q in range(wl.workers):
-            if q not in own[g]:
+            if q not in own[g] or name == "mlr_bf16":          # bf16 MLR: own factors go the same way as received ones
                 ctx.sfb_set_factors(q, U_all[q * B:(q + 1) * B], V_all[q * B:(q + 1) * B])
         ctx.sfb_gather_factors()
         ctx.sfb_apply_update()

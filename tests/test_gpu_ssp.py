@@ -75,12 +75,23 @@ def test_dml_split_bf16_stale():
     _run("dml", S.PREC_BF16, 2, 10, 2e-4)
 
 
-def test_received_factors_are_refused_where_the_layout_has_none():
+def test_mlr_bf16_stale():
+    """The default precision: a worker sends the fp32 u formed from its logits (sfb_export_factors), the receiver splits
+    it again into bf16 operand and fp32 class entry."""
+    _run("mlr", S.PREC_BF16, 2, 10, 4e-3)
+
+
+def test_export_and_receive_call_order_and_refusals():
     W = torch.zeros((16, 8), dtype=torch.float32, device="cuda")
-    ctx = S.Context(S.make_config(S.MLR, 16, 8, 1, 4, 0.1, S.PREC_BF16), W)
     U = torch.zeros((4, 16), dtype=torch.float32, device="cuda")
     V = torch.zeros((4, 8), dtype=torch.float32, device="cuda")
-    with pytest.raises(S.SfbError) as e:
+    ctx = S.Context(S.make_config(S.MLR, 16, 8, 1, 4, 0.1, S.PREC_BF16), W)
+    with pytest.raises(S.SfbError) as e:                      # nothing computed yet: nothing to send
+        ctx.sfb_export_factors(0, U, V)
+    assert e.value.code == -9
+    ctx.close()
+    ctx = S.Context(S.make_config(S.L2MLR, 16, 8, 1, 4, 0.1, S.PREC_FP32, sdca_lambda=0.1, sdca_n=32), W)
+    with pytest.raises(S.SfbError) as e:                      # the dual step has no receiving side here
         ctx.sfb_set_factors(0, U, V)
     assert e.value.code == -10
     ctx.close()

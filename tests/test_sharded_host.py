@@ -169,8 +169,10 @@ class _FakeReplica:
         self.V[p * B:(p + 1) * B] = torch.from_numpy(V)
         self.have.add(p)
 
-    def factors_as_tensors(self):
-        return self.U, self.V
+    def sfb_export_factors(self, p, U_out, V_out):
+        B = self.cfg.batch
+        U_out.copy_(self.U[p * B:(p + 1) * B])
+        V_out.copy_(self.V[p * B:(p + 1) * B])
 
     def sfb_set_factors(self, q, U, V):
         B = self.cfg.batch
