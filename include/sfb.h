@@ -281,6 +281,15 @@ int sfb_set_row_shard(sfb_ctx* ctx, int64_t row_offset, int64_t global_rows);
 int sfb_forward_partials(sfb_ctx* ctx, const float* X_dev, const int32_t* labels_dev, float* partials_dev);
 int sfb_finish_factors(sfb_ctx* ctx, const float* partials_all_dev, int32_t shards);
 
+/* The same partition for DML (Section 2, DML; W is the k x D map): a context holds latent rows [row_offset, row_offset +
+ * rows) of W (sfb_set_row_shard), z_i = W v_i splits over the shards and the hinge of a dissimilar pair needs
+ * ||z_i||^2 = the sum over the shards of ||z_i,shard||^2.  sfb_forward_partials_pairs: v = x - y and this shard's z for all
+ * K pairs, partials_dev [K] fp32 = this shard's squared norms.  sfb_finish_factors with partials_all_dev [shards][K] (all
+ * shards' values, shard-major, summed in that order): u = 2 z (similar), -2 z if ||z||^2 < margin else 0.  Then
+ * sfb_gather_factors and sfb_apply_update as usual; u and the update stay local to the shard. */
+int sfb_forward_partials_pairs(sfb_ctx* ctx, const float* X_dev, const float* Y_dev, const int32_t* similar_dev,
+                               float* partials_dev);
+
 /* Full-matrix-synchronisation comparison path (Section 3 "SFB vs client-server", Section 5): every worker
  * materialises its dense update U_p^T V_p in scratch, the P matrices are summed, and W <- W - eta * sum.
  * scratch_dev: at least 2*rows*cols*4 bytes.  Same result as sfb_step up to summation order.  Built for

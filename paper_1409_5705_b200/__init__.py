@@ -23,7 +23,7 @@ EXPORTS = ("sfb_workspace_bytes", "sfb_init", "sfb_compute_factors", "sfb_gather
            "sfb_selftest_wait_timeout", "sfb_set_row_shard", "sfb_forward_partials", "sfb_finish_factors",
            "sfb_replay_update", "sfb_refresh_operands", "sfb_sdca_set_dual", "sfb_sdca_compute_factors",
            "sfb_sdca_step", "sfb_set_factors", "sfb_set_eta", "sfb_get_operand_copy", "sfb_compute_factors_csr",
-           "sfb_step_csr", "sfb_export_factors")
+           "sfb_step_csr", "sfb_export_factors", "sfb_forward_partials_pairs")
 NOALLOC_MAX_COLS = 16384
 
 
@@ -86,6 +86,7 @@ def lib() -> ctypes.CDLL:
         L.sfb_set_row_shard.argtypes = [vp, i64, i64]
         L.sfb_forward_partials.argtypes = [vp, vp, vp, vp]
         L.sfb_finish_factors.argtypes = [vp, vp, i32]
+        L.sfb_forward_partials_pairs.argtypes = [vp, vp, vp, vp, vp]
         L.sfb_replay_update.argtypes = [vp]
         L.sfb_refresh_operands.argtypes = [vp]
         L.sfb_sdca_set_dual.argtypes = [vp, vp, i64]
@@ -205,7 +206,7 @@ class Context:
                                                _ptr(labels)), "sfb_compute_factors_csr")
 
     def sfb_step_csr(self, indptr, indices, values, nnz, labels):
-        self._ck(lib().sfb_step_csr(self._h, _ptr(indptr), _ptr(indices), _ptr(values), nnz, _ptr(labels)), "sfb_step_csr", "sfb_export_factors")
+        self._ck(lib().sfb_step_csr(self._h, _ptr(indptr), _ptr(indices), _ptr(values), nnz, _ptr(labels)), "sfb_step_csr", "sfb_export_factors", "sfb_forward_partials_pairs")
 
     def sfb_step_host(self, X, Y=None, labels=None):
         """X, Y, labels: host tensors / numpy arrays (pinned recommended).  Returns (mean loss, status word)."""
@@ -283,6 +284,10 @@ class Context:
     def sfb_forward_partials(self, X, labels, partials):
         """partials: fp32 CUDA tensor [K, 4] that receives this shard's (max, sum exp, label logit, owner flag)."""
         self._ck(lib().sfb_forward_partials(self._h, _ptr(X), _ptr(labels), _ptr(partials)), "sfb_forward_partials")
+
+    def sfb_forward_partials_pairs(self, X, Y, similar, partials):
+        self._ck(lib().sfb_forward_partials_pairs(self._h, _ptr(X), _ptr(Y), _ptr(similar), _ptr(partials)),
+                 "sfb_forward_partials_pairs")
 
     def sfb_finish_factors(self, partials_all, shards):
         """partials_all: fp32 CUDA tensor [shards, K, 4], the partials of every shard in shard order."""

@@ -183,7 +183,7 @@ extern "C" int sfb_destroy(sfb_ctx* ctx) {
 // fp32-operand path
 // ---------------------------------------------------------------------------------------------------------
 static int factors_fp32(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float* Y,
-                        const int32_t* labels, bool sparse_fwd = false) {
+                        const int32_t* labels, bool sparse_fwd = false, float* dml_norm_out = nullptr) {
   const sfb_config& c = ctx->cfg;
   const int64_t rows = c.rows, cols = c.cols;
   float* V = ctx->at<float>(ctx->lay.V) + off * cols;
@@ -205,7 +205,7 @@ static int factors_fp32(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, co
     if (c.model == SFB_MLR)
       CK(mlr_softmax_rows(s, U, n, rows, labels, ctx->at<float>(ctx->lay.loss) + off, status));
     else
-      CK(dml_scale_rows(s, U, n, rows, rows, labels, c.dml_margin));
+      CK(dml_scale_rows(s, U, n, rows, rows, labels, c.dml_margin, nullptr, dml_norm_out));
     return SFB_OK;
   }
   // sparse coding: ISTA from a = 0, then u = W a - x, v = a
@@ -329,7 +329,7 @@ extern "C" int sfb_step_csr(sfb_ctx* ctx, const int64_t* indptr_dev, const int32
 // ---------------------------------------------------------------------------------------------------------
 extern "C" int sfb_set_row_shard(sfb_ctx* ctx, int64_t row_offset, int64_t global_rows) {
   if (!ctx) return SFB_ERR_ARG;
-  if (ctx->cfg.model != SFB_MLR || ctx->sdca) return SFB_ERR_UNSUPPORTED;
+  if ((ctx->cfg.model != SFB_MLR && ctx->cfg.model != SFB_DML) || ctx->sdca) return SFB_ERR_UNSUPPORTED;
   if (row_offset < 0 || global_rows < row_offset + ctx->cfg.rows || global_rows > (1LL << 31) - 1) return SFB_ERR_SHAPE;
   if (ctx->committed != 0 || ctx->partials_ready) return SFB_ERR_STATE;
   ctx->row_offset = row_offset;
@@ -372,13 +372,45 @@ extern "C" int sfb_forward_partials(sfb_ctx* ctx, const float* X_dev, const int3
   return SFB_OK;
 }
 
+// DML by rows: z = W v splits over the shards, the hinge needs ||z||^2 = sum over the shards of ||z_shard||^2.
+extern "C" int sfb_forward_partials_pairs(sfb_ctx* ctx, const float* X_dev, const float* Y_dev, const int32_t* similar_dev,
+                                          float* partials_dev) {
+  int rc = check_inputs(ctx, X_dev, Y_dev, similar_dev);
+  if (rc) return rc;
+  if (ctx->cfg.model != SFB_DML) return SFB_ERR_UNSUPPORTED;
+  if (!partials_dev) return SFB_ERR_ARG;
+  const sfb_config& c = ctx->cfg;
+  ctx->committed = 0;
+  ctx->sparse_mask = 0;
+  ctx->csr_fill = 0;
+  ctx->gathered = false;
+  CK(cudaEventRecord(ctx->ev[0], ctx->stream));
+  // the flags are kept for the finish (the caller's buffer may change before it)
+  CK(cudaMemcpyAsync(ctx->at<int32_t>(ctx->lay.stageL), similar_dev, static_cast<size_t>(ctx->K) * 4, cudaMemcpyDeviceToDevice,
+                     ctx->stream));
+  rc = c.precision == SFB_PREC_FP32 ? factors_fp32(ctx, 0, ctx->K, X_dev, Y_dev, similar_dev, false, partials_dev)
+                                    : tc_factors(ctx, 0, ctx->K, X_dev, Y_dev, similar_dev, partials_dev);
+  if (rc) return rc;
+  ctx->partials_ready = true;
+  return SFB_OK;
+}
+
 extern "C" int sfb_finish_factors(sfb_ctx* ctx, const float* partials_all_dev, int32_t shards) {
   if (!ctx || !partials_all_dev) return SFB_ERR_ARG;
-  if (ctx->cfg.model != SFB_MLR) return SFB_ERR_UNSUPPORTED;
+  if (ctx->cfg.model != SFB_MLR && ctx->cfg.model != SFB_DML) return SFB_ERR_UNSUPPORTED;
   if (shards < 1 || shards > 4096) return SFB_ERR_ARG;
   if (!al16(partials_all_dev)) return SFB_ERR_ALIGN;
   if (!ctx->partials_ready) return SFB_ERR_STATE;
   const sfb_config& c = ctx->cfg;
+  if (c.model == SFB_DML) {
+    const int64_t ldu = c.precision == SFB_PREC_FP32 ? c.rows : ctx->lay.ldu;
+    CK(dml_scale_rows(ctx->stream, ctx->at<float>(ctx->lay.U), ctx->K, c.rows, ldu, ctx->at<int32_t>(ctx->lay.stageL),
+                      c.dml_margin, nullptr, nullptr, partials_all_dev, shards, ctx->K));
+    ctx->partials_ready = false;
+    ctx->committed = c.workers == 64 ? ~0ull : ((1ull << c.workers) - 1);
+    ctx->gathered = false;
+    return SFB_OK;
+  }
   if (c.precision == SFB_PREC_BF16 || ctx->tf32) {
     const int rc = ctx->tf32 ? tc32_finish_factors(ctx, partials_all_dev, shards)
                              : tc_finish_factors(ctx, partials_all_dev, shards);

@@ -277,10 +277,14 @@ __global__ void __launch_bounds__(NTHREADS) sdca_dual_kernel(float* __restrict__
 }
 
 // One block per pair: q = ||z||^2; similar: u = 2z; dissimilar: u = -2z if q < margin else 0 (Section 2, DML).
+// Row-sharded form: with norm_out the block only stores its shard's q (after merging Z2) and leaves z as it is; with
+// norms_all it takes q as the sum, in shard order, of the shards' values and scales.
 template <int NTHREADS>
 __global__ void __launch_bounds__(NTHREADS) dml_scale_kernel(float* __restrict__ Z, const float* __restrict__ Z2,
                                                              int64_t rows, int64_t ld,
-                                                             const int32_t* __restrict__ similar, float margin) {
+                                                             const int32_t* __restrict__ similar, float margin,
+                                                             float* __restrict__ norm_out, const float* __restrict__ norms_all,
+                                                             int shards, int64_t nstride) {
   __shared__ float sh[32];
   float* z = Z + static_cast<int64_t>(blockIdx.x) * ld;
   if (Z2) {                      // z arrives as two partial sums over halves of the contraction (fixed order: Z + Z2)
@@ -289,8 +293,16 @@ __global__ void __launch_bounds__(NTHREADS) dml_scale_kernel(float* __restrict__
     __syncthreads();
   }
   float q = 0.f;
-  for (int64_t j = threadIdx.x; j < rows; j += NTHREADS) q = fmaf(z[j], z[j], q);
-  q = block_sum<NTHREADS>(q, sh);
+  if (norms_all) {
+    for (int g = 0; g < shards; ++g) q += norms_all[g * nstride + blockIdx.x];
+  } else {
+    for (int64_t j = threadIdx.x; j < rows; j += NTHREADS) q = fmaf(z[j], z[j], q);
+    q = block_sum<NTHREADS>(q, sh);
+  }
+  if (norm_out) {
+    if (threadIdx.x == 0) norm_out[blockIdx.x] = q;
+    return;
+  }
   const float c = similar[blockIdx.x] != 0 ? 2.f : (q < margin ? -2.f : 0.f);
   for (int64_t j = threadIdx.x; j < rows; j += NTHREADS) z[j] = c * z[j];
 }
@@ -529,9 +541,11 @@ cudaError_t sdca_dual_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows
 }
 
 cudaError_t dml_scale_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows, int64_t ld,
-                           const int32_t* similar, float margin, const float* Z2) {
+                           const int32_t* similar, float margin, const float* Z2, float* norm_out, const float* norms_all,
+                           int shards, int64_t nstride) {
   if (nsamp <= 0) return cudaSuccess;
-  dml_scale_kernel<256><<<static_cast<unsigned>(nsamp), 256, 0, s>>>(Z, Z2, rows, ld, similar, margin);
+  dml_scale_kernel<256><<<static_cast<unsigned>(nsamp), 256, 0, s>>>(Z, Z2, rows, ld, similar, margin, norm_out, norms_all,
+                                                                     shards, nstride);
   count_launch();
   return cudaGetLastError();
 }

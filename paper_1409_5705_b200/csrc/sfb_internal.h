@@ -145,9 +145,12 @@ cudaError_t mlr_shard_finish(cudaStream_t s, float* Z, int64_t nsamp, int64_t ro
 cudaError_t sdca_dual_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows, int64_t ldz, const float* X, int64_t cols,
                            const int32_t* labels, const int32_t* ids, float* Q, int64_t n_samples, float inv_lam_n,
                            float gamma, float* coef, float* loss, uint32_t* status);
-// Z2 (may be null): a second partial of z (the other half of the contraction), added to Z first.
+// Z2 (may be null): a second partial of z (the other half of the contraction), added to Z first.  Row-sharded form:
+// norm_out (may be null) receives the shard's ||z_i||^2 and z is left unscaled; norms_all (may be null), [shards][nstride],
+// supplies ||z_i||^2 as the sum over the shards instead of this context's own.
 cudaError_t dml_scale_rows(cudaStream_t s, float* Z, int64_t nsamp, int64_t rows, int64_t ld,
-                           const int32_t* similar, float margin, const float* Z2 = nullptr);
+                           const int32_t* similar, float margin, const float* Z2 = nullptr, float* norm_out = nullptr,
+                           const float* norms_all = nullptr, int shards = 0, int64_t nstride = 0);
 cudaError_t mean_of(cudaStream_t s, const float* v, int64_t n, float* out);
 cudaError_t prox_unit_columns(cudaStream_t s, float* W, int64_t rows, int64_t cols, float* colpart);
 cudaError_t estimate_lipschitz(cudaStream_t s, const float* W, int64_t rows, int64_t cols, float* b, float* y,

@@ -1051,7 +1051,8 @@ int split_product(sfb_ctx* ctx, int64_t off, int64_t n, __nv_bfloat16* A, __nv_b
 // Sufficient factors of distance metric learning and sparse coding in bf16 mode: the same steps as the fp32
 // path (Section 2: z = W v with v = x - y; Figure 3: ISTA codes, u = W a - x), every product on the tensor cores
 // with (hi | lo) bf16 operands.
-int factors_split(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float* Y, const int32_t* labels) {
+int factors_split(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float* Y, const int32_t* labels,
+                  float* dml_norm_out = nullptr) {
   const sfb_config& c = ctx->cfg;
   const Layout& L = ctx->lay;
   const int64_t rows = c.rows, cols = c.cols;
@@ -1082,7 +1083,8 @@ int factors_split(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const fl
     int parts = 1;
     int rc = split_product<F_STORE>(ctx, off, n, As, Ws, rows, L.colsp, U, L.ldu, p, U2 - U, &parts);   // z_i = W v_i
     if (rc) return rc;
-    CKC(dml_scale_rows(s, U + off * L.ldu, n, rows, L.ldu, labels, c.dml_margin, parts > 1 ? U2 + off * L.ldu : nullptr));
+    CKC(dml_scale_rows(s, U + off * L.ldu, n, rows, L.ldu, labels, c.dml_margin, parts > 1 ? U2 + off * L.ldu : nullptr,
+                       dml_norm_out));
     return SFB_OK;
   }
   // sparse coding: ISTA from a = 0, then u = W a - x, v = a
@@ -1406,8 +1408,9 @@ int tc_sdca_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const 
   return SFB_OK;
 }
 
-int tc_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float* Y, const int32_t* labels) {
-  if (ctx->cfg.model != SFB_MLR) return factors_split(ctx, off, n, X, Y, labels);
+int tc_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float* Y, const int32_t* labels,
+               float* dml_norm_out) {
+  if (ctx->cfg.model != SFB_MLR) return factors_split(ctx, off, n, X, Y, labels, dml_norm_out);
   const sfb_config& c = ctx->cfg;
   const Layout& L = ctx->lay;
   const int64_t rows = c.rows, K = ctx->K;

@@ -21,7 +21,9 @@ int tc_init(sfb_ctx* ctx);
 void tc_destroy(sfb_ctx* ctx);
 // Rebuilds the bf16 operand copy of W from the caller's fp32 W (MLR; the other models rebuild theirs every step).
 int tc_refresh_operands(sfb_ctx* ctx);
-int tc_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float* Y, const int32_t* labels);
+// dml_norm_out (DML, row-sharded form; may be null): receives ||z_i||^2 of this context's rows and z stays unscaled.
+int tc_factors(sfb_ctx* ctx, int64_t off, int64_t n, const float* X, const float* Y, const int32_t* labels,
+               float* dml_norm_out = nullptr);
 // Row-sharded MLR: logits and softmax partials of all K samples against this context's rows; then the factors from
 // the partials of all shards.
 int tc_forward_partials(sfb_ctx* ctx, const float* X, const int32_t* labels, float* part_out);

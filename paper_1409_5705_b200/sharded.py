@@ -59,26 +59,38 @@ def exchange_model_bytes(P: int, B: int, rows: int, cols: int, shards: int) -> d
     }
 
 
-def sharded_step(ctx, X_local, labels_local, partials, partials_all, X_all, labels_all, group=None, dist=None):
+def sharded_step(ctx, X_local, labels_local, partials, partials_all, X_all, labels_all, group=None, dist=None,
+                 Y_local=None, Y_all=None):
     """One row-sharded step on this rank.
 
     ctx            a context over this rank's rows, already told its shard with ``sfb_set_row_shard``
-    X_local        [K/shards, cols] this rank's samples; labels_local [K/shards] their (global) class ids
-    partials       [K, 4] scratch for this rank's partials;  partials_all  [shards, K, 4]
+    X_local        [K/shards, cols] this rank's samples; labels_local [K/shards] their (global) class ids (MLR) or
+                   similar / dissimilar flags (DML)
+    partials       scratch for this rank's partials, [K, 4] (MLR) or [K, 1] (DML);  partials_all  [shards, K, 4 | 1]
     X_all          [K, cols] and labels_all [K]: receive the gathered samples (rank-major = worker-major order)
+    Y_local, Y_all DML only: the pair partners, gathered like the samples
     dist           the ``torch.distributed`` module (or a stand-in with the same two calls); None: single shard
     Returns the ExchangeBytes of the step.
     """
     moved = ExchangeBytes()
+    pairs = Y_local is not None
     if dist is None:
         X_all.copy_(X_local)
         labels_all.copy_(labels_local)
+        if pairs:
+            Y_all.copy_(Y_local)
     else:
         dist.all_gather_into_tensor(X_all, X_local, group=group)
         dist.all_gather_into_tensor(labels_all, labels_local, group=group)
         moved.samples = (X_all.numel() - X_local.numel()) * X_all.element_size() + \
                         (labels_all.numel() - labels_local.numel()) * labels_all.element_size()
-    ctx.sfb_forward_partials(X_all, labels_all, partials)
+        if pairs:
+            dist.all_gather_into_tensor(Y_all, Y_local, group=group)
+            moved.samples += (Y_all.numel() - Y_local.numel()) * Y_all.element_size()
+    if pairs:
+        ctx.sfb_forward_partials_pairs(X_all, Y_all, labels_all, partials)
+    else:
+        ctx.sfb_forward_partials(X_all, labels_all, partials)
     if dist is None:
         partials_all.view(-1).copy_(partials.view(-1))
     else:

@@ -144,7 +144,7 @@ def test_row_shard_call_order_and_argument_errors():
     ctx.sfb_finish_factors(parts, 1)
     assert ctx.sfb_get_status() & S.STATUS_LABEL_RANGE
     ctx.close()
-    wd = I.scaled(I.WORKLOADS["dml"], "d", rows=64, cols=64, workers=1, batch=8)
+    wd = I.scaled(I.WORKLOADS["sc"], "d", rows=64, cols=64, workers=1, batch=8)
     Wd = to_dev(I.initial_W(wd), torch)
     cd = S.Context(config_for(wd, S.PREC_FP32), Wd)
     with pytest.raises(S.SfbError) as e:
@@ -218,3 +218,57 @@ def test_a_shard_that_owns_no_class_of_the_batch():
         assert rel_err(W, ref, W0) <= TOL[prec]
         assert parts[0, :, 3].sum() == wl.K and parts[1:, :, 3].sum() == 0
         assert np.abs(W[111:] - W0[111:]).max() > 0            # the other shards' rows moved too
+
+
+@pytest.mark.parametrize("G", [1, 2, 3])
+@pytest.mark.parametrize("prec", [pytest.param(S.PREC_FP32, id="fp32"), pytest.param(S.PREC_BF16, id="bf16")])
+def test_dml_row_shards_match_the_unsharded_oracle_step(prec, G):
+    """DML with the latent rows of W dealt to G contexts: every shard computes its part of z = W (x - y) and its
+    partial ||z||^2, the partials are exchanged (here through one device buffer), every shard decides the hinge on the
+    summed norm and updates its rows.  Both hinge branches occur in the batch."""
+    from paper_1409_5705_b200.sharded import sharded_step
+    wl = I.scaled(I.WORKLOADS["dml"], "dml_shard", rows=150, cols=388, workers=4, batch=33, eta=1e-3)
+    W0 = I.initial_W(wl)
+    inp = I.step_inputs(wl, 0)
+    zq = ((inp.X - inp.Y).astype(np.float64) @ W0.astype(np.float64).T)
+    # the margin near the median norm of the dissimilar pairs: about half of them inside the hinge, half outside
+    qs = np.sort((zq * zq).sum(axis=1)[inp.labels == 0])
+    mid = len(qs) // 2
+    k = max(range(mid - 5, mid + 5), key=lambda t: qs[t + 1] - qs[t])          # the widest gap near the middle: no pair
+    wl = I.scaled(wl, "dml_shard_m", dml_margin=float(0.5 * (qs[k] + qs[k + 1])))    # sits on the margin itself
+    ref = oracle_step(wl, W0, inp)
+    K = wl.K
+    X, Y, lab = to_dev(inp.X, torch), to_dev(inp.Y, torch), to_dev(inp.labels, torch)
+    parts_all = torch.zeros((G, K, 1), dtype=torch.float32, device="cuda")
+    shards = []
+    for g in range(G):
+        r0, r1 = row_shard_bounds(wl.rows, G, g)
+        Wg = to_dev(W0[r0:r1], torch)
+        cfg = S.make_config(S.DML, r1 - r0, wl.cols, wl.workers, wl.batch, wl.eta, prec, dml_margin=wl.dml_margin)
+        ctx = S.Context(cfg, Wg)
+        ctx.sfb_set_row_shard(r0, wl.rows)
+        ctx.sfb_forward_partials_pairs(X, Y, lab, parts_all[g])
+        shards.append((ctx, Wg))
+    q = parts_all.sum(dim=0).view(-1).cpu().numpy()
+    assert np.allclose(q, (zq * zq).sum(axis=1), rtol=2e-3 if prec == S.PREC_BF16 else 1e-5)
+    inside = (zq * zq).sum(axis=1) < wl.dml_margin
+    assert inside[inp.labels == 0].any() and (~inside[inp.labels == 0]).any()      # both branches of the hinge
+    for ctx, _ in shards:
+        ctx.sfb_finish_factors(parts_all, G)
+        ctx.sfb_gather_factors()
+        ctx.sfb_apply_update()
+        assert ctx.sfb_get_status() == 0
+    Wsh = np.concatenate([w.cpu().numpy() for _, w in shards], axis=0)
+    for ctx, _ in shards:
+        ctx.close()
+    err = rel_err(Wsh, ref, W0)
+    print(f"dml {G} shards: rel err {err:.3e} (tol {TOL[prec]})")
+    assert err <= TOL[prec]
+    if G == 1:                                             # the helper on a single shard gives the same step
+        W = to_dev(W0, torch)
+        ctx = S.Context(S.make_config(S.DML, wl.rows, wl.cols, wl.workers, wl.batch, wl.eta, prec, dml_margin=wl.dml_margin), W)
+        ctx.sfb_set_row_shard(0, wl.rows)
+        part = torch.zeros((K, 1), dtype=torch.float32, device="cuda")
+        sharded_step(ctx, X, lab, part, parts_all, torch.empty_like(X), torch.empty_like(lab), Y_local=Y, Y_all=torch.empty_like(Y))
+        assert np.array_equal(W.cpu().numpy(), Wsh)
+        ctx.close()

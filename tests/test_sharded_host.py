@@ -226,3 +226,76 @@ def test_two_gloo_ranks_keep_identical_replicas_equal_to_the_oracle_step(tmp_pat
     R0, R1 = np.load(tmp_path / "R0.npy"), np.load(tmp_path / "R1.npy")
     assert np.array_equal(R0, R1)
     assert np.linalg.norm(R0 - ref) <= 1e-12 * np.linalg.norm(ref - W0)
+
+
+class _FakeDmlShard:
+    """The DML calls of one row shard in numpy fp64 (a test double): partial squared norms, hinge on their sum."""
+
+    def __init__(self, W_shard, eta, margin):
+        self.W = W_shard.astype(np.float64)
+        self.eta, self.margin = eta, margin
+
+    def sfb_forward_partials_pairs(self, X_all, Y_all, similar_all, partials):
+        self.v = (X_all.numpy() - Y_all.numpy()).astype(np.float64)
+        self.sim = similar_all.numpy()
+        self.z = self.v @ self.W.T
+        partials.copy_(torch.from_numpy((self.z * self.z).sum(axis=1, keepdims=True)))
+
+    def sfb_finish_factors(self, partials_all, shards):
+        q = partials_all.numpy().astype(np.float64).sum(axis=0)[:, 0]
+        c = np.where(self.sim != 0, 2.0, np.where(q < self.margin, -2.0, 0.0))
+        self.u = c[:, None] * self.z
+
+    def sfb_gather_factors(self):
+        pass
+
+    def sfb_apply_update(self):
+        self.W -= self.eta * (self.u.T @ self.v)
+
+
+def _dml_workload():
+    import sfb_inputs as I
+    return I.scaled(I.WORKLOADS["dml"], "dml_gloo", rows=14, cols=20, workers=4, batch=5, eta=1e-2, dml_margin=0.8)
+
+
+def _dml_rank(rank, world, port, out_dir):
+    import torch.distributed as dist
+    sys.path.insert(0, ROOT)
+    import sfb_inputs as I
+    from paper_1409_5705_b200.sharded import row_shard_bounds, sharded_step
+    dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=rank, world_size=world)
+    wl = _dml_workload()
+    W0 = I.initial_W(wl)
+    inp = I.step_inputs(wl, 0)
+    K, n = wl.K, wl.K // world
+    r0, r1 = row_shard_bounds(wl.rows, world, rank)
+    ctx = _FakeDmlShard(W0[r0:r1], wl.eta, wl.dml_margin)
+    sl = slice(rank * n, (rank + 1) * n)
+    f64 = lambda a: torch.from_numpy(a.astype(np.float64))
+    partials = torch.zeros((K, 1), dtype=torch.float64)
+    partials_all = torch.zeros((world, K, 1), dtype=torch.float64)
+    X_all, Y_all = torch.zeros((K, wl.cols), dtype=torch.float64), torch.zeros((K, wl.cols), dtype=torch.float64)
+    s_all = torch.zeros((K,), dtype=torch.int32)
+    moved = sharded_step(ctx, f64(inp.X[sl]), torch.from_numpy(inp.labels[sl]), partials, partials_all, X_all, s_all, dist=dist,
+                         Y_local=f64(inp.Y[sl]), Y_all=Y_all)
+    np.save(os.path.join(out_dir, f"D{rank}.npy"), ctx.W)
+    assert moved.samples == 2 * (K - n) * wl.cols * 8 + (K - n) * 4 and moved.partials == K * 8
+    assert np.array_equal(Y_all.numpy(), inp.Y.astype(np.float64))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_step_dml_row_shards_to_the_oracle_result(tmp_path):
+    import torch.multiprocessing as mp
+    sys.path.insert(0, ROOT)
+    import sfb_inputs as I
+    from oracle import sfb_oracle as O
+    port = 33500 + os.getpid() % 2000
+    mp.spawn(_dml_rank, args=(2, port, str(tmp_path)), nprocs=2, join=True)
+    wl = _dml_workload()
+    W0 = I.initial_W(wl)
+    inp = I.step_inputs(wl, 0)
+    ref = O.sfb_step(O.DML, W0, inp.X, inp.Y, inp.labels, workers=wl.workers, eta=wl.eta, margin=wl.dml_margin)
+    W = np.concatenate([np.load(tmp_path / f"D{r}.npy") for r in range(2)], axis=0)
+    assert np.linalg.norm(W - ref) <= 1e-12 * np.linalg.norm(ref - W0)
+    assert np.linalg.norm(ref - W0) > 0
