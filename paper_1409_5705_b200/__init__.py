@@ -206,7 +206,7 @@ class Context:
                                                _ptr(labels)), "sfb_compute_factors_csr")
 
     def sfb_step_csr(self, indptr, indices, values, nnz, labels):
-        self._ck(lib().sfb_step_csr(self._h, _ptr(indptr), _ptr(indices), _ptr(values), nnz, _ptr(labels)), "sfb_step_csr", "sfb_export_factors", "sfb_forward_partials_pairs")
+        self._ck(lib().sfb_step_csr(self._h, _ptr(indptr), _ptr(indices), _ptr(values), nnz, _ptr(labels)), "sfb_step_csr")
 
     def sfb_step_host(self, X, Y=None, labels=None):
         """X, Y, labels: host tensors / numpy arrays (pinned recommended).  Returns (mean loss, status word)."""
