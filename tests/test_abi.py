@@ -50,3 +50,21 @@ def test_struct_layouts_match_the_header():
         subprocess.check_call(["gcc", "-I" + os.path.join(ROOT, "include"), c, "-o", exe])
         a, b = map(int, subprocess.check_output([exe]).split())
     assert a == ctypes.sizeof(S.sfb_config) and b == ctypes.sizeof(S.sfb_stats)
+
+
+def test_binding_error_checks_name_the_call_they_wrap():
+    """Every ``self._ck(lib().sfb_x(...), "sfb_x")`` in the binding passes exactly the return code and the name of the
+    entry point it called (a slip here only shows when that method runs on a GPU)."""
+    import ast
+    import os
+    src = open(os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "paper_1409_5705_b200",
+                            "__init__.py")).read()
+    seen = 0
+    for node in ast.walk(ast.parse(src)):
+        if isinstance(node, ast.Call) and isinstance(node.func, ast.Attribute) and node.func.attr == "_ck":
+            assert len(node.args) == 2 and not node.keywords, ast.unparse(node)
+            call, name = node.args
+            assert isinstance(name, ast.Constant) and isinstance(call, ast.Call) and isinstance(call.func, ast.Attribute)
+            assert call.func.attr == name.value, ast.unparse(node)
+            seen += 1
+    assert seen >= 25
